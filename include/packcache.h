@@ -1,0 +1,176 @@
+/*
+ * packcache.h — C ABI of the PackCache hot path on one B200 (sm_100a).
+ *
+ * The library keeps a video generator's KV cache small and runs the current
+ * frame's attention over it: text and conditioning-image tokens ("anchors") are
+ * always kept, every earlier frame keeps a number of tokens that shrinks with
+ * its temporal distance, and kept tokens carry their original (t, h, w)
+ * coordinates so that 3D rotary attention stays spatially coherent (paper
+ * Sec. 3.4; attention is Eq. 2 of Sec. 3.1).
+ *
+ * Conventions
+ *  - Plain C, no CUDA types: a stream is passed as void* (a cudaStream_t; NULL
+ *    is the default stream).
+ *  - Pointers marked "device" are device memory owned by the caller and must be
+ *    16-byte aligned; pointers marked "host" are ordinary host memory, read
+ *    before the call returns.  The library never frees or keeps caller memory.
+ *    It owns only the context (rotary tables, a status word, scratch sized at
+ *    pc_create from the limits in pc_layer_desc).
+ *  - Layout is token-major: K/V [token][kv_head][head_dim], Q/O
+ *    [token][q_head][head_dim], pos [token][4] int32 = (t, h, w, tag) holding
+ *    already scaled integer coordinates (MM-RoPE scales latent coordinates by
+ *    (4, 8, 8), Sec. 3.1) and an opaque tag that compaction copies unchanged.
+ *    Element type is pc_layer_desc.dtype for K, V, Q and O.
+ *  - Errors the host can see (bad arguments, budgets, capacities) are returned
+ *    at once and nothing is enqueued.  Device work is asynchronous on the given
+ *    stream.  A kernel that meets a bad index, an out-of-table position or a
+ *    wait that ran out records the first such event in the context's status
+ *    word, skips the access and finishes; pc_poll_status returns it.
+ *  - Calls on one context must be issued from one host thread at a time, and
+ *    calls that share a context's scratch must be ordered on the GPU (same
+ *    stream or explicit dependencies).
+ */
+#ifndef PACKCACHE_H
+#define PACKCACHE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PC_OK = 0,
+    PC_ERR_INVALID_ARG = 1, /* null / misaligned pointer, bad size, position outside the rotary tables */
+    PC_ERR_BUDGET = 2,      /* a frame's budget exceeds its tokens, or kept-whole frames exceed the total */
+    PC_ERR_CAPACITY = 3,    /* destination segment or context scratch too small */
+    PC_ERR_UNSUPPORTED = 4, /* head_dim not 64/128, heads not divisible, dtype unknown */
+    PC_ERR_CUDA = 5,        /* a CUDA runtime call failed */
+    PC_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up */
+} pc_status;
+
+enum { PC_F32 = 0, PC_BF16 = 1 };
+
+/* decay kernels g(dist), dist = 1 for the most recent history frame (Eq. 5-7) */
+enum {
+    PC_GEOMETRIC = 0,   /* g = param^dist, 0 < param < 1 (Eq. 5) */
+    PC_CLOSED_HALF = 1, /* g = 2^-min(dist, W-1), the deployed closed form (Eq. 7) */
+    PC_LINEAR = 2,      /* g = W + 1 - dist */
+    PC_HALFLIFE = 3     /* g = 2^-((dist - 1 - keep_full) / param), param = half-life in frames */
+};
+
+#define PC_MAX_FRAMES 256 /* most history frames one pc_score call accepts */
+
+typedef struct pc_ctx pc_ctx;
+
+typedef struct {
+    int32_t n_q_heads;  /* Hq */
+    int32_t n_kv_heads; /* Hkv, divides Hq (grouped-query attention) */
+    int32_t head_dim;   /* 64 or 128 */
+    int32_t dtype;      /* PC_F32 or PC_BF16: storage type of Q, K, V, O */
+    double rope_base;   /* rotary base, e.g. 10000 */
+    int32_t max_pos[3]; /* exclusive upper bound of t, h, w: extents of the rotary tables */
+    int32_t max_q;      /* most query tokens in one call */
+    int32_t max_keys;   /* most keys attended in one call (anchors + history + current), and most
+                           history tokens scored in one call */
+} pc_layer_desc;
+
+/* A run of tokens: anchors, history, or the frame being generated. */
+typedef struct {
+    void *k;          /* device [capacity][Hkv][d] */
+    void *v;          /* device [capacity][Hkv][d] */
+    int32_t *pos;     /* device [capacity][4] */
+    int32_t n_tokens; /* tokens in use */
+    int32_t capacity; /* tokens allocated */
+} pc_segment;
+
+/* The cache C_t of Sec. 3.4: anchors held apart from the decayed history. */
+typedef struct {
+    pc_segment anchors;         /* [text | conditioning image]; never moved, never scored */
+    pc_segment history;         /* history frames, oldest -> newest, contiguous */
+    int32_t n_frames;           /* history frames */
+    const int32_t *frame_count; /* host [n_frames]: tokens of each frame; sums to history.n_tokens */
+} pc_cache;
+
+typedef struct {
+    int32_t kind;      /* PC_GEOMETRIC ... PC_HALFLIFE */
+    double param;      /* rho or half-life, see the enum */
+    int64_t total;     /* history tokens to retain in all, anchors not counted (B_one of Eq. 8) */
+    int32_t keep_full; /* most recent frames kept whole (counted inside total) */
+    int32_t min_quota; /* reserved (minimum per-frame quota b_min); must be 0 */
+} pc_budget_params;
+
+/* Create / destroy a context on the current CUDA device.  Builds the rotary
+ * cos/sin tables (Sec. 3.1: pair i of d/2 turns with axis i mod 3 at frequency
+ * base^(-(i div 3)/n_axis)) and allocates scratch for max_q / max_keys.
+ * Errors: PC_ERR_UNSUPPORTED, PC_ERR_INVALID_ARG, PC_ERR_CUDA. */
+pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out);
+pc_status pc_destroy(pc_ctx *ctx);
+
+/* Per-frame token budgets (Sec. 3.4, Eq. 5-8; anchors are excluded from the
+ * decay and always kept).  Host only, integers after one quantisation of the
+ * weights to 2^-32: the keep_full newest frames keep everything; the rest of
+ * `total` is shared in proportion to g(dist) by largest remainder (ties to the
+ * nearer frame); a frame granted more than avail keeps avail and the surplus is
+ * re-shared.  avail and budget are host arrays [n_frames], oldest -> newest.
+ * The result sums to min(total, sum(avail)).
+ * Errors: PC_ERR_INVALID_ARG (null, negative, bad param, min_quota != 0),
+ * PC_ERR_BUDGET (kept-whole frames exceed total). */
+pc_status pc_plan_budget(const pc_budget_params *params, int32_t n_frames, const int32_t *avail,
+                         int32_t *budget);
+
+/* Score every history token and pick each frame's budget[f] best (Sec. 3.4,
+ * "attention-relevant" retention).  score_j = mean over the n_q queries and all
+ * query heads of the scaled rotary logit (R q).(R k_j)/sqrt(d), computed in
+ * fp32 through a pooled query.  Per frame the budget[f] highest scores are
+ * kept, equal scores by lower index (-0 == +0), and written to sel_idx as
+ * ascending global history indices, frames oldest -> newest.
+ *   q device [n_q][Hq][d]; q_pos device [n_q][4]; budget host [n_frames];
+ *   valid device [n_src] bytes or NULL (0 = masked cache position, Eq. 1: never
+ *   kept unless the budget exceeds the valid tokens);
+ *   scores_override device [n_src] fp32 or NULL: skip scoring, select on these;
+ *   scores device out [n_src] fp32 (may be NULL with an override);
+ *   sel_idx device out [sum(budget)].
+ * Errors: PC_ERR_INVALID_ARG, PC_ERR_BUDGET (budget[f] > frame_count[f]),
+ * PC_ERR_CAPACITY (n_src > max_keys, n_q > max_q, n_frames > PC_MAX_FRAMES). */
+pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q,
+                   const int32_t *budget, const uint8_t *valid, const float *scores_override,
+                   float *scores, int32_t *sel_idx, void *stream);
+
+/* Pack the selected rows into dst (Fig. 6b: evicted positions are removed, not
+ * zero-filled) with the spatially preserving rebase (Eq. 9): dst history row r
+ * is src history row sel_idx[r]; K, V, (h, w, tag) are bit copies, t has
+ * delta_t subtracted.  dst.history.n_tokens / n_frames are set by the caller to
+ * sum(budget) / src.n_frames; dst anchors are not touched (anchors never move).
+ *   sel_idx device [sum(budget)]; budget host [src.n_frames].
+ * Errors: PC_ERR_INVALID_ARG (dst aliases src, null), PC_ERR_BUDGET,
+ * PC_ERR_CAPACITY (sum(budget) > dst.history.capacity). */
+pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget,
+                     int32_t delta_t, pc_cache *dst, void *stream);
+
+/* Attention of the current frame's queries over anchors ++ history ++ current
+ * (Eq. 2; a whole-frame query block sees every cached key, so no mask is left):
+ *   out[i][h] = softmax_j((R q_ih).(R k_j,g)/sqrt(d)) v_j,g,  g = h / (Hq/Hkv).
+ * Rotary embedding is applied from the stored positions inside the call.
+ *   current may be NULL; q device [n_q][Hq][d]; out device [n_q][Hq][d];
+ *   lse device [n_q][Hq] fp32 natural-log sum of exponentials, or NULL.
+ * bf16 runs on tcgen05 tensor cores (fp32 accumulate and softmax); fp32 runs on
+ * CUDA cores.  Errors: PC_ERR_INVALID_ARG, PC_ERR_CAPACITY (keys > max_keys,
+ * n_q > max_q), PC_ERR_CUDA. */
+pc_status pc_attend_frame(pc_ctx *ctx, const pc_cache *cache, const pc_segment *current, const void *q,
+                          const int32_t *q_pos, int32_t n_q, void *out, float *lse, void *stream);
+
+/* Wait for the stream, then return and clear the first device-side event
+ * recorded since the last poll (PC_OK if none). */
+pc_status pc_poll_status(pc_ctx *ctx, void *stream);
+
+/* Choose the bf16 attention kernel: 0 = tcgen05 tensor-core kernel (default),
+ * 1 = CUDA-core kernel (a slow second opinion).  Returns PC_ERR_INVALID_ARG otherwise. */
+pc_status pc_set_attend_impl(pc_ctx *ctx, int32_t impl);
+
+const char *pc_status_string(pc_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PACKCACHE_H */

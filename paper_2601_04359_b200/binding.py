@@ -1,0 +1,221 @@
+"""ctypes binding of ``libpackcache.so`` — same names as the C ABI, argument marshalling only.
+
+Every step of the path (scoring, selection, packing, rotary embedding, attention) runs in the library's CUDA
+kernels; PyTorch is used here for device memory and streams.  There is no CPU fallback: if the library cannot be
+loaded, importing callers get an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+PC_OK, PC_ERR_INVALID_ARG, PC_ERR_BUDGET, PC_ERR_CAPACITY, PC_ERR_UNSUPPORTED, PC_ERR_CUDA, PC_ERR_TIMEOUT = range(7)
+PC_F32, PC_BF16 = 0, 1
+PC_GEOMETRIC, PC_CLOSED_HALF, PC_LINEAR, PC_HALFLIFE = 0, 1, 2, 3
+PC_MAX_FRAMES = 256
+
+EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact", "pc_attend_frame",
+           "pc_poll_status", "pc_set_attend_impl", "pc_status_string"]
+
+
+class pc_layer_desc(C.Structure):
+    _fields_ = [("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("dtype", C.c_int32),
+                ("rope_base", C.c_double), ("max_pos", C.c_int32 * 3), ("max_q", C.c_int32), ("max_keys", C.c_int32)]
+
+
+class pc_segment(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("pos", C.c_void_p), ("n_tokens", C.c_int32),
+                ("capacity", C.c_int32)]
+
+
+class pc_cache(C.Structure):
+    _fields_ = [("anchors", pc_segment), ("history", pc_segment), ("n_frames", C.c_int32),
+                ("frame_count", C.POINTER(C.c_int32))]
+
+
+class pc_budget_params(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("param", C.c_double), ("total", C.c_int64), ("keep_full", C.c_int32),
+                ("min_quota", C.c_int32)]
+
+
+class PackCacheError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        msg = _lib.pc_status_string(status).decode() if _lib is not None else str(status)
+        super().__init__(f"{what}: {msg} (pc_status {status})")
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load the CUDA library (building it with nvcc if the .so is absent).  Raises if that is impossible."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = C.CDLL(path)
+    lib.pc_status_string.restype = C.c_char_p
+    lib.pc_status_string.argtypes = [C.c_int]
+    lib.pc_create.argtypes = [C.POINTER(pc_layer_desc), C.POINTER(C.c_void_p)]
+    lib.pc_destroy.argtypes = [C.c_void_p]
+    lib.pc_plan_budget.argtypes = [C.POINTER(pc_budget_params), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.pc_score.argtypes = [C.c_void_p, C.POINTER(pc_cache), C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32),
+                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.pc_compact.argtypes = [C.c_void_p, C.POINTER(pc_cache), C.c_void_p, C.POINTER(C.c_int32), C.c_int32,
+                               C.POINTER(pc_cache), C.c_void_p]
+    lib.pc_attend_frame.argtypes = [C.c_void_p, C.POINTER(pc_cache), C.POINTER(pc_segment), C.c_void_p, C.c_void_p,
+                                    C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.pc_poll_status.argtypes = [C.c_void_p, C.c_void_p]
+    lib.pc_set_attend_impl.argtypes = [C.c_void_p, C.c_int32]
+    _lib = lib
+    return lib
+
+
+def _check(status: int, what: str) -> None:
+    if status != PC_OK:
+        raise PackCacheError(status, what)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors passed to the library must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _i32p(a: np.ndarray):
+    return a.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+@dataclass
+class Segment:
+    """A run of tokens on the device: K/V [capacity][Hkv][d], pos [capacity][4] int32."""
+    k: Optional[torch.Tensor]
+    v: Optional[torch.Tensor]
+    pos: Optional[torch.Tensor]
+    n_tokens: int
+
+    @staticmethod
+    def empty() -> "Segment":
+        return Segment(None, None, None, 0)
+
+    @property
+    def capacity(self) -> int:
+        return 0 if self.k is None else self.k.shape[0]
+
+    def c(self) -> pc_segment:
+        return pc_segment(_ptr(self.k), _ptr(self.v), _ptr(self.pos), self.n_tokens, self.capacity)
+
+
+@dataclass
+class Cache:
+    """Anchors held apart from the history frames (oldest -> newest); frame_count lives on the host."""
+    anchors: Segment
+    history: Segment
+    frame_count: np.ndarray
+
+    def c(self) -> pc_cache:
+        self._fc = _i32(self.frame_count)            # keep alive for the duration of the call
+        return pc_cache(self.anchors.c(), self.history.c(), len(self._fc), _i32p(self._fc))
+
+
+class Context:
+    """Owns a pc_ctx (rotary tables, status word, scratch) on the current CUDA device."""
+
+    def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: int, rope_base: float,
+                 max_pos: Sequence[int], max_q: int, max_keys: int):
+        lib = load()
+        self.desc = pc_layer_desc(n_q_heads, n_kv_heads, head_dim, dtype, rope_base, (C.c_int32 * 3)(*max_pos),
+                                  max_q, max_keys)
+        self.torch_dtype = torch.bfloat16 if dtype == PC_BF16 else torch.float32
+        h = C.c_void_p()
+        _check(lib.pc_create(C.byref(self.desc), C.byref(h)), "pc_create")
+        self.handle = h
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            load().pc_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def pc_plan_budget(kind: int, param: float, total: int, keep_full: int, avail: Sequence[int],
+                   min_quota: int = 0) -> np.ndarray:
+    avail = _i32(avail)
+    out = np.zeros(len(avail), dtype=np.int32)
+    p = pc_budget_params(kind, param, total, keep_full, min_quota)
+    _check(load().pc_plan_budget(C.byref(p), len(avail), _i32p(avail), _i32p(out)), "pc_plan_budget")
+    return out
+
+
+def pc_score(ctx: Context, src: Cache, q: Optional[torch.Tensor], q_pos: Optional[torch.Tensor], budget,
+             valid: Optional[torch.Tensor] = None, scores_override: Optional[torch.Tensor] = None,
+             scores: Optional[torch.Tensor] = None, sel_idx: Optional[torch.Tensor] = None, stream=None):
+    """Returns (scores [n_src] fp32, sel_idx [sum(budget)] int32), both on the device."""
+    budget = _i32(budget)
+    dev = src.history.k.device if src.history.k is not None else torch.device("cuda")
+    if scores is None and scores_override is None:
+        scores = torch.empty(max(src.history.n_tokens, 1), dtype=torch.float32, device=dev)
+    if sel_idx is None:
+        sel_idx = torch.empty(max(int(budget.sum()), 1), dtype=torch.int32, device=dev)
+    n_q = 0 if q is None else q.shape[0]
+    c = src.c()
+    _check(load().pc_score(ctx.handle, C.byref(c), _ptr(q), _ptr(q_pos), n_q, _i32p(budget), _ptr(valid),
+                           _ptr(scores_override), _ptr(scores), _ptr(sel_idx), _stream(stream)), "pc_score")
+    return scores, sel_idx
+
+
+def pc_compact(ctx: Context, src: Cache, sel_idx: torch.Tensor, budget, delta_t: int, dst: Cache, stream=None) -> None:
+    budget = _i32(budget)
+    cs, cd = src.c(), dst.c()
+    _check(load().pc_compact(ctx.handle, C.byref(cs), _ptr(sel_idx), _i32p(budget), delta_t, C.byref(cd),
+                             _stream(stream)), "pc_compact")
+    dst.history.n_tokens = int(budget.sum())
+    dst.frame_count = budget.copy()
+
+
+def pc_attend_frame(ctx: Context, cache: Cache, current: Optional[Segment], q: torch.Tensor, q_pos: torch.Tensor,
+                    out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None, want_lse: bool = False,
+                    stream=None):
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None and want_lse:
+        lse = torch.empty(q.shape[0], q.shape[1], dtype=torch.float32, device=q.device)
+    c = cache.c()
+    cur = current.c() if current is not None else None
+    _check(load().pc_attend_frame(ctx.handle, C.byref(c), C.byref(cur) if cur is not None else None, _ptr(q),
+                                  _ptr(q_pos), q.shape[0], _ptr(out), _ptr(lse), _stream(stream)), "pc_attend_frame")
+    return (out, lse) if want_lse else out
+
+
+def pc_poll_status(ctx: Context, stream=None) -> int:
+    return load().pc_poll_status(ctx.handle, _stream(stream))
+
+
+def pc_set_attend_impl(ctx: Context, impl: int) -> None:
+    _check(load().pc_set_attend_impl(ctx.handle, impl), "pc_set_attend_impl")

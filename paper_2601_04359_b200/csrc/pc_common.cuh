@@ -1,0 +1,113 @@
+// Shared declarations of the PackCache CUDA library (sm_100a).  Nothing here is used by the CPU oracle.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "packcache.h"
+
+#define PC_CUDA_TRY(expr)                                                                     \
+    do {                                                                                      \
+        cudaError_t _e = (expr);                                                              \
+        if (_e != cudaSuccess) {                                                              \
+            fprintf(stderr, "packcache: %s failed: %s (%s:%d)\n", #expr, cudaGetErrorString(_e), \
+                    __FILE__, __LINE__);                                                      \
+            return PC_ERR_CUDA;                                                               \
+        }                                                                                     \
+    } while (0)
+
+// "where" codes stored beside a device-side status (second status word)
+enum {
+    PC_WHERE_SCORE_POS = 1,
+    PC_WHERE_QPOOL_POS = 2,
+    PC_WHERE_SELECT_NAN = 3,
+    PC_WHERE_PACK_INDEX = 4,
+    PC_WHERE_ATTN_POS = 5,
+    PC_WHERE_ATTN_WAIT = 6,
+    PC_WHERE_ROPE_POS = 7,
+};
+
+constexpr int PC_QPOOL_BLOCKS = 64;
+constexpr int PC_MAX_SEGMENTS = 3;
+
+// Rotary tables: for axis a (t, h, w) a [max_pos[a]][n_axis[a]] array of (cos, sin) of pos * base^(-m/n_axis[a]).
+// Pair i of a head uses axis i % 3 and column m = i / 3.
+struct pc_rope_dev {
+    const float2 *tab;   // device, the three tables back to back
+    int32_t off[3];      // offset (in float2) of each axis table
+    int32_t n_axis[3];   // pairs per axis
+    int32_t max_pos[3];
+};
+
+struct pc_ctx {
+    pc_layer_desc desc;
+    int device;
+    int sm_count;
+    int group;                 // Hq / Hkv
+    int elem_size;             // bytes per element
+    int attend_impl;           // 0 tensor-core (bf16), 1 CUDA-core
+    pc_rope_dev rope;
+    float2 *rope_tab;          // owned
+    int32_t *status;           // device [2]: code, where
+    int32_t *host_status;      // pinned [2]
+    float *qpool_partial;      // device [PC_QPOOL_BLOCKS][Hkv*d]
+    float *qpool;              // device [Hkv*d]
+    unsigned int *ticket;      // device, zero between calls
+    // attention scratch (tensor-core path)
+    void *k_rot;               // rotated keys, bf16 [rows][Hkv][d]
+    size_t k_rot_rows;
+    float *part_o;             // split-KV partial outputs
+    float *part_ml;            // split-KV partial (max, sum)
+    size_t part_o_floats, part_ml_floats;
+};
+
+__device__ __forceinline__ void pc_flag(int32_t *status, int code, int where) {
+    if (atomicCAS(status, 0, code) == 0) status[1] = where;
+}
+
+// (cos, sin) for pair i of a head at position p[0..2]; flags and clamps a position outside the table.
+__device__ __forceinline__ float2 pc_rope_cs(const pc_rope_dev &r, int pair, int pt, int ph, int pw, int32_t *status,
+                                             int where) {
+    int a = pair % 3, m = pair / 3;
+    int pa = a == 0 ? pt : (a == 1 ? ph : pw);
+    if (pa < 0 || pa >= r.max_pos[a]) {
+        pc_flag(status, PC_ERR_INVALID_ARG, where);
+        pa = pa < 0 ? 0 : r.max_pos[a] - 1;
+    }
+    return __ldg(r.tab + r.off[a] + (size_t)pa * r.n_axis[a] + m);
+}
+
+__device__ __forceinline__ float pc_bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float pc_bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint32_t pc_pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+__device__ __forceinline__ uint4 pc_ldg_stream(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void pc_stg_stream(void *p, uint4 v) {
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+                 "r"(v.w)
+                 : "memory");
+}
+
+// host-side helpers implemented in pc_api.cu
+bool pc_aligned16(const void *p);
+pc_status pc_check_segment(const pc_segment *s, bool allow_empty);
+
+// stage launchers (each validates nothing: the pc_* entry points did)
+pc_status pc_launch_attend_simt(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
+                                int32_t n_q, void *out, float *lse, cudaStream_t stream);
+pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
+                              int32_t n_q, void *out, float *lse, cudaStream_t stream);
+pc_status pc_attend_tc_scratch(const pc_layer_desc *d, int sm_count, size_t *k_rot_rows, size_t *part_o_floats,
+                               size_t *part_ml_floats);

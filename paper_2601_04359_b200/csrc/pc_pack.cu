@@ -1,0 +1,100 @@
+// Gather/pack of retained K/V rows into a contiguous cache (Fig. 6b) with the temporal rebase of Eq. 9.
+//
+// One warp moves one retained token: its K row and V row over all KV heads (16-byte vector loads and stores,
+// consecutive lanes on consecutive 16-byte chunks, so every request is a full 512-byte line run) and its position
+// record with t shifted by delta_t.  Rows are streamed (no L1 allocation): nothing here is read twice.
+#include "pc_common.cuh"
+
+namespace {
+
+constexpr int PACK_THREADS = 256;
+
+template <int CPL /* 16-byte chunks per lane per row; 0 = generic loop */>
+__global__ void __launch_bounds__(PACK_THREADS) k_pack(const char *__restrict__ src_k, const char *__restrict__ src_v,
+                                                       const int32_t *__restrict__ src_pos,
+                                                       const int32_t *__restrict__ sel_idx, int n_sel, int n_src,
+                                                       int row_bytes, int delta_t, char *__restrict__ dst_k,
+                                                       char *__restrict__ dst_v, int32_t *__restrict__ dst_pos,
+                                                       int32_t *status) {
+    const int lane = threadIdx.x & 31;
+    const int r = (blockIdx.x * PACK_THREADS + threadIdx.x) >> 5;
+    if (r >= n_sel) return;
+    const int s = __ldg(sel_idx + r);
+    if (s < 0 || s >= n_src) {                      // a bad index is recorded and the row skipped
+        if (lane == 0) pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_PACK_INDEX);
+        return;
+    }
+    const char *sk = src_k + (size_t)s * row_bytes, *sv = src_v + (size_t)s * row_bytes;
+    char *dk = dst_k + (size_t)r * row_bytes, *dv = dst_v + (size_t)r * row_bytes;
+    if constexpr (CPL > 0) {
+        uint4 a[CPL], b[CPL];
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) a[c] = pc_ldg_stream(sk + (size_t)(c * 32 + lane) * 16);
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) b[c] = pc_ldg_stream(sv + (size_t)(c * 32 + lane) * 16);
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) pc_stg_stream(dk + (size_t)(c * 32 + lane) * 16, a[c]);
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) pc_stg_stream(dv + (size_t)(c * 32 + lane) * 16, b[c]);
+    } else {
+        for (int off = lane * 16; off < row_bytes; off += 32 * 16) {
+            const uint4 a = pc_ldg_stream(sk + off), b = pc_ldg_stream(sv + off);
+            pc_stg_stream(dk + off, a);
+            pc_stg_stream(dv + off, b);
+        }
+    }
+    if (lane == 0) {
+        int4 p = __ldg(reinterpret_cast<const int4 *>(src_pos) + s);
+        p.x -= delta_t;                              // only t moves; h, w and the tag are carried as they are
+        reinterpret_cast<int4 *>(dst_pos)[r] = p;
+    }
+}
+
+bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
+    const char *x = static_cast<const char *>(a), *y = static_cast<const char *>(b);
+    return x < y + nb && y < x + na;
+}
+
+}  // namespace
+
+extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget,
+                                int32_t delta_t, pc_cache *dst, void *stream_) {
+    if (!ctx || !src || !dst || !budget) return PC_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (src->n_frames < 0 || (src->n_frames > 0 && !src->frame_count)) return PC_ERR_INVALID_ARG;
+    pc_status st = pc_check_segment(&src->history, true);
+    if (st != PC_OK) return st;
+    int64_t n_sel = 0, n_src = 0;
+    for (int f = 0; f < src->n_frames; ++f) {
+        if (budget[f] < 0 || src->frame_count[f] < 0) return PC_ERR_INVALID_ARG;
+        if (budget[f] > src->frame_count[f]) return PC_ERR_BUDGET;
+        n_sel += budget[f];
+        n_src += src->frame_count[f];
+    }
+    if (n_src != src->history.n_tokens) return PC_ERR_INVALID_ARG;
+    if (n_sel > dst->history.capacity) return PC_ERR_CAPACITY;
+    if (n_sel == 0) return PC_OK;
+    if (!sel_idx || !pc_aligned16(sel_idx)) return PC_ERR_INVALID_ARG;
+    const pc_segment &D = dst->history;
+    if (!D.k || !D.v || !D.pos || !pc_aligned16(D.k) || !pc_aligned16(D.v) || !pc_aligned16(D.pos))
+        return PC_ERR_INVALID_ARG;
+    const int row_bytes = ctx->desc.n_kv_heads * ctx->desc.head_dim * ctx->elem_size;
+    const size_t src_bytes = (size_t)n_src * row_bytes, dst_bytes = (size_t)n_sel * row_bytes;
+    if (overlaps(src->history.k, src_bytes, D.k, dst_bytes) || overlaps(src->history.v, src_bytes, D.v, dst_bytes) ||
+        overlaps(src->history.k, src_bytes, D.v, dst_bytes) || overlaps(src->history.v, src_bytes, D.k, dst_bytes) ||
+        overlaps(src->history.pos, (size_t)n_src * 16, D.pos, (size_t)n_sel * 16))
+        return PC_ERR_INVALID_ARG;
+    const int blocks = (int)((n_sel * 32 + PACK_THREADS - 1) / PACK_THREADS);
+    const char *sk = static_cast<const char *>(src->history.k), *sv = static_cast<const char *>(src->history.v);
+    char *dk = static_cast<char *>(D.k), *dv = static_cast<char *>(D.v);
+#define PC_PACK_ARGS sk, sv, src->history.pos, sel_idx, (int)n_sel, (int)n_src, row_bytes, delta_t, dk, dv, D.pos, ctx->status
+    switch (row_bytes) {
+    case 512: k_pack<1><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
+    case 1024: k_pack<2><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
+    case 2048: k_pack<4><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
+    default: k_pack<0><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
+    }
+#undef PC_PACK_ARGS
+    PC_CUDA_TRY(cudaGetLastError());
+    return PC_OK;
+}

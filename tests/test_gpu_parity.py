@@ -1,0 +1,333 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Integer results (budgets, selected indices, packed rows and positions) must match bit for bit; fp32 scores
+within 1e-4 relative; attention within 1e-4 relative (fp32) or 2e-2 max-abs (bf16, unit-variance inputs)."""
+from __future__ import annotations
+
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_04359_b200 import binding as pc
+from paper_2601_04359_b200 import workload as wl
+from tests.gpu_util import DeviceLayer, dev, host, idev, make_ctx, score_tolerance, segment
+
+pytestmark = pytest.mark.gpu
+
+BF16_ATOL = 2e-2
+F32_RTOL = 1e-4
+
+
+def _plan(cfg, n_frames=None):
+    b = cfg.budget
+    avail = [cfg.frame_tokens] * (n_frames if n_frames is not None else cfg.n_frames)
+    got = pc.pc_plan_budget(b.kind, b.param, b.total, b.keep_full, avail)
+    assert got.tolist() == oracle.plan_budget(b.kind, b.param, b.total, b.keep_full, avail).tolist()
+    return got
+
+
+def _ok(ctx):
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+
+
+def _check_attention(cfg, got: np.ndarray, want: np.ndarray):
+    if cfg.dtype == wl.BF16:
+        assert np.abs(got - want).max() <= BF16_ATOL
+    else:
+        scale = np.abs(want).max()
+        assert np.abs(got - want).max() <= F32_RTOL * scale
+
+
+def _pipeline(cfg, impl=None, with_current=False, delta_t=0):
+    """plan -> score -> select -> pack -> attend, each stage checked against the oracle."""
+    L = wl.make_layer(cfg, with_current=with_current)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    if impl is not None:
+        pc.pc_set_attend_impl(ctx, impl)
+    budget = _plan(cfg)
+
+    # scores: fp32 within 1e-4 relative of the fp64 mean logit
+    scores, sel = pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget)
+    ref = oracle.score(L.hist_k, L.hist_pos, L.q, L.q_pos, cfg.rope_base)
+    got = host(scores)[:cfg.n_src].astype(np.float64)
+    assert (np.abs(got - ref) <= score_tolerance(ref, L.frame_count)).all()
+    # the GPU's own selection must be a valid top-k of the GPU's own scores
+    sel_np = sel.cpu().numpy()[:budget.sum()]
+    _valid_topk(host(scores)[:cfg.n_src], sel_np, L.frame_count, budget)
+
+    # selection: bit-exact when both sides see the same fp32 scores (the oracle's, rounded to fp32)
+    ref32 = ref.astype(np.float32)
+    _, sel2 = pc.pc_score(ctx, D.cache, None, None, budget, scores_override=torch.from_numpy(ref32).cuda())
+    want_sel = oracle.select(ref32, L.frame_count, budget)
+    assert sel2.cpu().numpy()[:len(want_sel)].tolist() == want_sel.tolist()
+
+    # pack: bit copies of the selected rows, positions carried, t rebased
+    dst = D.empty_packed(int(budget.sum()) + 5, poison=3.0)
+    pc.pc_compact(ctx, D.cache, sel2, budget, delta_t, dst)
+    wk, wv, wp = oracle.pack(L.hist_k, L.hist_v, L.hist_pos, want_sel, delta_t)
+    n = len(want_sel)
+    assert np.array_equal(host(dst.history.k)[:n], wk) and np.array_equal(host(dst.history.v)[:n], wv)
+    assert np.array_equal(dst.history.pos.cpu().numpy()[:n], wp)
+    assert (host(dst.history.k)[n:] == 3.0).all() and (dst.history.pos.cpu().numpy()[n:] == -7).all()
+    assert dst.history.n_tokens == n
+
+    # attention over anchors ++ packed (++ current)
+    segs = [(L.anchor_k, L.anchor_v, L.anchor_pos), (wk, wv, wp)]
+    if with_current:
+        segs.append((L.cur_k, L.cur_v, L.q_pos))
+    want, want_lse = oracle.attend(L.q, L.q_pos, segs, cfg.rope_base, want_lse=True)
+    out, lse = pc.pc_attend_frame(ctx, dst, D.current if with_current else None, D.q, D.q_pos, want_lse=True)
+    _ok(ctx)
+    _check_attention(cfg, host(out).astype(np.float64), want)
+    assert np.abs(host(lse) - want_lse).max() <= (2e-2 if cfg.dtype == wl.BF16 else 1e-4)
+    ctx.close()
+
+
+def _valid_topk(scores, sel, frame_count, budget):
+    """Property check at any size: per frame, ascending unique indices of the right count, and no unselected token
+    beats a selected one under (score desc, index asc)."""
+    base = out = 0
+    for n, t in zip(frame_count, budget):
+        s = sel[out:out + t]
+        assert (np.diff(s) > 0).all() and (s >= base).all() and (s < base + n).all()
+        if 0 < t < n:
+            mask = np.zeros(n, bool)
+            mask[s - base] = True
+            fr = scores[base:base + n]
+            worst_in = min(zip(fr[mask], -(np.nonzero(mask)[0])))        # lowest score, then highest index
+            best_out = max(zip(fr[~mask], -(np.nonzero(~mask)[0])))      # highest score, then lowest index
+            assert worst_in > best_out
+        base += n
+        out += t
+
+
+# ------------------------------------------------------------------------------------------- whole pipeline
+def test_tiny_fp32_pipeline_closed_half():
+    _pipeline(wl.CONFIGS["tiny"])
+
+
+def test_tiny_fp32_pipeline_geometric_capped():
+    _pipeline(wl.with_budget(wl.CONFIGS["tiny"], kind=wl.GEOMETRIC, param=0.5), with_current=True, delta_t=4)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_small_bf16_pipeline(impl):
+    _pipeline(wl.small_bf16(), impl=impl)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_small_bf16_pipeline_with_current_and_rebase(impl):
+    _pipeline(wl.small_bf16(n_frames=3, grid=(11, 13), n_text=130, total=260, kind=wl.LINEAR, param=0.0, keep_full=0,
+                            seed=5), impl=impl, with_current=True, delta_t=8)
+
+
+def test_unlimited_budget_equals_full_cache_attention():
+    cfg = wl.with_budget(wl.small_bf16(n_frames=2, grid=(8, 9)), total=10 ** 6, keep_full=0)
+    L = wl.make_layer(cfg, with_current=True)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    budget = _plan(cfg)
+    assert budget.tolist() == L.frame_count.tolist()
+    _, sel = pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget)
+    assert sel.cpu().numpy().tolist() == list(range(cfg.n_src))
+    dst = D.empty_packed(cfg.n_src)
+    pc.pc_compact(ctx, D.cache, sel, budget, 0, dst)
+    a = pc.pc_attend_frame(ctx, dst, D.current, D.q, D.q_pos)
+    b = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos)
+    _ok(ctx)
+    assert torch.equal(a, b)
+    k = np.concatenate([L.anchor_k, L.hist_k, L.cur_k]); v = np.concatenate([L.anchor_v, L.hist_v, L.cur_v])
+    pos = np.concatenate([L.anchor_pos, L.hist_pos, L.q_pos])
+    n = cfg.frame_tokens
+    block = np.concatenate([np.zeros(cfg.n_text), np.ones(n)] + [np.full(n, 2 + f) for f in range(cfg.n_frames + 1)])
+    q_all = np.zeros((len(k),) + L.q.shape[1:], np.float32)
+    q_all[-cfg.n_q:] = L.q
+    full = oracle.full_block_causal_attention(q_all, k, v, pos, block.astype(np.int32))[-cfg.n_q:]
+    assert np.abs(host(a) - full).max() <= BF16_ATOL
+
+
+# ------------------------------------------------------------------------------------------- select
+def _select_case(frame_count, budget, scores, cfg=None):
+    cfg = cfg or wl.CONFIGS["tiny"]
+    ctx = make_ctx(cfg, max_keys=max(int(np.sum(frame_count)), 1) + 16)
+    n = int(np.sum(frame_count))
+    z = torch.zeros((max(n, 1), cfg.n_kv_heads, cfg.head_dim), device="cuda")
+    cache = pc.Cache(pc.Segment.empty(), pc.Segment(z, z, torch.zeros((max(n, 1), 4), dtype=torch.int32, device="cuda"), n),
+                     np.asarray(frame_count, np.int32))
+    _, sel = pc.pc_score(ctx, cache, None, None, budget, scores_override=torch.from_numpy(scores).cuda())
+    _ok(ctx)
+    want = oracle.select(scores, frame_count, budget)
+    assert sel.cpu().numpy()[:len(want)].tolist() == want.tolist()
+    ctx.close()
+
+
+def test_select_ties_and_edges():
+    rng = np.random.default_rng(0)
+    for trial in range(12):
+        F = int(rng.integers(1, 9))
+        fc = rng.integers(0, 1700, size=F)
+        if trial == 0:
+            fc[0] = 0
+        bud = np.array([int(rng.integers(0, n + 1)) for n in fc])
+        if trial % 3 == 0:
+            bud[-1] = fc[-1]
+        if trial % 4 == 0:
+            bud[0] = 0
+        n = int(fc.sum())
+        if n == 0:
+            continue
+        s = wl.tie_scores(rng, n) if trial % 2 else rng.standard_normal(n).astype(np.float32)
+        if trial % 5 == 0:
+            s[rng.random(n) < 0.2] = -np.inf
+        _select_case(fc, bud, s)
+
+
+def test_select_all_equal_and_tiny_values():
+    _select_case([1008], [300], np.zeros(1008, np.float32))
+    s = np.full(600, 1e-40, np.float32)            # denormals and signed zeros keep their order
+    s[::3] = -1e-40
+    s[1::7] = -0.0
+    s[2::11] = 0.0
+    _select_case([600], [333], s)
+
+
+def test_select_full_size_headline_shape():
+    cfg = wl.CONFIGS["lumos47"]
+    rng = np.random.default_rng(1)
+    fc = [cfg.frame_tokens] * cfg.n_frames
+    budget = _plan(cfg)
+    _select_case(fc, budget, rng.standard_normal(cfg.n_src).astype(np.float32), cfg)
+    _select_case(fc, budget, wl.tie_scores(rng, cfg.n_src, levels=41), cfg)
+
+
+# ------------------------------------------------------------------------------------------- score
+def test_score_valid_mask_and_pooling_at_scale():
+    cfg = wl.small_bf16(n_frames=4, grid=(12, 21), total=300, keep_full=0)
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    budget = _plan(cfg)
+    valid = (np.random.default_rng(0).random(cfg.n_src) < 0.7).astype(np.uint8)
+    scores, sel = pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget, valid=torch.from_numpy(valid).cuda())
+    _ok(ctx)
+    ref = oracle.score(L.hist_k, L.hist_pos, L.q, L.q_pos, valid=valid)
+    got = host(scores).astype(np.float64)
+    assert np.array_equal(np.isneginf(got), valid == 0)
+    m = valid == 1
+    assert (np.abs(got[m] - ref[m]) <= score_tolerance(ref, L.frame_count)[m]).all()
+    _valid_topk(host(scores), sel.cpu().numpy()[:budget.sum()], L.frame_count, budget)
+    assert valid[sel.cpu().numpy()[:budget.sum()]].all()       # budgets fit inside the valid tokens here
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------------- errors
+def test_host_detected_errors():
+    cfg = wl.CONFIGS["tiny"]
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    budget = _plan(cfg)
+    bad = budget.copy(); bad[0] = cfg.frame_tokens + 1
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_score(ctx, D.cache, D.q, D.q_pos, bad)
+    assert e.value.status == pc.PC_ERR_BUDGET
+    _, sel = pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget)
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_compact(ctx, D.cache, sel, budget, 0, D.empty_packed(int(budget.sum()) - 1))
+    assert e.value.status == pc.PC_ERR_CAPACITY
+    with pytest.raises(pc.PackCacheError) as e:                   # destination aliases the source
+        pc.pc_compact(ctx, D.cache, sel, budget, 0, D.cache)
+    assert e.value.status == pc.PC_ERR_INVALID_ARG
+    with pytest.raises(pc.PackCacheError) as e:                   # misaligned query pointer
+        pc.pc_attend_frame(ctx, D.cache, None, D.q.view(-1)[1:1 + 64 * 4 * 64].view(64, 4, 64), D.q_pos,
+                           out=torch.empty_like(D.q))
+    assert e.value.status == pc.PC_ERR_INVALID_ARG
+    wrong = pc.Cache(D.cache.anchors, D.cache.history, np.array([64] * 5, np.int32))   # frame table does not sum up
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_score(ctx, wrong, D.q, D.q_pos, budget[:5])
+    assert e.value.status == pc.PC_ERR_INVALID_ARG
+    small = make_ctx(cfg, max_keys=100)
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_attend_frame(small, D.cache, None, D.q, D.q_pos)
+    assert e.value.status == pc.PC_ERR_CAPACITY
+    with pytest.raises(pc.PackCacheError):
+        pc.Context(5, 2, 64, pc.PC_F32, 10000.0, (8, 8, 8), 8, 8)
+    with pytest.raises(pc.PackCacheError):
+        pc.Context(4, 2, 48, pc.PC_F32, 10000.0, (8, 8, 8), 8, 8)
+    _ok(ctx)
+
+
+def test_device_side_checks_record_instead_of_faulting():
+    cfg = wl.CONFIGS["tiny"]
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    budget = _plan(cfg)
+    _, sel = pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget)
+    _ok(ctx)
+    # an index outside the source is recorded and its row skipped
+    bad_sel = sel.clone(); bad_sel[3] = cfg.n_src + 100
+    dst = D.empty_packed(int(budget.sum()), poison=9.0)
+    pc.pc_compact(ctx, D.cache, bad_sel, budget, 0, dst)
+    assert pc.pc_poll_status(ctx) == pc.PC_ERR_INVALID_ARG
+    assert (host(dst.history.k)[3] == 9.0).all()
+    assert pc.pc_poll_status(ctx) == pc.PC_OK                     # polling clears the word
+    # a position outside the rotary tables is recorded (and clamped)
+    tight = make_ctx(cfg, max_pos=(16, 16, 16))
+    pc.pc_score(tight, D.cache, D.q, D.q_pos, budget)
+    assert pc.pc_poll_status(tight) == pc.PC_ERR_INVALID_ARG
+    pc.pc_attend_frame(tight, D.cache, None, D.q, D.q_pos)
+    assert pc.pc_poll_status(tight) == pc.PC_ERR_INVALID_ARG
+    # NaN scores are an error for selection
+    s = np.zeros(cfg.n_src, np.float32); s[5] = np.nan
+    pc.pc_score(ctx, D.cache, None, None, budget, scores_override=torch.from_numpy(s).cuda())
+    assert pc.pc_poll_status(ctx) == pc.PC_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------------------------------- full size
+@pytest.mark.parametrize("name", ["lumos12", "lumos47"])
+def test_full_size_sampled_against_oracle(name):
+    """The benchmark's launch configuration at full size: scores against the pooled fp64 oracle on every token and
+    the mean-logit oracle on a sample; selection and packing bit-exact; attention on sampled (query, head) rows."""
+    cfg = wl.CONFIGS[name]
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    budget = _plan(cfg)
+    rng = np.random.default_rng(0)
+
+    scores, sel = pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget)
+    got = host(scores).astype(np.float64)
+    ref = oracle.score_pooled(L.hist_k, L.hist_pos, L.q, L.q_pos)
+    tol = score_tolerance(ref, L.frame_count)
+    assert (np.abs(got - ref) <= tol).all()
+    idx = rng.choice(cfg.n_src, size=24, replace=False)
+    naive = oracle.score(L.hist_k, L.hist_pos, L.q, L.q_pos, idx=idx)
+    assert (np.abs(got[idx] - naive) <= tol[idx]).all()
+    _valid_topk(host(scores), sel.cpu().numpy(), L.frame_count, budget)
+
+    ref32 = ref.astype(np.float32)
+    _, sel2 = pc.pc_score(ctx, D.cache, None, None, budget, scores_override=torch.from_numpy(ref32).cuda())
+    want_sel = oracle.select(ref32, L.frame_count, budget)
+    assert np.array_equal(sel2.cpu().numpy(), want_sel)
+
+    dst = D.empty_packed(int(budget.sum()))
+    pc.pc_compact(ctx, D.cache, sel2, budget, 0, dst)
+    wk, wv, wp = oracle.pack(L.hist_k, L.hist_v, L.hist_pos, want_sel, 0)
+    assert np.array_equal(host(dst.history.k), wk) and np.array_equal(host(dst.history.v), wv)
+    assert np.array_equal(dst.history.pos.cpu().numpy(), wp)
+
+    out, lse = pc.pc_attend_frame(ctx, dst, None, D.q, D.q_pos, want_lse=True)
+    _ok(ctx)
+    rows = np.stack([rng.integers(0, cfg.n_q, size=96), rng.integers(0, cfg.n_q_heads, size=96)], axis=1).astype(np.int32)
+    rows[0] = (0, 0); rows[1] = (cfg.n_q - 1, cfg.n_q_heads - 1); rows[2] = (1007, 5); rows[3] = (896, 23)
+    want, want_lse = oracle.attend(L.q, L.q_pos, [(L.anchor_k, L.anchor_v, L.anchor_pos), (wk, wv, wp)], rows=rows,
+                                   want_lse=True)
+    o = host(out)
+    assert np.abs(o[rows[:, 0], rows[:, 1]] - want).max() <= BF16_ATOL
+    assert np.abs(host(lse)[rows[:, 0], rows[:, 1]] - want_lse).max() <= 2e-2
+    assert np.isfinite(o).all()
+    ctx.close()
