@@ -168,6 +168,10 @@ pc_status pc_poll_status(pc_ctx *ctx, void *stream);
  * 1 = CUDA-core kernel (a slow second opinion).  Returns PC_ERR_INVALID_ARG otherwise. */
 pc_status pc_set_attend_impl(pc_ctx *ctx, int32_t impl);
 
+/* Fix the number of key ranges the tensor-core attention kernel splits the keys into (1..4); 0 lets each call
+ * choose the count that fills the GPU's SMs best.  Results agree up to fp32 rounding order. */
+pc_status pc_set_kv_splits(pc_ctx *ctx, int32_t n);
+
 const char *pc_status_string(pc_status s);
 
 #ifdef __cplusplus

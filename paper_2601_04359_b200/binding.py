@@ -22,7 +22,7 @@ PC_GEOMETRIC, PC_CLOSED_HALF, PC_LINEAR, PC_HALFLIFE = 0, 1, 2, 3
 PC_MAX_FRAMES = 256
 
 EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact", "pc_attend_frame",
-           "pc_poll_status", "pc_set_attend_impl", "pc_status_string"]
+           "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_status_string"]
 
 
 class pc_layer_desc(C.Structure):
@@ -77,6 +77,7 @@ def load() -> C.CDLL:
                                     C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.pc_poll_status.argtypes = [C.c_void_p, C.c_void_p]
     lib.pc_set_attend_impl.argtypes = [C.c_void_p, C.c_int32]
+    lib.pc_set_kv_splits.argtypes = [C.c_void_p, C.c_int32]
     _lib = lib
     return lib
 
@@ -219,3 +220,7 @@ def pc_poll_status(ctx: Context, stream=None) -> int:
 
 def pc_set_attend_impl(ctx: Context, impl: int) -> None:
     _check(load().pc_set_attend_impl(ctx.handle, impl), "pc_set_attend_impl")
+
+
+def pc_set_kv_splits(ctx: Context, n: int) -> None:
+    _check(load().pc_set_kv_splits(ctx.handle, n), "pc_set_kv_splits")

@@ -50,6 +50,7 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
     c->group = desc->n_q_heads / desc->n_kv_heads;
     c->elem_size = desc->dtype == PC_BF16 ? 2 : 4;
     c->attend_impl = 0;
+    c->kv_splits = 0;
     PC_CUDA_TRY(cudaGetDevice(&c->device));
     PC_CUDA_TRY(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
 
@@ -89,6 +90,7 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
         if (st != PC_OK) return st;
         PC_CUDA_TRY(cudaMalloc(&c->k_rot, c->k_rot_rows * row * sizeof(__nv_bfloat16)));
         PC_CUDA_TRY(cudaMemset(c->k_rot, 0, c->k_rot_rows * row * sizeof(__nv_bfloat16)));
+        PC_CUDA_TRY(cudaMalloc(&c->q_rot, (size_t)desc->max_q * desc->n_q_heads * desc->head_dim * sizeof(__nv_bfloat16)));
         PC_CUDA_TRY(cudaMalloc(&c->part_o, std::max<size_t>(c->part_o_floats, 1) * sizeof(float)));
         PC_CUDA_TRY(cudaMalloc(&c->part_ml, std::max<size_t>(c->part_ml_floats, 1) * sizeof(float)));
     }
@@ -105,6 +107,7 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
     cudaFree(c->qpool);
     cudaFree(c->ticket);
     cudaFree(c->k_rot);
+    cudaFree(c->q_rot);
     cudaFree(c->part_o);
     cudaFree(c->part_ml);
     delete c;
@@ -114,6 +117,12 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
 extern "C" pc_status pc_set_attend_impl(pc_ctx *c, int32_t impl) {
     if (!c || impl < 0 || impl > 1) return PC_ERR_INVALID_ARG;
     c->attend_impl = impl;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_set_kv_splits(pc_ctx *c, int32_t n) {
+    if (!c || n < 0 || n > 4) return PC_ERR_INVALID_ARG;
+    c->kv_splits = n;
     return PC_OK;
 }
 

@@ -1,11 +1,617 @@
-// placeholder until the tcgen05 kernel lands
+// bf16 attention of one frame's queries over the compacted cache on tcgen05 tensor cores (Eq. 2, all keys visible).
+//
+// Launch sequence of pc_launch_attend_tc:
+//   k_rope_rows   rotates K of every segment (3D rotary tables, from the stored positions) into a bf16 scratch whose
+//                 segments start on 128-row boundaries, and rotates Q with log2(e)/sqrt(d) folded in.
+//   k_attend_tc   one CTA = two 128-row query tiles that share a KV head (grouped-query packing) x one KV range.
+//                 Warp 0 lane 0 drives TMA (K and V tiles, 128B swizzle, two stages each), warp 1 lane 0 issues
+//                 tcgen05.mma: S_t = Q_t K^T (both operands K-major in shared memory) into TMEM, and
+//                 O_t += P_t V with P_t read from TMEM and V MN-major in shared memory.  Warps 4-7 / 8-11 are the
+//                 softmax groups of tile 0 / 1: tcgen05.ld the S row, running max and sum in fp32 (base 2), write
+//                 bf16 P over S in TMEM, and rescale O in TMEM only when the running max moved by more than 2^8.
+//                 While one tile's softmax runs, the tensor core works on the other tile.
+//   k_combine     merges the KV ranges' (max, sum, O) partials when the keys were split across CTAs.
+//
+// TMEM columns: S0/P0 0-127, S1/P1 128-255, O0 256-383, O1 384-511 (fp32, 128 lanes = the tile's rows).
+// Every wait is bounded: a wait that runs out records PC_ERR_TIMEOUT, raises a CTA-wide abort flag that makes every
+// later wait return at once, and the CTA still drains its copies, frees TMEM and exits.
+#include <cuda.h>
+
+#include <algorithm>
+
 #include "pc_common.cuh"
+
+namespace {
+
+constexpr int TC_THREADS = 384;
+constexpr int TILE = 128;                 // query rows per tile, keys per tile, head dim
+constexpr int HALF_BYTES = TILE * 64 * 2; // one [128][64] bf16 box: 16 KB
+constexpr int TILE_BYTES = 2 * HALF_BYTES;
+constexpr int KV_STAGES = 2;
+constexpr int MAX_SPLITS = 4;
+constexpr float RESCALE_THRESHOLD = 8.0f;
+
+// shared memory map (dynamic, 1024-byte aligned)
+constexpr int SM_Q = 0;                                   // 2 tiles
+constexpr int SM_K = SM_Q + 2 * TILE_BYTES;               // KV_STAGES tiles
+constexpr int SM_V = SM_K + KV_STAGES * TILE_BYTES;       // KV_STAGES tiles
+constexpr int SM_BAR = SM_V + KV_STAGES * TILE_BYTES;     // barriers etc.
+constexpr int SM_TOTAL = SM_BAR + 256;
+constexpr int SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
+
+enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PFULL = 11,
+       BAR_DONE = 13, N_BARS = 14 };
+
+struct TcParams {
+    int n_q, n_q_heads, group, n_tb, tiles_per_g, pairs_per_g, n_splits, n_kv_tiles;
+    int n_seg;
+    int seg_tile_end[PC_MAX_SEGMENTS];
+    int seg_n[PC_MAX_SEGMENTS];
+    __nv_bfloat16 *out;
+    float *lse;
+    float *part_o;    // [item*S + s][2][128][128]
+    float *part_ml;   // [item*S + s][2][128][2]
+    int32_t *status;
+};
+
+// ------------------------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after about one second, or at once when another thread of the CTA already gave up.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
+    for (int i = 0; i < 2048; ++i)
+        if (mbar_try(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (;;) {
+        if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > 1000000000ull) {
+            *abort_flag = 1;
+            pc_flag(status, PC_ERR_TIMEOUT, PC_WHERE_ATTN_WAIT);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t *r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t *r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t *r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptors (128-byte swizzle, descriptor version 1).
+//   K-major operand (rows of 64 bf16 = 128 B, 8-row groups 1024 B apart): SBO = 1024, LBO unused.
+//   MN-major operand (V: a row = one key holding 64 contiguous head-dim elements): 8-key groups 1024 B apart
+//   (SBO), the second 64-element half of the head dim 16 KB further (LBO).
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)(HALF_BYTES >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 128
+constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t IDESC_QK = IDESC_BASE;               // A, B K-major
+constexpr uint32_t IDESC_PV = IDESC_BASE | (1u << 16);  // B (V) MN-major
+
+// ------------------------------------------------------------------------------------------------ rotary pre-pass
+struct RopeJob {
+    const __nv_bfloat16 *src;
+    const int32_t *pos;
+    __nv_bfloat16 *dst;
+    int n_rows, chunks_per_row /* 16-byte chunks */, first_warp;
+    float scale;
+};
+struct RopeJobs { RopeJob job[PC_MAX_SEGMENTS + 1]; int n_jobs, total_warps; };
+
+__global__ void __launch_bounds__(256) k_rope_rows(const __grid_constant__ RopeJobs jobs, pc_rope_dev rope, int d,
+                                                   int32_t *status) {
+    const int lane = threadIdx.x & 31;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (warp >= jobs.total_warps) return;
+    int ji = 0;
+    while (ji + 1 < jobs.n_jobs && warp >= jobs.job[ji + 1].first_warp) ++ji;
+    const RopeJob &J = jobs.job[ji];
+    const int row = warp - J.first_warp;
+    const int4 pp = __ldg(reinterpret_cast<const int4 *>(J.pos) + row);
+    // 32 lanes x 8 elements = 256 is a multiple of d: all of a lane's chunks hold the same four rotary pairs
+    const int pair0 = ((lane * 8) % d) / 2;
+    float2 cs[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_ROPE_POS);
+    const uint4 *src = reinterpret_cast<const uint4 *>(J.src) + (size_t)row * J.chunks_per_row;
+    uint4 *dst = reinterpret_cast<uint4 *>(J.dst) + (size_t)row * J.chunks_per_row;
+    for (int c = lane; c < J.chunks_per_row; c += 32) {
+        const uint4 v = pc_ldg_stream(src + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float x0 = pc_bf16_lo(w[u]), x1 = pc_bf16_hi(w[u]);
+            o[u] = pc_pack_bf16((x0 * cs[u].x - x1 * cs[u].y) * J.scale, (x0 * cs[u].y + x1 * cs[u].x) * J.scale);
+        }
+        dst[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ main kernel
+__device__ __forceinline__ void kv_tile_info(const TcParams &P, int jt, int &seg, int &local, int &n_valid) {
+    seg = 0;
+    int start = 0;
+    while (seg + 1 < P.n_seg && jt >= P.seg_tile_end[seg]) { start = P.seg_tile_end[seg]; ++seg; }
+    local = jt - start;
+    n_valid = min(TILE, P.seg_n[seg] - local * TILE);
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+            const __grid_constant__ CUtensorMap map_v0, const __grid_constant__ CUtensorMap map_v1,
+            const __grid_constant__ CUtensorMap map_v2, const __grid_constant__ TcParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(gen + SM_BAR + N_BARS * 8);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(gen + SM_BAR + N_BARS * 8 + 8);
+    const uint32_t bar0 = base + SM_BAR;
+    auto bar = [&](int i) { return bar0 + 8u * i; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // work item
+    const int item = blockIdx.x / P.n_splits, split = blockIdx.x % P.n_splits;
+    const int g = item / P.pairs_per_g, pair = item % P.pairs_per_g;
+    const int n_tiles_q = min(2, P.tiles_per_g - 2 * pair);            // 1 when the head group has an odd tile count
+    const int jt0 = (int)(((long long)P.n_kv_tiles * split) / P.n_splits);
+    const int jt1 = (int)(((long long)P.n_kv_tiles * (split + 1)) / P.n_splits);
+    const int n_j = jt1 - jt0;
+
+    if (threadIdx.x == 0) {
+        mbar_init(bar(BAR_Q), 1);
+        for (int s = 0; s < KV_STAGES; ++s) {
+            mbar_init(bar(BAR_KFULL + s), 1);
+            mbar_init(bar(BAR_KEMPTY + s), 1);
+            mbar_init(bar(BAR_VFULL + s), 1);
+            mbar_init(bar(BAR_VEMPTY + s), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar(BAR_SFULL + t), 1);
+            mbar_init(bar(BAR_PFULL + t), 128);
+        }
+        mbar_init(bar(BAR_DONE), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 2) {   // TMEM: all 512 columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(bar(BAR_Q), n_tiles_q * TILE_BYTES);
+            for (int t = 0; t < n_tiles_q; ++t) {
+                const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
+                tma_load_2d(base + SM_Q + t * TILE_BYTES, &map_q, h * TILE, tb * TILE, bar(BAR_Q));
+                tma_load_2d(base + SM_Q + t * TILE_BYTES + HALF_BYTES, &map_q, h * TILE + 64, tb * TILE, bar(BAR_Q));
+            }
+            bool alive = true;
+            for (int j = 0; j < n_j && alive; ++j) {
+                const int st = j % KV_STAGES, use = j / KV_STAGES;
+                int seg, local, n_valid;
+                kv_tile_info(P, jt0 + j, seg, local, n_valid);
+                const CUtensorMap *mv = seg == 0 ? &map_v0 : (seg == 1 ? &map_v1 : &map_v2);
+                if (use > 0) alive = mbar_wait(bar(BAR_KEMPTY + st), (use - 1) & 1, abort_flag, P.status);
+                if (!alive) break;
+                mbar_expect_tx(bar(BAR_KFULL + st), TILE_BYTES);
+                tma_load_2d(base + SM_K + st * TILE_BYTES, &map_k, g * TILE, (jt0 + j) * TILE, bar(BAR_KFULL + st));
+                tma_load_2d(base + SM_K + st * TILE_BYTES + HALF_BYTES, &map_k, g * TILE + 64, (jt0 + j) * TILE, bar(BAR_KFULL + st));
+                if (use > 0) alive = mbar_wait(bar(BAR_VEMPTY + st), (use - 1) & 1, abort_flag, P.status);
+                if (!alive) break;
+                mbar_expect_tx(bar(BAR_VFULL + st), TILE_BYTES);
+                tma_load_2d(base + SM_V + st * TILE_BYTES, mv, g * TILE, local * TILE, bar(BAR_VFULL + st));
+                tma_load_2d(base + SM_V + st * TILE_BYTES + HALF_BYTES, mv, g * TILE + 64, local * TILE, bar(BAR_VFULL + st));
+            }
+            if (*abort_flag) {
+                // give the copies already issued a bounded chance to land before the CTA's shared memory goes away
+                const uint64_t t0 = global_ns();
+                while (global_ns() - t0 < 2000000ull) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            bool alive = mbar_wait(bar(BAR_Q), 0, abort_flag, P.status);
+            auto issue_qk = [&](int t, int st) {
+                const uint32_t qa = base + SM_Q + t * TILE_BYTES, ka = base + SM_K + st * TILE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                    mma_ss(tmem + t * TILE, desc_kmajor(qa + off), desc_kmajor(ka + off), IDESC_QK, ks > 0);
+                }
+            };
+            if (alive && n_j > 0) alive = mbar_wait(bar(BAR_KFULL + 0), 0, abort_flag, P.status);
+            if (alive && n_j > 0) {
+                tc_fence_after();
+                for (int t = 0; t < n_tiles_q; ++t) {
+                    issue_qk(t, 0);
+                    tc_commit(bar(BAR_SFULL + t));
+                }
+                tc_commit(bar(BAR_KEMPTY + 0));
+            }
+            for (int j = 0; j < n_j && alive; ++j) {
+                const int st = j % KV_STAGES, use = j / KV_STAGES;
+                const int nst = (j + 1) % KV_STAGES, nuse = (j + 1) / KV_STAGES;
+                alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status);
+                if (alive && j + 1 < n_j) alive = mbar_wait(bar(BAR_KFULL + nst), nuse & 1, abort_flag, P.status);
+                for (int t = 0; t < n_tiles_q && alive; ++t) {
+                    alive = mbar_wait(bar(BAR_PFULL + t), j & 1, abort_flag, P.status);
+                    if (!alive) break;
+                    tc_fence_after();
+                    const uint32_t va = base + SM_V + st * TILE_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)   // 16 keys per step: P columns advance by 8 (two bf16 per column)
+                        mma_ts(tmem + 256 + t * TILE, tmem + t * TILE + ks * 8, desc_mnmajor(va + ks * 2048), IDESC_PV,
+                               (j > 0 || ks > 0));
+                    if (j + 1 < n_j) issue_qk(t, nst);
+                    tc_commit(bar(BAR_SFULL + t));          // S_t(j+1) ready, or after the last tile: O_t final
+                }
+                if (alive) {
+                    tc_commit(bar(BAR_VEMPTY + st));
+                    if (j + 1 < n_j) tc_commit(bar(BAR_KEMPTY + nst));
+                }
+            }
+            // make sure nothing of ours is still running on the tensor core before TMEM is freed
+            tc_commit(bar(BAR_DONE));
+            mbar_wait(bar(BAR_DONE), 0, abort_flag, P.status);
+        }
+    } else if (warp >= 4) {
+        // ---------------------------------------------------------------- softmax + correction + epilogue
+        const int t = (warp - 4) >> 2;
+        const int quad = warp & 3;                       // TMEM lane quadrant this warp may touch
+        const int r = quad * 32 + lane;                  // row of the tile
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const uint32_t s_addr = tmem + lane_addr + t * TILE;
+        const uint32_t o_addr = tmem + lane_addr + 256 + t * TILE;
+        float m_used = -INFINITY, l = 0.f;
+        bool alive = t < n_tiles_q;
+        for (int j = 0; j < n_j && alive; ++j) {
+            int seg, local, n_valid;
+            kv_tile_info(P, jt0 + j, seg, local, n_valid);
+            alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), j & 1, abort_flag, P.status));
+            if (!alive) break;
+            tc_fence_after();
+            uint32_t v[32];
+            // pass 1: row maximum
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                tmem_ld32(s_addr + c * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float x = (c * 32 + i < n_valid) ? __uint_as_float(v[i]) : -INFINITY;
+                    mx = fmaxf(mx, x);
+                }
+            }
+            // lazy rescale: move the reference maximum only when it grew by more than the threshold
+            const bool grow = mx > m_used + RESCALE_THRESHOLD;
+            if (__any_sync(0xffffffffu, grow)) {
+                const float m_new = fmaxf(m_used, mx);
+                const float corr = fast_exp2(m_used - m_new);       // 0 on the first tile (m_used = -inf)
+                l *= corr;
+                if (j > 0) {
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        tmem_ld32(o_addr + c * 32, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
+                        tmem_st32(o_addr + c * 32, v);
+                    }
+                }
+                m_used = m_new;
+            }
+            // pass 2: p = 2^(s - m), written as bf16 over the S columns
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                tmem_ld32(s_addr + c * 32, v);
+                tmem_wait_ld();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float p0 = fast_exp2(__uint_as_float(v[2 * i]) - m_used);
+                    float p1 = fast_exp2(__uint_as_float(v[2 * i + 1]) - m_used);
+                    if (c * 32 + 2 * i >= n_valid) p0 = 0.f;
+                    if (c * 32 + 2 * i + 1 >= n_valid) p1 = 0.f;
+                    l += p0 + p1;
+                    pk[i] = pc_pack_bf16(p0, p1);
+                }
+                tmem_st16(s_addr + c * 16, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(BAR_PFULL + t));
+        }
+        // epilogue: O_t is final once the last PV has committed
+        if (alive && n_j > 0) alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), n_j & 1, abort_flag, P.status));
+        if (alive && n_j > 0) {
+            tc_fence_after();
+            const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
+            const int row = tb * TILE + r;
+            uint32_t v[32];
+            if (P.n_splits == 1) {
+                const float inv = 1.f / l;
+                __nv_bfloat16 *orow = P.out + ((size_t)row * P.n_q_heads + h) * TILE;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    tmem_ld32(o_addr + c * 32, v);
+                    tmem_wait_ld();
+                    if (row < P.n_q) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 w;
+                            w.x = pc_pack_bf16(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
+                            w.y = pc_pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
+                            w.z = pc_pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
+                            w.w = pc_pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(orow + c * 32 + i * 8) = w;
+                        }
+                    }
+                }
+                if (P.lse && row < P.n_q) P.lse[(size_t)row * P.n_q_heads + h] = (m_used + log2f(l)) * 0.6931471805599453f;
+            } else {
+                const size_t slot = ((size_t)blockIdx.x * 2 + t) * TILE + r;
+                float *prow = P.part_o + slot * TILE;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    tmem_ld32(o_addr + c * 32, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        *reinterpret_cast<uint4 *>(prow + c * 32 + i * 4) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                }
+                *reinterpret_cast<float2 *>(P.part_ml + slot * 2) = make_float2(m_used, l);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ combine
+// One warp per (query row, head): merges the KV ranges' partials in range order.
+__global__ void __launch_bounds__(256) k_combine(const TcParams P) {
+    const int lane = threadIdx.x & 31;
+    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (w >= P.n_q * P.n_q_heads) return;
+    const int row = w / P.n_q_heads, h = w % P.n_q_heads;
+    const int g = h / P.group, T = (row / TILE) * P.group + h % P.group;
+    const int item = g * P.pairs_per_g + T / 2, t = T & 1, r = row % TILE;
+    float m = -INFINITY;
+    for (int s = 0; s < P.n_splits; ++s) {
+        const size_t slot = ((size_t)(item * P.n_splits + s) * 2 + t) * TILE + r;
+        m = fmaxf(m, __ldcg(P.part_ml + slot * 2));
+    }
+    float l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < P.n_splits; ++s) {
+        const size_t slot = ((size_t)(item * P.n_splits + s) * 2 + t) * TILE + r;
+        const float2 ml = __ldcg(reinterpret_cast<const float2 *>(P.part_ml + slot * 2));
+        const float sc = exp2f(ml.x - m);
+        const float4 o = __ldcg(reinterpret_cast<const float4 *>(P.part_o + slot * TILE) + lane);
+        l = fmaf(ml.y, sc, l);
+        acc.x = fmaf(o.x, sc, acc.x); acc.y = fmaf(o.y, sc, acc.y); acc.z = fmaf(o.z, sc, acc.z); acc.w = fmaf(o.w, sc, acc.w);
+    }
+    const float inv = 1.f / l;
+    uint2 out = make_uint2(pc_pack_bf16(acc.x * inv, acc.y * inv), pc_pack_bf16(acc.z * inv, acc.w * inv));
+    *reinterpret_cast<uint2 *>(P.out + ((size_t)row * P.n_q_heads + h) * TILE + lane * 4) = out;
+    if (P.lse && lane == 0) P.lse[(size_t)row * P.n_q_heads + h] = (m + log2f(l)) * 0.6931471805599453f;
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [rows][cols] bf16 row-major, box = 128 rows x 64 columns, 128-byte swizzle, out-of-range rows read as zero
+bool make_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, TILE};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int div_up(int a, int b) { return (a + b - 1) / b; }
+
+// number of KV ranges: fewest waves of CTAs, a fixed cost per CTA standing in for prologue and epilogue
+int choose_splits(int n_items, int n_kv_tiles, int sm_count) {
+    int best = 1;
+    long best_cost = -1;
+    for (int s = 1; s <= MAX_SPLITS && s <= n_kv_tiles; ++s) {
+        const long waves = div_up(n_items * s, sm_count);
+        const long cost = waves * (div_up(n_kv_tiles, s) + 3) + (s > 1 ? 2 : 0);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    return best;
+}
+
+}  // namespace
+
 pc_status pc_attend_tc_scratch(const pc_layer_desc *d, int sm_count, size_t *k_rot_rows, size_t *part_o_floats,
                                size_t *part_ml_floats) {
-    *k_rot_rows = 1; *part_o_floats = 1; *part_ml_floats = 1;
+    (void)sm_count;
+    // every segment starts on a tile boundary; the query rows follow the keys in the same scratch
+    *k_rot_rows = (size_t)(div_up(d->max_keys, TILE) + PC_MAX_SEGMENTS) * TILE;
+    const int group = d->n_q_heads / d->n_kv_heads;
+    const int n_items = d->n_kv_heads * div_up(group * div_up(d->max_q, TILE), 2);
+    *part_o_floats = (size_t)n_items * MAX_SPLITS * 2 * TILE * TILE;
+    *part_ml_floats = (size_t)n_items * MAX_SPLITS * 2 * TILE * 2;
     return PC_OK;
 }
+
 pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
                               int32_t n_q, void *out, float *lse, cudaStream_t stream) {
-    return pc_launch_attend_simt(ctx, n_seg, segs, q, q_pos, n_q, out, lse, stream);
+    const pc_layer_desc &D = ctx->desc;
+    if (D.head_dim != TILE || D.dtype != PC_BF16) return PC_ERR_UNSUPPORTED;
+    const int row_elems = D.n_kv_heads * D.head_dim;
+    __nv_bfloat16 *k_rot = static_cast<__nv_bfloat16 *>(ctx->k_rot);
+
+    TcParams P{};
+    RopeJobs jobs{};
+    int tiles = 0, warps = 0;
+    for (int s = 0; s < n_seg; ++s) {
+        jobs.job[s] = RopeJob{static_cast<const __nv_bfloat16 *>(segs[s].k), segs[s].pos,
+                              k_rot + (size_t)tiles * TILE * row_elems, segs[s].n_tokens, row_elems / 8, warps, 1.0f};
+        warps += segs[s].n_tokens;
+        tiles += div_up(segs[s].n_tokens, TILE);
+        P.seg_tile_end[s] = tiles;
+        P.seg_n[s] = segs[s].n_tokens;
+    }
+    if ((size_t)tiles * TILE > ctx->k_rot_rows) return PC_ERR_CAPACITY;
+    __nv_bfloat16 *q_rot = static_cast<__nv_bfloat16 *>(ctx->q_rot);
+    jobs.job[n_seg] = RopeJob{static_cast<const __nv_bfloat16 *>(q), q_pos, q_rot, n_q, D.n_q_heads * D.head_dim / 8, warps,
+                              (float)(1.4426950408889634 / std::sqrt((double)D.head_dim))};
+    warps += n_q;
+    jobs.n_jobs = n_seg + 1;
+    jobs.total_warps = warps;
+    k_rope_rows<<<div_up(warps, 8), 256, 0, stream>>>(jobs, ctx->rope, D.head_dim, ctx->status);
+    PC_CUDA_TRY(cudaGetLastError());
+
+    P.n_q = n_q;
+    P.n_q_heads = D.n_q_heads;
+    P.group = ctx->group;
+    P.n_tb = div_up(n_q, TILE);
+    P.tiles_per_g = P.group * P.n_tb;
+    P.pairs_per_g = div_up(P.tiles_per_g, 2);
+    P.n_kv_tiles = tiles;
+    P.n_seg = n_seg;
+    const int n_items = D.n_kv_heads * P.pairs_per_g;
+    P.n_splits = ctx->kv_splits > 0 ? std::min(ctx->kv_splits, tiles) : choose_splits(n_items, tiles, ctx->sm_count);
+    P.out = static_cast<__nv_bfloat16 *>(out);
+    P.lse = lse;
+    P.part_o = ctx->part_o;
+    P.part_ml = ctx->part_ml;
+    P.status = ctx->status;
+    if (P.n_splits > 1 && (size_t)n_items * P.n_splits * 2 * TILE * TILE > ctx->part_o_floats) return PC_ERR_CAPACITY;
+
+    CUtensorMap mq, mk, mv[PC_MAX_SEGMENTS];
+    bool ok = make_map(&mq, q_rot, (uint64_t)n_q, (uint64_t)D.n_q_heads * D.head_dim) &&
+              make_map(&mk, k_rot, (uint64_t)tiles * TILE, (uint64_t)row_elems);
+    for (int s = 0; s < PC_MAX_SEGMENTS; ++s) {
+        const pc_segment &sg = segs[s < n_seg ? s : 0];
+        ok = ok && make_map(&mv[s], sg.v, (uint64_t)sg.n_tokens, (uint64_t)row_elems);
+    }
+    if (!ok) {
+        fprintf(stderr, "packcache: cuTensorMapEncodeTiled failed\n");
+        return PC_ERR_CUDA;
+    }
+    static bool attr_set = false;
+    if (!attr_set) {
+        PC_CUDA_TRY(cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
+        attr_set = true;
+    }
+    k_attend_tc<<<n_items * P.n_splits, TC_THREADS, SM_ALLOC, stream>>>(mq, mk, mv[0], mv[1], mv[2], P);
+    PC_CUDA_TRY(cudaGetLastError());
+    if (P.n_splits > 1) {
+        k_combine<<<div_up(n_q * D.n_q_heads, 8), 256, 0, stream>>>(P);
+        PC_CUDA_TRY(cudaGetLastError());
+    }
+    return PC_OK;
 }

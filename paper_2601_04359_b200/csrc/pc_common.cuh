@@ -57,6 +57,8 @@ struct pc_ctx {
     // attention scratch (tensor-core path)
     void *k_rot;               // rotated keys, bf16 [rows][Hkv][d]
     size_t k_rot_rows;
+    void *q_rot;               // rotated, pre-scaled queries, bf16 [max_q][Hq][d]
+    int kv_splits;             // 0 = chosen per call
     float *part_o;             // split-KV partial outputs
     float *part_ml;            // split-KV partial (max, sum)
     size_t part_o_floats, part_ml_floats;

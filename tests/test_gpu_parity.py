@@ -242,8 +242,8 @@ def test_host_detected_errors():
         pc.pc_compact(ctx, D.cache, sel, budget, 0, D.cache)
     assert e.value.status == pc.PC_ERR_INVALID_ARG
     with pytest.raises(pc.PackCacheError) as e:                   # misaligned query pointer
-        pc.pc_attend_frame(ctx, D.cache, None, D.q.view(-1)[1:1 + 64 * 4 * 64].view(64, 4, 64), D.q_pos,
-                           out=torch.empty_like(D.q))
+        shifted = torch.zeros(D.q.numel() + 4, device="cuda")[1:1 + D.q.numel()].view(D.q.shape)
+        pc.pc_attend_frame(ctx, D.cache, None, shifted, D.q_pos, out=torch.empty_like(D.q))
     assert e.value.status == pc.PC_ERR_INVALID_ARG
     wrong = pc.Cache(D.cache.anchors, D.cache.history, np.array([64] * 5, np.int32))   # frame table does not sum up
     with pytest.raises(pc.PackCacheError) as e:
