@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the PackCache hot path on B200: late-frame attention + compaction latency.
+
+A step is one pass of the whole path for one frame of the 48-frame workload (47 history frames of 1008 tokens,
+1136 anchors, 24 query / 8 KV heads of 128, bf16): plan the per-frame budgets, score the history, select per frame,
+pack the retained rows, and attend the 1008 current-frame queries over anchors ++ packed history.  Steps rotate over
+several layers' K/V (each layer its own seeded tensors, about 0.2 GB per layer) so that every step's inputs come
+from HBM, not from L2.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One JSON line is printed by rank 0.  With --impl reference the CPU oracle is timed instead (bounded samples).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "late_frame_attn_plus_compaction_latency"
+UNIT = "ms/frame"
+WORKLOAD = "lumos47"
+N_LAYERS = 4          # rotated input sets; 4 x ~0.2 GB > L2 (--layers changes it for small profiler captures)
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed regions run."""
+
+    def __init__(self, index: int, uuid: str = ""):
+        self.samples, self.reasons, self.max_mhz, self._stop = [], set(), None, threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if uuid else b"")
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                 "sw_power_cap": 0x4, "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                util = nv.nvmlDeviceGetUtilizationRates(self.h).gpu
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((mhz, util))
+                for n, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        mhz = [m for m, _ in self.samples]
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(mhz)}
+
+
+# --------------------------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(cfg, layer, n_score: int, n_rows: int, s32=None):
+    """Time the oracle on a bounded sample of one frame step and extrapolate to the whole frame.
+    Returns (ms_per_frame, description)."""
+    import oracle
+    L = layer
+    b = cfg.budget
+    rng = np.random.default_rng(0)
+    t0 = time.perf_counter()
+    budget = oracle.plan_budget(b.kind, b.param, b.total, b.keep_full, L.frame_count)
+    t_plan = time.perf_counter() - t0
+    idx = np.sort(rng.choice(cfg.n_src, size=n_score, replace=False))
+    t0 = time.perf_counter()
+    oracle.score(L.hist_k, L.hist_pos, L.q, L.q_pos, cfg.rope_base, idx=idx)
+    t_score = (time.perf_counter() - t0) * (cfg.n_src / n_score)
+    # the remaining stages need all scores: take them from the oracle's pooled form (not timed)
+    if s32 is None:
+        s32 = oracle.score_pooled(L.hist_k, L.hist_pos, L.q, L.q_pos, cfg.rope_base).astype(np.float32)
+    t0 = time.perf_counter()
+    sel = oracle.select(s32, L.frame_count, budget)
+    t_select = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    pk, pv, pp = oracle.pack(L.hist_k, L.hist_v, L.hist_pos, sel, 0)
+    t_pack = time.perf_counter() - t0
+    rows = np.stack([rng.integers(0, cfg.n_q, size=n_rows), rng.integers(0, cfg.n_q_heads, size=n_rows)], axis=1)
+    t0 = time.perf_counter()
+    oracle.attend(L.q, L.q_pos, [(L.anchor_k, L.anchor_v, L.anchor_pos), (pk, pv, pp)], cfg.rope_base,
+                  rows=rows.astype(np.int32))
+    t_att = (time.perf_counter() - t0) * (cfg.n_q * cfg.n_q_heads / n_rows)
+    total = t_plan + t_score + t_select + t_pack + t_att
+    what = (f"{n_score}/{cfg.n_src} tokens scored and {n_rows}/{cfg.n_q * cfg.n_q_heads} attention rows, "
+            f"select and pack in full; scaled to one frame")
+    return total * 1e3, what
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2601_04359_b200 import workload as wl
+    cfg = wl.CONFIGS[WORKLOAD]
+    L = wl.make_layer(cfg, 0)
+    n_iter = args.steps + args.warmup
+    n_score = max(8, min(2000, 12000 // n_iter))
+    n_rows = max(32, min(4096, 24000 // n_iter))
+    s32 = oracle.score_pooled(L.hist_k, L.hist_pos, L.q, L.q_pos, cfg.rope_base).astype(np.float32)
+    vals = []
+    for i in range(n_iter):
+        ms, what = oracle_sample(cfg, L, n_score, n_rows, s32)
+        if i >= args.warmup:
+            vals.append(ms)
+    v = float(np.mean(vals))
+    cores = oracle.max_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": v, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "n_frames": cfg.n_frames, "frame_tokens": cfg.frame_tokens,
+                       "n_anchor": cfg.n_anchor, "retained": cfg.budget.total},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------- CUDA arm
+def run_cuda(args):
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200 import workload as wl
+    from paper_2601_04359_b200.device import DeviceLayer, make_ctx
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pc.load()
+
+    global N_LAYERS
+    N_LAYERS = args.layers
+    cfg = wl.CONFIGS[WORKLOAD]
+    b = cfg.budget
+    # every rank draws its own layers (weak scaling: independent layers, no exchange on the data path)
+    host_layers = [wl.make_layer(cfg, layer=rank * N_LAYERS + i) for i in range(N_LAYERS)]
+    layers = [DeviceLayer(L) for L in host_layers]
+    ctx = make_ctx(cfg)
+    n_sel = b.total
+    dsts = [D.empty_packed(n_sel) for D in layers]
+    scores = torch.empty(cfg.n_src, dtype=torch.float32, device="cuda")
+    sel = torch.empty(n_sel, dtype=torch.int32, device="cuda")
+    out = torch.empty_like(layers[0].q)
+    avail = layers[0].L.frame_count
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        D, dst = layers[i % N_LAYERS], dsts[i % N_LAYERS]
+        budget = pc.pc_plan_budget(b.kind, b.param, b.total, b.keep_full, avail)
+        pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget, scores=scores, sel_idx=sel, stream=stream)
+        pc.pc_compact(ctx, D.cache, sel, budget, 0, dst, stream=stream)
+        pc.pc_attend_frame(ctx, dst, None, D.q, D.q_pos, out=out, stream=stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local, "GPU-" + str(torch.cuda.get_device_properties(local).uuid))
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    assert pc.pc_poll_status(ctx) == pc.PC_OK, "device-side error during warm-up"
+    sampler.start()
+
+    # ---- timed region: K steps, device time between two events on the launching stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    assert pc.pc_poll_status(ctx) == pc.PC_OK, "device-side error in the timed region"
+
+    # ---- per-kernel durations (CUDA events recorded by the library at kernel boundaries, same steps again)
+    pc.pc_set_timing(ctx, True)
+    acc = {k: [] for k in pc.STAGES}
+    for i in range(min(args.steps, 200)):
+        step(i)
+        for k, v in pc.pc_get_timing(ctx).items():
+            if v >= 0:
+                acc[k].append(v)
+    pc.pc_set_timing(ctx, False)
+    kern_ms = {k: (float(np.mean(v)) if v else None) for k, v in acc.items()}
+
+    # ---- end to end from pinned host memory through the host-buffer entry point
+    L0 = host_layers[0]
+    td = torch.bfloat16
+    pin = lambda a, dt=None: (torch.from_numpy(np.ascontiguousarray(a)).to(dt) if dt else
+                              torch.from_numpy(np.ascontiguousarray(a))).pin_memory()
+    hostbuf = {"q": pin(L0.q, td), "q_pos": pin(L0.q_pos), "anchor_k": pin(L0.anchor_k, td),
+               "anchor_v": pin(L0.anchor_v, td), "anchor_pos": pin(L0.anchor_pos), "hist_k": pin(L0.hist_k, td),
+               "hist_v": pin(L0.hist_v, td), "hist_pos": pin(L0.hist_pos), "frame_count": L0.frame_count,
+               "out": torch.empty(L0.q.shape, dtype=td).pin_memory()}
+    ws = {"q": torch.empty_like(layers[0].q), "q_pos": torch.empty_like(layers[0].q_pos), "scores": scores,
+          "sel_idx": sel, "out": out}
+    ws_src = pc.Cache(pc.Segment(torch.empty_like(layers[0].cache.anchors.k), torch.empty_like(layers[0].cache.anchors.v),
+                                 torch.empty_like(layers[0].cache.anchors.pos), 0),
+                      pc.Segment(torch.empty_like(layers[0].cache.history.k), torch.empty_like(layers[0].cache.history.v),
+                                 torch.empty_like(layers[0].cache.history.pos), 0), L0.frame_count)
+    h2d = sum(hostbuf[k].numel() * hostbuf[k].element_size() for k in
+              ("q", "q_pos", "anchor_k", "anchor_v", "anchor_pos", "hist_k", "hist_v", "hist_pos"))
+    d2h = hostbuf["out"].numel() * hostbuf["out"].element_size()
+    n_e2e = max(3, min(args.steps, 20))
+
+    def e2e_step():
+        pc.pc_frame_step_host(ctx, hostbuf, ws_src, dsts[0], ws, b.kind, b.param, b.total, b.keep_full, 0, stream)
+
+    if args.no_e2e:
+        n_e2e = 0
+    for _ in range(2 if n_e2e else 0):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(n_e2e):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(n_e2e, 1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    clocks = sampler.stop()
+    status = pc.pc_poll_status(ctx)
+    assert status == pc.PC_OK, f"device-side status {status}"
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (attention: a dense contraction on the tensor cores)
+    peaks = _peaks()
+    n_keys = cfg.n_anchor + n_sel
+    flops = 4.0 * cfg.n_q * n_keys * cfg.head_dim * cfg.n_q_heads
+    att_ms = kern_ms["attend"]
+    achieved = flops / (att_ms * 1e-3) / 1e12
+    row = cfg.n_kv_heads * cfg.head_dim * 2
+    score_bytes = cfg.n_src * (row + 16 + 4)
+    pack_bytes = n_sel * (4 * row + 32 + 4)
+    hbm = lambda nbytes, ms: (nbytes / (ms * 1e-3) / 1e9) if ms else None
+    stages = {k: (round(v, 5) if v is not None else None) for k, v in kern_ms.items()}
+    line = {
+        "metric": METRIC, "value": ms_step / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "n_frames": cfg.n_frames, "frame_tokens": cfg.frame_tokens,
+                   "n_anchor": cfg.n_anchor, "retained": n_sel, "keys_attended": n_keys, "n_q": cfg.n_q,
+                   "heads": f"{cfg.n_q_heads}q/{cfg.n_kv_heads}kv", "head_dim": cfg.head_dim,
+                   "budget": "2 newest frames whole + 6048 at half-life 4", "mode": "one-shot compaction every frame",
+                   "l2": f"inputs rotate over {N_LAYERS} layers (~{0.2 * N_LAYERS:.1f} GB; L2 is 126 MB)", "parallelism": f"replicas x{world}"},
+        "clocks": clocks,
+        "e2e": {"value": (e2e_ms / world) if n_e2e else None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": n_e2e},
+        "gpu_launches": 7 * args.steps,
+        "roofline": {"kernel": "k_attend_tc", "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                     "peak_source": f"{peaks['source']} (burst; sustained {peaks['bf16_tflops_sustained']})",
+                     "flops_per_launch": flops, "ms_per_launch": att_ms},
+        "kernels_ms": stages,
+        "hbm_kernels": {
+            "score": {"GBps": hbm(score_bytes, kern_ms["score"]), "bytes": score_bytes,
+                      "frac": (hbm(score_bytes, kern_ms["score"]) or 0) / peaks["hbm_gbs"]},
+            "pack": {"GBps": hbm(pack_bytes, kern_ms["pack"]), "bytes": pack_bytes,
+                     "frac": (hbm(pack_bytes, kern_ms["pack"]) or 0) / peaks["hbm_gbs"]},
+            "peak": peaks["hbm_gbs"], "peak_source": peaks["source"]},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        t0 = time.perf_counter()
+        v, what = oracle_sample(cfg, host_layers[0], n_score=2000, n_rows=4096)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+                                "sample": what, "sample_seconds": round(time.perf_counter() - t0, 1)}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--layers", type=int, default=N_LAYERS, help="rotated input sets (default 4, > L2)")
+    args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand with --gpus N: relaunch as one rank per GPU
+        os.execvp(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node",
+                                   str(args.gpus), "--master-addr", "127.0.0.1", "--master-port", "29511"] + sys.argv)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

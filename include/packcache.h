@@ -160,6 +160,37 @@ pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, c
 pc_status pc_attend_frame(pc_ctx *ctx, const pc_cache *cache, const pc_segment *current, const void *q,
                           const int32_t *q_pos, int32_t n_q, void *out, float *lse, void *stream);
 
+/* One frame step with inputs and output in HOST memory (pinned memory keeps the copies asynchronous): copies Q,
+ * positions, anchors and the history frames into the caller's device workspace, plans the budget, scores, selects,
+ * packs and attends (anchors ++ packed history), copies the output back and waits for the stream.  Everything the
+ * four calls above state applies; the workspace capacities bound the sizes (PC_ERR_CAPACITY). */
+typedef struct {
+    const void *q;              /* host [n_q][Hq][d] */
+    const int32_t *q_pos;       /* host [n_q][4] */
+    int32_t n_q;
+    const void *anchor_k, *anchor_v; /* host [n_anchor][Hkv][d] */
+    const int32_t *anchor_pos;  /* host [n_anchor][4] */
+    int32_t n_anchor;
+    const void *hist_k, *hist_v; /* host [sum(frame_count)][Hkv][d] */
+    const int32_t *hist_pos;    /* host [sum(frame_count)][4] */
+    int32_t n_frames;
+    const int32_t *frame_count; /* host [n_frames] */
+    void *out;                  /* host out [n_q][Hq][d] */
+} pc_host_frame;
+
+typedef struct {
+    pc_cache src;     /* device staging for anchors and history (capacities used, counts ignored) */
+    pc_cache dst;     /* device destination of the packed history (its anchors field is ignored) */
+    void *q;          /* device [>= n_q][Hq][d] */
+    int32_t *q_pos;   /* device [>= n_q][4] */
+    float *scores;    /* device [>= history tokens] */
+    int32_t *sel_idx; /* device [>= retained tokens] */
+    void *out;        /* device [>= n_q][Hq][d] */
+} pc_device_workspace;
+
+pc_status pc_frame_step_host(pc_ctx *ctx, const pc_host_frame *in, pc_device_workspace *ws,
+                             const pc_budget_params *params, int32_t delta_t, void *stream);
+
 /* Wait for the stream, then return and clear the first device-side event
  * recorded since the last poll (PC_OK if none). */
 pc_status pc_poll_status(pc_ctx *ctx, void *stream);
@@ -171,6 +202,15 @@ pc_status pc_set_attend_impl(pc_ctx *ctx, int32_t impl);
 /* Fix the number of key ranges the tensor-core attention kernel splits the keys into (1..4); 0 lets each call
  * choose the count that fills the GPU's SMs best.  Results agree up to fp32 rounding order. */
 pc_status pc_set_kv_splits(pc_ctx *ctx, int32_t n);
+
+/* Per-kernel timing for benchmarks.  With timing on, each call records CUDA events on its stream at the boundaries
+ * of its kernels (a few microseconds of overhead per call); pc_get_timing waits for the last recorded events and
+ * writes the duration in milliseconds of each kernel of the most recent calls, -1 for a kernel that did not run.
+ * ms is a host array [PC_N_STAGES]. */
+enum { PC_STAGE_QPOOL = 0, PC_STAGE_SCORE = 1, PC_STAGE_SELECT = 2, PC_STAGE_PACK = 3, PC_STAGE_ROPE = 4,
+       PC_STAGE_ATTEND = 5, PC_STAGE_COMBINE = 6, PC_N_STAGES = 7 };
+pc_status pc_set_timing(pc_ctx *ctx, int32_t on);
+pc_status pc_get_timing(pc_ctx *ctx, float *ms);
 
 const char *pc_status_string(pc_status s);
 

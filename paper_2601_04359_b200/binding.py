@@ -22,7 +22,8 @@ PC_GEOMETRIC, PC_CLOSED_HALF, PC_LINEAR, PC_HALFLIFE = 0, 1, 2, 3
 PC_MAX_FRAMES = 256
 
 EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact", "pc_attend_frame",
-           "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_status_string"]
+           "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_set_timing", "pc_get_timing",
+           "pc_frame_step_host", "pc_status_string"]
 
 
 class pc_layer_desc(C.Structure):
@@ -43,6 +44,21 @@ class pc_cache(C.Structure):
 class pc_budget_params(C.Structure):
     _fields_ = [("kind", C.c_int32), ("param", C.c_double), ("total", C.c_int64), ("keep_full", C.c_int32),
                 ("min_quota", C.c_int32)]
+
+
+class pc_host_frame(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("q_pos", C.c_void_p), ("n_q", C.c_int32), ("anchor_k", C.c_void_p),
+                ("anchor_v", C.c_void_p), ("anchor_pos", C.c_void_p), ("n_anchor", C.c_int32), ("hist_k", C.c_void_p),
+                ("hist_v", C.c_void_p), ("hist_pos", C.c_void_p), ("n_frames", C.c_int32),
+                ("frame_count", C.POINTER(C.c_int32)), ("out", C.c_void_p)]
+
+
+class pc_device_workspace(C.Structure):
+    _fields_ = [("src", pc_cache), ("dst", pc_cache), ("q", C.c_void_p), ("q_pos", C.c_void_p), ("scores", C.c_void_p),
+                ("sel_idx", C.c_void_p), ("out", C.c_void_p)]
+
+
+STAGES = ["qpool", "score", "select", "pack", "rope", "attend", "combine"]
 
 
 class PackCacheError(RuntimeError):
@@ -78,6 +94,10 @@ def load() -> C.CDLL:
     lib.pc_poll_status.argtypes = [C.c_void_p, C.c_void_p]
     lib.pc_set_attend_impl.argtypes = [C.c_void_p, C.c_int32]
     lib.pc_set_kv_splits.argtypes = [C.c_void_p, C.c_int32]
+    lib.pc_set_timing.argtypes = [C.c_void_p, C.c_int32]
+    lib.pc_get_timing.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
+    lib.pc_frame_step_host.argtypes = [C.c_void_p, C.POINTER(pc_host_frame), C.POINTER(pc_device_workspace),
+                                       C.POINTER(pc_budget_params), C.c_int32, C.c_void_p]
     _lib = lib
     return lib
 
@@ -224,3 +244,30 @@ def pc_set_attend_impl(ctx: Context, impl: int) -> None:
 
 def pc_set_kv_splits(ctx: Context, n: int) -> None:
     _check(load().pc_set_kv_splits(ctx.handle, n), "pc_set_kv_splits")
+
+
+def pc_set_timing(ctx: Context, on: bool) -> None:
+    _check(load().pc_set_timing(ctx.handle, 1 if on else 0), "pc_set_timing")
+
+
+def pc_get_timing(ctx: Context) -> dict:
+    """Milliseconds of each kernel of the most recent calls (see STAGES); -1 for a kernel that did not run."""
+    ms = (C.c_float * len(STAGES))()
+    _check(load().pc_get_timing(ctx.handle, ms), "pc_get_timing")
+    return {name: float(ms[i]) for i, name in enumerate(STAGES)}
+
+
+def pc_frame_step_host(ctx: Context, host: dict, ws_src: Cache, ws_dst: Cache, ws: dict, kind: int, param: float,
+                       total: int, keep_full: int, delta_t: int = 0, stream=None) -> None:
+    """host: pinned CPU tensors q, q_pos, anchor_k, anchor_v, anchor_pos, hist_k, hist_v, hist_pos, out and the numpy
+    frame_count; ws: device tensors q, q_pos, scores, sel_idx, out.  Blocks until the output is in host['out']."""
+    fc = _i32(host["frame_count"])
+    hf = pc_host_frame(_ptr(host["q"]), _ptr(host["q_pos"]), host["q"].shape[0], _ptr(host["anchor_k"]),
+                       _ptr(host["anchor_v"]), _ptr(host["anchor_pos"]), host["anchor_k"].shape[0],
+                       _ptr(host["hist_k"]), _ptr(host["hist_v"]), _ptr(host["hist_pos"]), len(fc), _i32p(fc),
+                       _ptr(host["out"]))
+    w = pc_device_workspace(ws_src.c(), ws_dst.c(), _ptr(ws["q"]), _ptr(ws["q_pos"]), _ptr(ws["scores"]),
+                            _ptr(ws["sel_idx"]), _ptr(ws["out"]))
+    p = pc_budget_params(kind, param, total, keep_full, 0)
+    _check(load().pc_frame_step_host(ctx.handle, C.byref(hf), C.byref(w), C.byref(p), delta_t, _stream(stream)),
+           "pc_frame_step_host")

@@ -51,6 +51,9 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
     c->elem_size = desc->dtype == PC_BF16 ? 2 : 4;
     c->attend_impl = 0;
     c->kv_splits = 0;
+    c->timing_on = 0;
+    c->ev_mask = 0;
+    for (int i = 0; i < PC_N_MARKS; ++i) c->ev[i] = nullptr;
     PC_CUDA_TRY(cudaGetDevice(&c->device));
     PC_CUDA_TRY(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
 
@@ -106,6 +109,8 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
     cudaFree(c->qpool_partial);
     cudaFree(c->qpool);
     cudaFree(c->ticket);
+    for (int i = 0; i < PC_N_MARKS; ++i)
+        if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     cudaFree(c->k_rot);
     cudaFree(c->q_rot);
     cudaFree(c->part_o);
@@ -123,6 +128,32 @@ extern "C" pc_status pc_set_attend_impl(pc_ctx *c, int32_t impl) {
 extern "C" pc_status pc_set_kv_splits(pc_ctx *c, int32_t n) {
     if (!c || n < 0 || n > 4) return PC_ERR_INVALID_ARG;
     c->kv_splits = n;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_set_timing(pc_ctx *c, int32_t on) {
+    if (!c) return PC_ERR_INVALID_ARG;
+    if (on)
+        for (int i = 0; i < PC_N_MARKS; ++i)
+            if (!c->ev[i]) PC_CUDA_TRY(cudaEventCreate(&c->ev[i]));
+    c->timing_on = on ? 1 : 0;
+    c->ev_mask = 0;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_get_timing(pc_ctx *c, float *ms) {
+    if (!c || !ms) return PC_ERR_INVALID_ARG;
+    static const int span[PC_N_STAGES][2] = {{PC_MARK_SCORE0, PC_MARK_QPOOL}, {PC_MARK_QPOOL, PC_MARK_SCORE},
+                                             {PC_MARK_SCORE, PC_MARK_SELECT}, {PC_MARK_PACK0, PC_MARK_PACK},
+                                             {PC_MARK_ATT0, PC_MARK_ROPE},    {PC_MARK_ROPE, PC_MARK_ATTEND},
+                                             {PC_MARK_ATTEND, PC_MARK_COMBINE}};
+    for (int s = 0; s < PC_N_STAGES; ++s) {
+        ms[s] = -1.f;
+        const int a = span[s][0], b = span[s][1];
+        if (!((c->ev_mask >> a) & 1u) || !((c->ev_mask >> b) & 1u)) continue;
+        PC_CUDA_TRY(cudaEventSynchronize(c->ev[b]));
+        PC_CUDA_TRY(cudaEventElapsedTime(&ms[s], c->ev[a], c->ev[b]));
+    }
     return PC_OK;
 }
 

@@ -158,6 +158,7 @@ pc_status pc_launch_attend_simt(pc_ctx *ctx, int n_seg, const pc_segment *segs, 
     }
     t.n_keys = total;
     dim3 grid((n_q + AT_ROWS - 1) / AT_ROWS, D.n_q_heads);
+    pc_mark(ctx, PC_MARK_ROPE, stream);
 #define PC_AT_LAUNCH(T, DIM)                                                                                          \
     k_attend_simt<T, DIM><<<grid, AT_THREADS, 0, stream>>>(static_cast<const T *>(q), q_pos, n_q, D.n_q_heads,         \
                                                           D.n_kv_heads, t, ctx->rope, static_cast<T *>(out), lse,    \
@@ -169,5 +170,6 @@ pc_status pc_launch_attend_simt(pc_ctx *ctx, int n_seg, const pc_segment *segs, 
     }
 #undef PC_AT_LAUNCH
     PC_CUDA_TRY(cudaGetLastError());
+    pc_mark(ctx, PC_MARK_ATTEND, stream);
     return PC_OK;
 }

@@ -571,8 +571,10 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     warps += n_q;
     jobs.n_jobs = n_seg + 1;
     jobs.total_warps = warps;
+    pc_mark(ctx, PC_MARK_ATT0, stream);
     k_rope_rows<<<div_up(warps, 8), 256, 0, stream>>>(jobs, ctx->rope, D.head_dim, ctx->status);
     PC_CUDA_TRY(cudaGetLastError());
+    pc_mark(ctx, PC_MARK_ROPE, stream);
 
     P.n_q = n_q;
     P.n_q_heads = D.n_q_heads;
@@ -609,9 +611,11 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     }
     k_attend_tc<<<n_items * P.n_splits, TC_THREADS, SM_ALLOC, stream>>>(mq, mk, mv[0], mv[1], mv[2], P);
     PC_CUDA_TRY(cudaGetLastError());
+    pc_mark(ctx, PC_MARK_ATTEND, stream);
     if (P.n_splits > 1) {
         k_combine<<<div_up(n_q * D.n_q_heads, 8), 256, 0, stream>>>(P);
         PC_CUDA_TRY(cudaGetLastError());
+        pc_mark(ctx, PC_MARK_COMBINE, stream);
     }
     return PC_OK;
 }

@@ -28,6 +28,10 @@ enum {
     PC_WHERE_ROPE_POS = 7,
 };
 
+// event marks: score call 0-3, pack 4-5, attend 6-9
+enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT = 3, PC_MARK_PACK0 = 4, PC_MARK_PACK = 5,
+       PC_MARK_ATT0 = 6, PC_MARK_ROPE = 7, PC_MARK_ATTEND = 8, PC_MARK_COMBINE = 9, PC_N_MARKS = 10 };
+
 constexpr int PC_QPOOL_BLOCKS = 64;
 constexpr int PC_MAX_SEGMENTS = 3;
 
@@ -59,6 +63,10 @@ struct pc_ctx {
     size_t k_rot_rows;
     void *q_rot;               // rotated, pre-scaled queries, bf16 [max_q][Hq][d]
     int kv_splits;             // 0 = chosen per call
+    // optional per-kernel timing (benchmarks): events at the boundaries of the kernels of each call
+    int timing_on;
+    unsigned ev_mask;
+    cudaEvent_t ev[PC_N_MARKS];
     float *part_o;             // split-KV partial outputs
     float *part_ml;            // split-KV partial (max, sum)
     size_t part_o_floats, part_ml_floats;
@@ -100,6 +108,10 @@ __device__ __forceinline__ void pc_stg_stream(void *p, uint4 v) {
     asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
                  "r"(v.w)
                  : "memory");
+}
+
+inline void pc_mark(pc_ctx *c, int idx, cudaStream_t s) {
+    if (c->timing_on && c->ev[idx] && cudaEventRecord(c->ev[idx], s) == cudaSuccess) c->ev_mask |= 1u << idx;
 }
 
 // host-side helpers implemented in pc_api.cu

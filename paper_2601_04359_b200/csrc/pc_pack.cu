@@ -88,6 +88,7 @@ extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t 
     const char *sk = static_cast<const char *>(src->history.k), *sv = static_cast<const char *>(src->history.v);
     char *dk = static_cast<char *>(D.k), *dv = static_cast<char *>(D.v);
 #define PC_PACK_ARGS sk, sv, src->history.pos, sel_idx, (int)n_sel, (int)n_src, row_bytes, delta_t, dk, dv, D.pos, ctx->status
+    pc_mark(ctx, PC_MARK_PACK0, stream);
     switch (row_bytes) {
     case 512: k_pack<1><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
     case 1024: k_pack<2><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
@@ -96,5 +97,6 @@ extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t 
     }
 #undef PC_PACK_ARGS
     PC_CUDA_TRY(cudaGetLastError());
+    pc_mark(ctx, PC_MARK_PACK, stream);
     return PC_OK;
 }

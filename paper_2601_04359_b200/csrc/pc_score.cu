@@ -258,10 +258,12 @@ pc_status launch_score(pc_ctx *ctx, const pc_cache *src, const void *q, const in
     const size_t smem = (size_t)D.n_q_heads * D.head_dim * sizeof(float);
     if (smem > 48 * 1024)
         PC_CUDA_TRY(cudaFuncSetAttribute(k_qpool<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    pc_mark(ctx, PC_MARK_SCORE0, stream);
     k_qpool<T><<<pool_blocks, 256, smem, stream>>>(static_cast<const T *>(q), q_pos, n_q, D.n_q_heads, ctx->group,
                                                    D.head_dim, ctx->rope, ctx->qpool_partial, ctx->qpool, ctx->ticket,
                                                    ctx->status);
     PC_CUDA_TRY(cudaGetLastError());
+    pc_mark(ctx, PC_MARK_QPOOL, stream);
     const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
     const int chunks = row / Elem<T>::PER16;          // 16-byte chunks per token row
     const int warps_needed = (n_src + 1) / 2;
@@ -279,6 +281,7 @@ pc_status launch_score(pc_ctx *ctx, const pc_cache *src, const void *q, const in
     }
 #undef PC_SCORE_CASE
     PC_CUDA_TRY(cudaGetLastError());
+    pc_mark(ctx, PC_MARK_SCORE, stream);
     return PC_OK;
 }
 
@@ -324,8 +327,10 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
         return PC_ERR_INVALID_ARG;
     }
     if (n_frames > 0 && out > 0) {
+        if (scores_override) pc_mark(ctx, PC_MARK_SCORE, stream);
         k_select<<<n_frames, SEL_THREADS, 0, stream>>>(select_on, tab, sel_idx, ctx->status);
         PC_CUDA_TRY(cudaGetLastError());
+        pc_mark(ctx, PC_MARK_SELECT, stream);
     }
     return PC_OK;
 }

@@ -1,11 +1,12 @@
-"""Helpers for the GPU parity tests: move a seeded workload to the device and wrap it for the binding."""
+"""Device-side plumbing shared by the tests, the smoke check and the benchmark: move a seeded workload into GPU
+memory (PyTorch tensors) and wrap it in the binding's Segment / Cache records.  No arithmetic of the method here."""
 from __future__ import annotations
 
 import numpy as np
 import torch
 
-from paper_2601_04359_b200 import binding as pc
-from paper_2601_04359_b200 import workload as wl
+from . import binding as pc
+from . import workload as wl
 
 
 def dev(x: np.ndarray, dtype: str) -> torch.Tensor:

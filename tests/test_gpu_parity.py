@@ -12,7 +12,7 @@ import torch
 import oracle
 from paper_2601_04359_b200 import binding as pc
 from paper_2601_04359_b200 import workload as wl
-from tests.gpu_util import DeviceLayer, dev, host, idev, make_ctx, score_tolerance, segment
+from paper_2601_04359_b200.device import DeviceLayer, dev, host, idev, make_ctx, score_tolerance, segment
 
 pytestmark = pytest.mark.gpu
 
