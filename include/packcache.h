@@ -191,6 +191,31 @@ typedef struct {
 pc_status pc_frame_step_host(pc_ctx *ctx, const pc_host_frame *in, pc_device_workspace *ws,
                              const pc_budget_params *params, int32_t delta_t, void *stream);
 
+/* Scoring for callers that cannot allocate.  (The paper has no counterpart: this entry point exists for the sake of
+ * host programs, not of the method.)  Some hosts cannot call cudaMalloc where they need scores — their device memory
+ * was given to an arena of their own at start-up and driver allocations are forbidden afterwards, or they sit on a
+ * latency-critical thread that cannot take the device-wide synchronisation an allocation or a free implies — and so
+ * cannot create a pc_ctx either.  This call needs no context and calls neither cudaMalloc nor cudaFree nor any
+ * allocating routine: the rotary table, the pooled query and its reduction scratch live in one fixed device array
+ * of 528,640 bytes that is part of the library image (every GPU that loads the library holds it until exit).
+ *
+ * Computes the same scores as pc_score (mean scaled rotary logit of every history token over the n_q queries and
+ * all query heads, fp32); selection is not included.  desc->max_q / max_keys are ignored.
+ *   hist_k device [n_src][Hkv][d]; hist_pos device [n_src][4]; q device [n_q][Hq][d]; q_pos device [n_q][4];
+ *   valid device [n_src] bytes or NULL; scores device out [n_src] fp32;
+ *   status device [2] int32, zeroed by the caller: receives (PC_ERR_INVALID_ARG, where) if a position lies outside
+ *   desc->max_pos (the position is clamped and the call completes); the caller copies it back when it wants it.
+ * Limits (PC_ERR_CAPACITY with a message on stderr beyond them): n_kv_heads*head_dim <= 1024;
+ * sum over the three axes of max_pos[a] * (rotary pairs on axis a) <= 32768; n_q_heads*head_dim <= 12288.
+ * The first call on each device looks up the array's device address (that device must be current); make that
+ * first call outside any stream capture.  All calls share the one array, which keeps the previous call's
+ * contents (the call rewrites or clears what it relies on): two calls that may overlap on the GPU — different
+ * streams without an ordering between them — race; order them.  Work is asynchronous on the given stream.
+ * Other errors: PC_ERR_INVALID_ARG (null or misaligned pointer, n_src or n_q <= 0), PC_ERR_UNSUPPORTED, PC_ERR_CUDA. */
+pc_status pc_score_tokens_static(const pc_layer_desc *desc, const void *hist_k, const int32_t *hist_pos,
+                                 int32_t n_src, const void *q, const int32_t *q_pos, int32_t n_q,
+                                 const uint8_t *valid, float *scores, int32_t *status, void *stream);
+
 /* Wait for the stream, then return and clear the first device-side event
  * recorded since the last poll (PC_OK if none). */
 pc_status pc_poll_status(pc_ctx *ctx, void *stream);

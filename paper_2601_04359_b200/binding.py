@@ -23,7 +23,7 @@ PC_MAX_FRAMES = 256
 
 EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact", "pc_attend_frame",
            "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_set_timing", "pc_get_timing",
-           "pc_frame_step_host", "pc_status_string"]
+           "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static"]
 
 
 class pc_layer_desc(C.Structure):
@@ -98,6 +98,8 @@ def load() -> C.CDLL:
     lib.pc_get_timing.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
     lib.pc_frame_step_host.argtypes = [C.c_void_p, C.POINTER(pc_host_frame), C.POINTER(pc_device_workspace),
                                        C.POINTER(pc_budget_params), C.c_int32, C.c_void_p]
+    lib.pc_score_tokens_static.argtypes = [C.POINTER(pc_layer_desc), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                           C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     _lib = lib
     return lib
 
@@ -271,3 +273,14 @@ def pc_frame_step_host(ctx: Context, host: dict, ws_src: Cache, ws_dst: Cache, w
     p = pc_budget_params(kind, param, total, keep_full, 0)
     _check(load().pc_frame_step_host(ctx.handle, C.byref(hf), C.byref(w), C.byref(p), delta_t, _stream(stream)),
            "pc_frame_step_host")
+
+
+def pc_score_tokens_static(desc: pc_layer_desc, hist_k: torch.Tensor, hist_pos: torch.Tensor, n_src: int,
+                           q: torch.Tensor, q_pos: torch.Tensor, scores: torch.Tensor, status: torch.Tensor,
+                           valid: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Context-free scoring that allocates nothing: every buffer, including the [n_src] fp32 ``scores`` output and the
+    zeroed [2] int32 ``status`` word, is the caller's; the library's scratch is a fixed device array."""
+    _check(load().pc_score_tokens_static(C.byref(desc), _ptr(hist_k), _ptr(hist_pos), n_src, _ptr(q), _ptr(q_pos),
+                                         q.shape[0], _ptr(valid), _ptr(scores), _ptr(status), _stream(stream)),
+           "pc_score_tokens_static")
+    return scores

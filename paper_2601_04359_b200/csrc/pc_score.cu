@@ -334,3 +334,151 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
     }
     return PC_OK;
 }
+
+// ---------------------------------------------------------------------------------------------------------
+// Scoring without a context and without any allocation.
+//
+// Meant for hosts that cannot call cudaMalloc at the point where they need scores: a process whose device memory
+// was handed to its own arena at start-up and whose policy forbids driver allocations afterwards, or a
+// latency-critical thread that cannot take the device-wide synchronisation a cudaMalloc / cudaFree implies.  Such
+// callers cannot create a pc_ctx (pc_create allocates), so everything a context would hold for scoring — the rotary
+// table, the pooled query and its per-block partials, the completion ticket — lives in one file-scope device array
+// of fixed size that every GPU loading this library carries until the process exits.
+//
+// In host code the array's name is only a handle; the device address is obtained once per device with
+// cudaGetSymbolAddress while that device is current, and that pointer (never the symbol) is what kernels receive.
+// ---------------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int STATIC_MAX_ROW = 1024;          // n_kv_heads * head_dim
+constexpr int STATIC_MAX_ROPE = 32768;        // rotary table entries: sum over axes of max_pos * pairs on that axis
+constexpr int STATIC_MAX_DEVICES = 64;
+
+constexpr size_t STATIC_OFF_TICKET = 0;                                                    // unsigned, 256-byte slot
+constexpr size_t STATIC_OFF_POOLED = 256;                                                  // float [STATIC_MAX_ROW]
+constexpr size_t STATIC_OFF_PARTIAL = STATIC_OFF_POOLED + STATIC_MAX_ROW * sizeof(float);  // float [64][STATIC_MAX_ROW]
+constexpr size_t STATIC_OFF_ROPE = STATIC_OFF_PARTIAL + (size_t)PC_QPOOL_BLOCKS * STATIC_MAX_ROW * sizeof(float);
+constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);   // 528,640 bytes
+
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
+
+// Rotary table in fp64, stored as fp32 (cos, sin): entry (axis a, position p, column m) = p * base^(-m / n_axis[a]).
+__global__ void __launch_bounds__(256) k_rope_table(float2 *__restrict__ tab, pc_rope_dev rope, double base, int total) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const int a = e >= rope.off[2] ? 2 : (e >= rope.off[1] ? 1 : 0);
+    const int na = rope.n_axis[a], local = e - rope.off[a];
+    const int p = local / na, m = local % na;
+    const double ang = (double)p * pow(base, -(double)m / (double)na);
+    tab[e] = make_float2((float)cos(ang), (float)sin(ang));
+}
+
+// Device address of the static scratch on the current device; looked up on the first call per device.
+pc_status static_scratch_base(unsigned char **base) {
+    static unsigned char *addr[STATIC_MAX_DEVICES] = {};
+    int dev = -1;
+    PC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return PC_ERR_UNSUPPORTED;
+    unsigned char *p = __atomic_load_n(&addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        void *sym = nullptr;
+        PC_CUDA_TRY(cudaGetSymbolAddress(&sym, g_static_scratch));
+        if (!sym) return PC_ERR_CUDA;
+        p = static_cast<unsigned char *>(sym);
+        __atomic_store_n(&addr[dev], p, __ATOMIC_RELEASE);   // every thread resolves the same address
+    }
+    *base = p;
+    return PC_OK;
+}
+
+template <typename T>
+pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const void *hist_k, const int32_t *hist_pos,
+                              int32_t n_src, const void *q, const int32_t *q_pos, int32_t n_q, const uint8_t *valid,
+                              float *scores, int32_t *status, cudaStream_t stream) {
+    unsigned int *ticket = reinterpret_cast<unsigned int *>(base + STATIC_OFF_TICKET);
+    float *pooled = reinterpret_cast<float *>(base + STATIC_OFF_POOLED);
+    float *partial = reinterpret_cast<float *>(base + STATIC_OFF_PARTIAL);
+    float2 *tab = reinterpret_cast<float2 *>(base + STATIC_OFF_ROPE);
+
+    pc_rope_dev rope;
+    int total = 0;
+    for (int a = 0; a < 3; ++a) {
+        rope.n_axis[a] = (D.head_dim / 2 - a + 2) / 3;
+        rope.max_pos[a] = D.max_pos[a];
+        rope.off[a] = total;
+        total += D.max_pos[a] * rope.n_axis[a];
+    }
+    rope.tab = tab;
+    // the array keeps whatever the last call left: the ticket must start at zero, the table is rewritten
+    PC_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), stream));
+    k_rope_table<<<(total + 255) / 256, 256, 0, stream>>>(tab, rope, D.rope_base, total);
+    PC_CUDA_TRY(cudaGetLastError());
+
+    const int row = D.n_kv_heads * D.head_dim;
+    const int pool_blocks = std::min<int>(PC_QPOOL_BLOCKS, n_q);
+    const size_t smem = (size_t)D.n_q_heads * D.head_dim * sizeof(float);
+    k_qpool<T><<<pool_blocks, 256, smem, stream>>>(static_cast<const T *>(q), q_pos, n_q, D.n_q_heads,
+                                                   D.n_q_heads / D.n_kv_heads, D.head_dim, rope, partial, pooled, ticket,
+                                                   status);
+    PC_CUDA_TRY(cudaGetLastError());
+    const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
+    const int chunks = row / Elem<T>::PER16;
+    const int warps_needed = (n_src + 1) / 2;
+    int sm_count = 0, dev = 0;
+    PC_CUDA_TRY(cudaGetDevice(&dev));
+    PC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    const int blocks = std::max(1, std::min((warps_needed + 7) / 8, sm_count * 6));
+    const T *k = static_cast<const T *>(hist_k);
+#define PC_SCORE_CASE(CPL)                                                                                         \
+    case CPL:                                                                                                      \
+        k_score<T, CPL><<<blocks, 256, 0, stream>>>(k, hist_pos, valid, n_src, D.head_dim, scale, rope, pooled, scores, \
+                                                    status);                                                      \
+        break;
+    switch (chunks / 32) {
+        PC_SCORE_CASE(1) PC_SCORE_CASE(2) PC_SCORE_CASE(3) PC_SCORE_CASE(4) PC_SCORE_CASE(6) PC_SCORE_CASE(8)
+    default: return PC_ERR_UNSUPPORTED;
+    }
+#undef PC_SCORE_CASE
+    PC_CUDA_TRY(cudaGetLastError());
+    return PC_OK;
+}
+
+}  // namespace
+
+extern "C" pc_status pc_score_tokens_static(const pc_layer_desc *desc, const void *hist_k, const int32_t *hist_pos,
+                                            int32_t n_src, const void *q, const int32_t *q_pos, int32_t n_q,
+                                            const uint8_t *valid, float *scores, int32_t *status, void *stream_) {
+    if (!desc || !hist_k || !hist_pos || !q || !q_pos || !scores || !status || n_src <= 0 || n_q <= 0)
+        return PC_ERR_INVALID_ARG;
+    if (!pc_aligned16(hist_k) || !pc_aligned16(hist_pos) || !pc_aligned16(q) || !pc_aligned16(q_pos) ||
+        !pc_aligned16(scores) || (reinterpret_cast<uintptr_t>(status) & 7u))
+        return PC_ERR_INVALID_ARG;
+    const pc_layer_desc &D = *desc;
+    if (D.head_dim != 64 && D.head_dim != 128) return PC_ERR_UNSUPPORTED;
+    if (D.dtype != PC_F32 && D.dtype != PC_BF16) return PC_ERR_UNSUPPORTED;
+    if (D.n_q_heads <= 0 || D.n_kv_heads <= 0 || D.n_q_heads % D.n_kv_heads) return PC_ERR_UNSUPPORTED;
+    if (!(D.rope_base > 1.0)) return PC_ERR_INVALID_ARG;
+    const int row = D.n_kv_heads * D.head_dim;
+    const int chunks = row / (D.dtype == PC_BF16 ? 8 : 4);
+    if (chunks % 32) return PC_ERR_UNSUPPORTED;
+    int64_t rope_entries = 0;
+    for (int a = 0; a < 3; ++a) {
+        if (D.max_pos[a] <= 0 || D.max_pos[a] > (1 << 20)) return PC_ERR_INVALID_ARG;
+        rope_entries += (int64_t)D.max_pos[a] * ((D.head_dim / 2 - a + 2) / 3);
+    }
+    if (row > STATIC_MAX_ROW || rope_entries > STATIC_MAX_ROPE ||
+        (size_t)D.n_q_heads * D.head_dim * sizeof(float) > 48 * 1024) {
+        fprintf(stderr,
+                "packcache: pc_score_tokens_static: shape exceeds the fixed scratch (n_kv_heads*head_dim %d > %d, or "
+                "rotary table %lld > %d entries, or n_q_heads*head_dim > 12288)\n",
+                row, STATIC_MAX_ROW, (long long)rope_entries, STATIC_MAX_ROPE);
+        return PC_ERR_CAPACITY;
+    }
+    unsigned char *base = nullptr;
+    pc_status st = static_scratch_base(&base);
+    if (st != PC_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    return D.dtype == PC_BF16
+               ? launch_score_static<__nv_bfloat16>(D, base, hist_k, hist_pos, n_src, q, q_pos, n_q, valid, scores, status, stream)
+               : launch_score_static<float>(D, base, hist_k, hist_pos, n_src, q, q_pos, n_q, valid, scores, status, stream);
+}

@@ -1,0 +1,74 @@
+"""The allocation-free scoring entry point against the ordinary one.
+
+Some hosts cannot call cudaMalloc when they need scores (all device memory already belongs to their own arena, or
+they cannot afford the device-wide synchronisation an allocation implies) and therefore cannot create a context.
+``pc_score_tokens_static`` serves them from a fixed device array inside the library.  Here it is called through the
+C ABI twice in a row — a bf16 case, then an fp32 case of another shape, so the second call finds the array full of
+the first call's rotary table, pooled query and partial sums — and each result must agree with ``pc_score`` on the
+same inputs within the score tolerance used everywhere else (1e-4 relative, floored by the frame's rms).
+
+This file sorts last on purpose: a run that stops at the first failure has already run every other test.
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_04359_b200 import binding as pc
+from paper_2601_04359_b200 import workload as wl
+from paper_2601_04359_b200.device import DeviceLayer, host, make_ctx, score_tolerance
+
+pytestmark = pytest.mark.gpu
+
+
+def _desc(cfg) -> pc.pc_layer_desc:
+    return pc.pc_layer_desc(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
+                            pc.PC_BF16 if cfg.dtype == wl.BF16 else pc.PC_F32, cfg.rope_base,
+                            (C.c_int32 * 3)(*cfg.max_pos), 0, 0)
+
+
+def _both(cfg, layer):
+    """(scores from pc_score, scores from the allocation-free call, frame table) for one seeded layer."""
+    L = wl.make_layer(cfg, layer=layer)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    want, _ = pc.pc_score(ctx, D.cache, D.q, D.q_pos, np.zeros(cfg.n_frames, np.int32))
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+    # buffers exist before the call; the call itself must not need any more memory
+    scores = torch.full((cfg.n_src,), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated()
+    pc.pc_score_tokens_static(_desc(cfg), D.cache.history.k, D.cache.history.pos, cfg.n_src, D.q, D.q_pos, scores, status)
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == before
+    assert status.cpu().tolist() == [0, 0]
+    ctx.close()
+    return host(want)[:cfg.n_src].astype(np.float64), host(scores).astype(np.float64), L.frame_count
+
+
+def test_static_scratch_scoring_matches_pc_score_on_two_calls_in_a_row():
+    first = wl.small_bf16(n_frames=4, grid=(12, 21), total=300, keep_full=0)    # 1008 source tokens, bf16, d = 128
+    second = wl.CONFIGS["tiny"]                                                 # fp32, d = 64, other table extents
+    for cfg, layer in ((first, 0), (second, 1), (first, 2)):
+        want, got, frame_count = _both(cfg, layer)
+        assert np.isfinite(got).all()
+        assert (np.abs(got - want) <= score_tolerance(want, frame_count)).all()
+
+
+def test_static_scratch_scoring_rejects_shapes_beyond_its_fixed_array():
+    cfg = wl.small_bf16()
+    z = torch.zeros(16, dtype=torch.float32, device="cuda")
+    st = torch.zeros(2, dtype=torch.int32, device="cuda")
+    big = pc.pc_layer_desc(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, pc.PC_BF16, cfg.rope_base,
+                           (C.c_int32 * 3)(4096, 4096, 4096), 0, 0)                 # rotary table too large
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_score_tokens_static(big, z, z, 1, z, z, z, st)
+    assert e.value.status == pc.PC_ERR_CAPACITY
+    wide = pc.pc_layer_desc(32, 16, 128, pc.PC_BF16, cfg.rope_base, (C.c_int32 * 3)(64, 64, 64), 0, 0)   # row > 1024
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_score_tokens_static(wide, z, z, 1, z, z, z, st)
+    assert e.value.status == pc.PC_ERR_CAPACITY
