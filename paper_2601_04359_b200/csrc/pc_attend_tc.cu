@@ -78,7 +78,7 @@ __device__ __forceinline__ uint64_t global_ns() {
     return t;
 }
 // Bounded wait: gives up after about one second, or at once when another thread of the CTA already gave up.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
     for (int i = 0; i < 2048; ++i)
         if (mbar_try(bar, parity)) return true;
     const uint64_t t0 = global_ns();
@@ -140,6 +140,17 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t *r) {
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// (a.x + b.x, a.y + b.y) in one instruction
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tadd.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -260,8 +271,10 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    // the softmax warps hold a whole 128-column score row per thread: registers move from warps 0-3 to warps 4-11
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
+        reg_dealloc<72>();
         if (lane == 0) {
             mbar_expect_tx(bar(BAR_Q), n_tiles_q * TILE_BYTES);
             for (int t = 0; t < n_tiles_q; ++t) {
@@ -294,6 +307,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
+        reg_dealloc<72>();
         if (lane == 0) {
             bool alive = mbar_wait(bar(BAR_Q), 0, abort_flag, P.status);
             auto issue_qk = [&](int t, int st) {
@@ -339,8 +353,11 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             tc_commit(bar(BAR_DONE));
             mbar_wait(bar(BAR_DONE), 0, abort_flag, P.status);
         }
-    } else if (warp >= 4) {
+    } else if (warp < 4) {
+        reg_dealloc<72>();
+    } else {
         // ---------------------------------------------------------------- softmax + correction + epilogue
+        reg_alloc<208>();
         const int t = (warp - 4) >> 2;
         const int quad = warp & 3;                       // TMEM lane quadrant this warp may touch
         const int r = quad * 32 + lane;                  // row of the tile
@@ -355,19 +372,27 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), j & 1, abort_flag, P.status));
             if (!alive) break;
             tc_fence_after();
-            uint32_t v[32];
-            // pass 1: row maximum
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(s_addr + c * 32, v);
-                tmem_wait_ld();
+            // the whole score row of this thread: one TMEM pass
+            uint32_t sv[128];
+            tmem_ld32(s_addr, sv);
+            tmem_ld32(s_addr + 32, sv + 32);
+            tmem_ld32(s_addr + 64, sv + 64);
+            tmem_ld32(s_addr + 96, sv + 96);
+            tmem_wait_ld();
+            if (n_valid < TILE) {                        // ragged last tile of a segment: keys past its end score -inf
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float x = (c * 32 + i < n_valid) ? __uint_as_float(v[i]) : -INFINITY;
-                    mx = fmaxf(mx, x);
-                }
+                for (int i = 0; i < TILE; ++i)
+                    if (i >= n_valid) sv[i] = 0xFF800000u;
             }
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < TILE; i += 4) {
+                mx0 = fmaxf(mx0, __uint_as_float(sv[i]));
+                mx1 = fmaxf(mx1, __uint_as_float(sv[i + 1]));
+                mx2 = fmaxf(mx2, __uint_as_float(sv[i + 2]));
+                mx3 = fmaxf(mx3, __uint_as_float(sv[i + 3]));
+            }
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             // lazy rescale: move the reference maximum only when it grew by more than the threshold
             const bool grow = mx > m_used + RESCALE_THRESHOLD;
             if (__any_sync(0xffffffffu, grow)) {
@@ -375,6 +400,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 const float corr = fast_exp2(m_used - m_new);       // 0 on the first tile (m_used = -inf)
                 l *= corr;
                 if (j > 0) {
+                    uint32_t v[32];
 #pragma unroll 1
                     for (int c = 0; c < 4; ++c) {
                         tmem_ld32(o_addr + c * 32, v);
@@ -386,23 +412,26 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 }
                 m_used = m_new;
             }
-            // pass 2: p = 2^(s - m), written as bf16 over the S columns
-#pragma unroll 1
+            // p = 2^(s - m) as bf16 pairs, written over the S columns; the row sum runs on two-lane adds
+            const float2 neg_m = make_float2(-m_used, -m_used);
+            float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+#pragma unroll
             for (int c = 0; c < 4; ++c) {
-                tmem_ld32(s_addr + c * 32, v);
-                tmem_wait_ld();
                 uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float p0 = fast_exp2(__uint_as_float(v[2 * i]) - m_used);
-                    float p1 = fast_exp2(__uint_as_float(v[2 * i + 1]) - m_used);
-                    if (c * 32 + 2 * i >= n_valid) p0 = 0.f;
-                    if (c * 32 + 2 * i + 1 >= n_valid) p1 = 0.f;
-                    l += p0 + p1;
-                    pk[i] = pc_pack_bf16(p0, p1);
+                for (int i = 0; i < 16; i += 2) {
+                    float2 x = add2(make_float2(__uint_as_float(sv[c * 32 + 2 * i]), __uint_as_float(sv[c * 32 + 2 * i + 1])), neg_m);
+                    float2 y = add2(make_float2(__uint_as_float(sv[c * 32 + 2 * i + 2]), __uint_as_float(sv[c * 32 + 2 * i + 3])), neg_m);
+                    x.x = fast_exp2(x.x); x.y = fast_exp2(x.y);
+                    y.x = fast_exp2(y.x); y.y = fast_exp2(y.y);
+                    la = add2(la, x);
+                    lb = add2(lb, y);
+                    pk[i] = pc_pack_bf16(x.x, x.y);
+                    pk[i + 1] = pc_pack_bf16(y.x, y.y);
                 }
                 tmem_st16(s_addr + c * 16, pk);
             }
+            l += (la.x + la.y) + (lb.x + lb.y);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(BAR_PFULL + t));

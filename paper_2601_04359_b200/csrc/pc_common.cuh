@@ -26,6 +26,7 @@ enum {
     PC_WHERE_ATTN_POS = 5,
     PC_WHERE_ATTN_WAIT = 6,
     PC_WHERE_ROPE_POS = 7,
+    PC_WHERE_SCORE_WAIT = 8,
 };
 
 // event marks: score call 0-3, pack 4-5, attend 6-9
@@ -108,6 +109,61 @@ __device__ __forceinline__ void pc_stg_stream(void *p, uint4 v) {
     asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
                  "r"(v.w)
                  : "memory");
+}
+
+// ---- mbarrier / bulk-copy helpers (shared::cta addresses as 32-bit integers)
+__device__ __forceinline__ uint32_t pc_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void pc_mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void pc_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void pc_mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool pc_mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t pc_global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait on an mbarrier phase: gives up after about one second, or at once when another thread of the CTA
+// already gave up (abort_flag), records PC_ERR_TIMEOUT with `where`, and returns false.
+static __device__ __noinline__ bool pc_mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status, int where) {
+    for (int i = 0; i < 2048; ++i)
+        if (pc_mbar_try(bar, parity)) return true;
+    const uint64_t t0 = pc_global_ns();
+    for (;;) {
+        if (pc_mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (pc_global_ns() - t0 > 1000000000ull) {
+            *abort_flag = 1;
+            pc_flag(status, PC_ERR_TIMEOUT, where);
+            return false;
+        }
+    }
+}
+// global -> shared bulk copy (both 16-byte aligned, size a multiple of 16), completion counted on an mbarrier
+__device__ __forceinline__ void pc_bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 pc_lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+// d += a * b on two fp32 lanes with one instruction
+__device__ __forceinline__ void pc_fma2(float2 &d, float2 a, float2 b) {
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%0, %1};\n\t"
+        "fma.rn.f32x2 rc, ra, rb, rc;\n\tmov.b64 {%0, %1}, rc;\n\t}"
+        : "+f"(d.x), "+f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
 }
 
 inline void pc_mark(pc_ctx *c, int idx, cudaStream_t s) {

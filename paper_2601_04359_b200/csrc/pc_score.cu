@@ -29,45 +29,89 @@ template <> struct Elem<__nv_bfloat16> {
 };
 
 // ---------------------------------------------------------------------------------------------------------
-// Pooled query.  Block b owns query tokens b, b + gridDim.x, ...; thread t owns rotary pairs t, t + blockDim.x, ...
-// of the [Hq][d/2] pair grid and accumulates them in shared memory (one owner per slot, fixed order).  The last
-// block to finish adds the per-block partials in block order, so the result does not depend on scheduling.
+// Pooled query.  The rotation is the same for every head at a given token and rotary pair, so the heads of a group
+// are added first and the sum is rotated once:  q~[g] = (1/n_q) sum_i R(p_i) (sum_{h in g} q_ih).
+// A block owns a contiguous run of query tokens.  Its 1024 threads form `slices` token slices x n_cols pair-columns
+// of the [Hkv][d/2] pooled grid (a warp reads 128 contiguous bytes of each head); a thread walks its slice's tokens
+// eight at a time with all loads of a batch issued before any is used.  Slices are added in slice order through
+// shared memory, and the last block to finish adds the per-block partials in block order, so the result does not
+// depend on scheduling.
 // ---------------------------------------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(256) k_qpool(const T *__restrict__ q, const int32_t *__restrict__ q_pos, int n_q,
-                                               int n_q_heads, int group, int d, pc_rope_dev rope,
-                                               float *__restrict__ partial, float *__restrict__ pooled,
-                                               unsigned int *ticket, int32_t *status) {
-    extern __shared__ float acc[];   // [Hq][d]
+constexpr int QPOOL_THREADS = 1024;
+constexpr int QPOOL_BATCH = 8;
+
+template <typename T, int GROUP /* query heads per KV head; 0 = any */>
+__global__ void __launch_bounds__(QPOOL_THREADS) k_qpool(const T *__restrict__ q, const int32_t *__restrict__ q_pos, int n_q,
+                                                         int n_q_heads, int group_rt, int d, pc_rope_dev rope,
+                                                         float *__restrict__ partial, float *__restrict__ pooled,
+                                                         unsigned int *ticket, int32_t *status) {
+    __shared__ float2 slice_sum[QPOOL_THREADS];
     __shared__ bool last;
-    const int half = d / 2, n_pairs = n_q_heads * half;
-    for (int p = threadIdx.x; p < n_pairs; p += blockDim.x) { acc[2 * p] = 0.f; acc[2 * p + 1] = 0.f; }
-    for (int i = blockIdx.x; i < n_q; i += gridDim.x) {
-        const int4 pp = *reinterpret_cast<const int4 *>(q_pos + 4 * (size_t)i);
-        const T *row = q + (size_t)i * n_q_heads * d;
-        for (int p = threadIdx.x; p < n_pairs; p += blockDim.x) {
-            const int pair = p % half;
-            const float2 cs = pc_rope_cs(rope, pair, pp.x, pp.y, pp.z, status, PC_WHERE_QPOOL_POS);
-            float x0, x1;
-            if constexpr (sizeof(T) == 2) {
-                const uint32_t w = *reinterpret_cast<const uint32_t *>(row + 2 * p);
-                x0 = pc_bf16_lo(w); x1 = pc_bf16_hi(w);
-            } else {
-                const float2 w = *reinterpret_cast<const float2 *>(row + 2 * p);
-                x0 = w.x; x1 = w.y;
+    const int group = GROUP > 0 ? GROUP : group_rt;
+    const int half = d / 2, n_kv = n_q_heads / group, n_cols = n_kv * half, row_len = n_kv * d;
+    const size_t q_row = (size_t)n_q_heads * d;
+    const int per_block = (n_q + gridDim.x - 1) / gridDim.x;
+    const int first = blockIdx.x * per_block, end = min(n_q, first + per_block);
+    const int slices = max(1, QPOOL_THREADS / n_cols);
+    const int sl = threadIdx.x / n_cols;
+    for (int col0 = 0; col0 < n_cols; col0 += QPOOL_THREADS) {        // one pass unless n_cols > 1024
+        const int col = col0 + (n_cols >= QPOOL_THREADS ? threadIdx.x : threadIdx.x % n_cols);
+        const bool active = sl < slices && col < n_cols;
+        float acc0 = 0.f, acc1 = 0.f;
+        if (active) {
+            const int g = col / half, pair = col % half;
+            const T *base = q + (size_t)g * group * d + 2 * pair;
+            const int axis = pair % 3, amax = rope.max_pos[axis], astride = rope.n_axis[axis];
+            const float2 *tab = rope.tab + rope.off[axis] + pair / 3;
+            for (int i0 = first + sl; i0 < end; i0 += slices * QPOOL_BATCH) {
+                int pa[QPOOL_BATCH];                                   // this pair's own coordinate of each token
+                float x0[QPOOL_BATCH], x1[QPOOL_BATCH];
+#pragma unroll
+                for (int t = 0; t < QPOOL_BATCH; ++t) {
+                    const int i = min(i0 + t * slices, end - 1);       // out-of-range slots re-read the last token, unused
+                    pa[t] = __ldg(q_pos + 4 * (size_t)i + axis);
+                    const T *row = base + (size_t)i * q_row;
+                    x0[t] = 0.f; x1[t] = 0.f;
+#pragma unroll
+                    for (int u = 0; u < (GROUP > 0 ? GROUP : 1); ++u) {
+                        for (int uu = u; uu < group; uu += (GROUP > 0 ? group : 1)) {
+                            if constexpr (sizeof(T) == 2) {
+                                const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(row + (size_t)uu * d));
+                                x0[t] += pc_bf16_lo(w); x1[t] += pc_bf16_hi(w);
+                            } else {
+                                const float2 w = __ldg(reinterpret_cast<const float2 *>(row + (size_t)uu * d));
+                                x0[t] += w.x; x1[t] += w.y;
+                            }
+                        }
+                    }
+                }
+                float2 cs[QPOOL_BATCH];
+#pragma unroll
+                for (int t = 0; t < QPOOL_BATCH; ++t) {
+                    int p = pa[t];
+                    if ((unsigned)p >= (unsigned)amax) {               // outside the table: record, clamp
+                        pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_QPOOL_POS);
+                        p = p < 0 ? 0 : amax - 1;
+                    }
+                    cs[t] = __ldg(tab + (size_t)p * astride);
+                }
+#pragma unroll
+                for (int t = 0; t < QPOOL_BATCH; ++t)
+                    if (i0 + t * slices < end) {
+                        acc0 += x0[t] * cs[t].x - x1[t] * cs[t].y;
+                        acc1 += x0[t] * cs[t].y + x1[t] * cs[t].x;
+                    }
             }
-            acc[2 * p] += x0 * cs.x - x1 * cs.y;
-            acc[2 * p + 1] += x0 * cs.y + x1 * cs.x;
         }
-    }
-    __syncthreads();
-    // fold the heads of each group, in head order
-    const int n_kv = n_q_heads / group, row_len = n_kv * d;
-    for (int e = threadIdx.x; e < row_len; e += blockDim.x) {
-        const int g = e / d, c = e % d;
-        float s = 0.f;
-        for (int u = 0; u < group; ++u) s += acc[(g * group + u) * d + c];
-        partial[(size_t)blockIdx.x * row_len + e] = s;
+        slice_sum[threadIdx.x] = make_float2(acc0, acc1);
+        __syncthreads();
+        if (active && sl == 0) {
+            float2 tot = make_float2(0.f, 0.f);
+            const int stride = n_cols >= QPOOL_THREADS ? QPOOL_THREADS : n_cols;
+            for (int k = 0; k < slices; ++k) { const float2 v = slice_sum[k * stride + threadIdx.x]; tot.x += v.x; tot.y += v.y; }
+            *reinterpret_cast<float2 *>(partial + (size_t)blockIdx.x * row_len + 2 * col) = tot;
+        }
+        __syncthreads();
     }
     __threadfence();
     __syncthreads();
@@ -76,8 +120,9 @@ __global__ void __launch_bounds__(256) k_qpool(const T *__restrict__ q, const in
     if (!last) return;
     __threadfence();
     const float inv_n = 1.f / (float)n_q;
-    for (int e = threadIdx.x; e < row_len; e += blockDim.x) {
+    for (int e = threadIdx.x; e < row_len; e += QPOOL_THREADS) {
         float s = 0.f;
+#pragma unroll 16
         for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(partial + (size_t)b * row_len + e);
         pooled[e] = s * inv_n;
     }
@@ -85,72 +130,156 @@ __global__ void __launch_bounds__(256) k_qpool(const T *__restrict__ q, const in
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Score: one warp per token.  A token's K row over all KV heads is CH = Hkv*d/PER16 16-byte chunks; lane l reads
-// chunks l, l+32, ... .  Because 32*PER16 is a multiple of d, all of a lane's chunks cover the same PER16/2 rotary
-// pairs (of different heads), so the lane sums the two brackets over its chunks and needs PER16/2 table look-ups.
-// Two tokens are in flight per warp to keep enough bytes outstanding.
+// Score.  History keys are contiguous, so a tile of 8 tokens is one run of 8 rows (16 KB at 8 KV heads x 128 bf16)
+// plus 128 bytes of positions.  A producer warp streams tiles into a four-stage shared-memory ring with bulk
+// asynchronous copies tracked by mbarriers; eight consumer warps take one token each.  A token's row over all KV
+// heads is CPL x 32 sixteen-byte chunks; lane l reads chunks l, l+32, ...  Because 32 chunks span a multiple of d,
+// all of a lane's chunks cover the same PER16/2 rotary pairs (of different heads), so the lane sums the two brackets
+// over its chunks and needs PER16/2 table look-ups per token.  Chunks are processed two at a time so that every
+// multiply-add is a two-lane fp32 instruction.  Blocks are persistent and take tiles round-robin.
 // ---------------------------------------------------------------------------------------------------------
-template <typename T, int CPL /* chunks per lane */>
-__global__ void __launch_bounds__(256) k_score(const T *__restrict__ k, const int32_t *__restrict__ k_pos,
-                                               const uint8_t *__restrict__ valid, int n_src, int d, float scale,
-                                               pc_rope_dev rope, const float *__restrict__ pooled,
-                                               float *__restrict__ scores, int32_t *status) {
-    constexpr int PER = Elem<T>::PER16, NP = PER / 2;
-    const int lane = threadIdx.x & 31;
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int n_warps = (gridDim.x * blockDim.x) >> 5;
-    const size_t row_bytes = (size_t)CPL * 32 * 16;
+constexpr int SCORE_TOK = 8;                       // tokens per tile = consumer warps
+constexpr int SCORE_STAGES = 4;
+constexpr int SCORE_THREADS = (SCORE_TOK + 1) * 32;
 
-    // this lane's slice of the pooled query stays in registers
-    float qv[CPL][PER];
+template <typename T, int CPL /* chunks per lane */>
+__global__ void __launch_bounds__(SCORE_THREADS) k_score(const T *__restrict__ k, const int32_t *__restrict__ k_pos,
+                                                         const uint8_t *__restrict__ valid, int n_src, int d, float scale,
+                                                         pc_rope_dev rope, const float *__restrict__ pooled,
+                                                         float *__restrict__ scores, int32_t *status) {
+    constexpr int PER = Elem<T>::PER16, NP = PER / 2;
+    constexpr uint32_t ROW_BYTES = CPL * 32 * 16;
+    constexpr uint32_t STAGE_BYTES = SCORE_TOK * ROW_BYTES + SCORE_TOK * 16;
+    extern __shared__ __align__(128) uint8_t ring[];
+    __shared__ __align__(8) uint64_t bars[2 * SCORE_STAGES];
+    __shared__ int abort_word;
+    volatile int *abort_flag = &abort_word;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t ring0 = pc_smem_u32(ring), bar0 = pc_smem_u32(bars);
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto empty = [&](int s) { return bar0 + 8u * (SCORE_STAGES + s); };
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < SCORE_STAGES; ++s) { pc_mbar_init(full(s), 1); pc_mbar_init(empty(s), SCORE_TOK); }
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int n_tiles = (n_src + SCORE_TOK - 1) / SCORE_TOK;
+
+    if (warp == SCORE_TOK) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            int it = 0;
+            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+                const int s = it % SCORE_STAGES, use = it / SCORE_STAGES;
+                if (use > 0 && !pc_mbar_wait(empty(s), (use - 1) & 1, abort_flag, status, PC_WHERE_SCORE_WAIT)) break;
+                const int tok0 = tile * SCORE_TOK, n_tok = min(SCORE_TOK, n_src - tok0);
+                const uint32_t dst = ring0 + s * STAGE_BYTES;
+                pc_mbar_expect_tx(full(s), n_tok * (ROW_BYTES + 16));
+                pc_bulk_g2s(dst, reinterpret_cast<const char *>(k) + (size_t)tok0 * ROW_BYTES, n_tok * ROW_BYTES, full(s));
+                pc_bulk_g2s(dst + SCORE_TOK * ROW_BYTES, k_pos + 4 * (size_t)tok0, n_tok * 16, full(s));
+            }
+            if (*abort_flag) {   // let copies already issued land before the block's shared memory goes away
+                const uint64_t t0 = pc_global_ns();
+                while (pc_global_ns() - t0 < 2000000ull) {}
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- consumers
+    // this lane's slice of the pooled query stays in registers, chunks paired for the two-lane multiply-adds
+    constexpr int CP = CPL / 2;                                     // chunk pairs; an odd CPL leaves one single chunk
+    float2 qa[CP > 0 ? CP : 1][NP], qb[CP > 0 ? CP : 1][NP];
+    float qa1[NP], qb1[NP];
 #pragma unroll
     for (int c = 0; c < CPL; ++c)
 #pragma unroll
-        for (int e = 0; e < PER; ++e) qv[c][e] = pooled[(size_t)(c * 32 + lane) * PER + e];
-    const int pair0 = ((lane * PER) % d) / 2;
-
-    for (int j0 = warp * 2; j0 < n_src; j0 += n_warps * 2) {
-        uint4 raw[2][CPL];
-        int4 pp[2];
-#pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const int j = min(j0 + t, n_src - 1);
-            const char *row = reinterpret_cast<const char *>(k) + (size_t)j * row_bytes;
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) raw[t][c] = pc_ldg_stream(row + (size_t)(c * 32 + lane) * 16);
-            pp[t] = __ldg(reinterpret_cast<const int4 *>(k_pos) + j);
+        for (int u = 0; u < NP; ++u) {
+            const float a = pooled[(size_t)(c * 32 + lane) * PER + 2 * u], b = pooled[(size_t)(c * 32 + lane) * PER + 2 * u + 1];
+            if (c < 2 * CP) {
+                if (c & 1) { qa[c / 2][u].y = a; qb[c / 2][u].y = b; } else { qa[c / 2][u].x = a; qb[c / 2][u].x = b; }
+            } else { qa1[u] = a; qb1[u] = b; }
         }
+    // table slots of this lane's pairs: entry = tbase + coordinate(axis) * stride
+    const int pair0 = ((lane * PER) % d) / 2;
+    int tbase[NP], tstride[NP], taxis[NP];
 #pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const int j = j0 + t;
-            float A[NP], B[NP];
+    for (int u = 0; u < NP; ++u) {
+        const int a = (pair0 + u) % 3;
+        taxis[u] = a;
+        tbase[u] = rope.off[a] + (pair0 + u) / 3;
+        tstride[u] = rope.n_axis[a];
+    }
+    const unsigned mt = rope.max_pos[0], mh = rope.max_pos[1], mw = rope.max_pos[2];
+
+    int it = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+        const int s = it % SCORE_STAGES, use = it / SCORE_STAGES;
+        if (!__all_sync(0xffffffffu, pc_mbar_wait(full(s), use & 1, abort_flag, status, PC_WHERE_SCORE_WAIT))) return;
+        const int j = tile * SCORE_TOK + warp;
+        if (j < n_src) {
+            const uint32_t row = ring0 + s * STAGE_BYTES + warp * ROW_BYTES + lane * 16;
+            uint4 raw[CPL];
 #pragma unroll
-            for (int u = 0; u < NP; ++u) { A[u] = 0.f; B[u] = 0.f; }
-#pragma unroll
-            for (int c = 0; c < CPL; ++c) {
-                float kv[PER];
-                Elem<T>::unpack(raw[t][c], kv);
-#pragma unroll
-                for (int u = 0; u < NP; ++u) {
-                    const float qa = qv[c][2 * u], qb = qv[c][2 * u + 1], ka = kv[2 * u], kb = kv[2 * u + 1];
-                    A[u] = fmaf(qa, ka, fmaf(qb, kb, A[u]));
-                    B[u] = fmaf(qb, ka, fmaf(-qa, kb, B[u]));
-                }
+            for (int c = 0; c < CPL; ++c) raw[c] = pc_lds128(row + c * 512);
+            const uint4 pw4 = pc_lds128(ring0 + s * STAGE_BYTES + SCORE_TOK * ROW_BYTES + warp * 16);
+            int pt = (int)pw4.x, ph = (int)pw4.y, pw = (int)pw4.z;
+            if (!((unsigned)pt < mt && (unsigned)ph < mh && (unsigned)pw < mw)) {   // outside the tables: record, clamp
+                pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_SCORE_POS);
+                pt = min(max(pt, 0), (int)mt - 1); ph = min(max(ph, 0), (int)mh - 1); pw = min(max(pw, 0), (int)mw - 1);
             }
-            float s = 0.f;
+            float2 cs[NP];
 #pragma unroll
             for (int u = 0; u < NP; ++u) {
-                const float2 cs = pc_rope_cs(rope, pair0 + u, pp[t].x, pp[t].y, pp[t].z, status, PC_WHERE_SCORE_POS);
-                s = fmaf(cs.x, A[u], fmaf(cs.y, B[u], s));
+                const int pa = taxis[u] == 0 ? pt : (taxis[u] == 1 ? ph : pw);
+                cs[u] = __ldg(rope.tab + tbase[u] + pa * tstride[u]);
+            }
+            // brackets per pair:  A = sum qa ka + qb kb,  B = sum qb ka - qa kb  (B kept as two sums)
+            float2 A2[NP], B2[NP], C2[NP];
+            float A1[NP], B1[NP];
+#pragma unroll
+            for (int u = 0; u < NP; ++u) { A2[u] = B2[u] = C2[u] = make_float2(0.f, 0.f); A1[u] = B1[u] = 0.f; }
+#pragma unroll
+            for (int c = 0; c < CP; ++c) {
+                float k0[PER], k1[PER];
+                Elem<T>::unpack(raw[2 * c], k0);
+                Elem<T>::unpack(raw[2 * c + 1], k1);
+#pragma unroll
+                for (int u = 0; u < NP; ++u) {
+                    const float2 ka = make_float2(k0[2 * u], k1[2 * u]), kb = make_float2(k0[2 * u + 1], k1[2 * u + 1]);
+                    pc_fma2(A2[u], qa[c][u], ka);
+                    pc_fma2(A2[u], qb[c][u], kb);
+                    pc_fma2(B2[u], qb[c][u], ka);
+                    pc_fma2(C2[u], qa[c][u], kb);
+                }
+            }
+            if constexpr (CPL & 1) {
+                float k0[PER];
+                Elem<T>::unpack(raw[CPL - 1], k0);
+#pragma unroll
+                for (int u = 0; u < NP; ++u) {
+                    A1[u] = fmaf(qa1[u], k0[2 * u], fmaf(qb1[u], k0[2 * u + 1], A1[u]));
+                    B1[u] = fmaf(qb1[u], k0[2 * u], fmaf(-qa1[u], k0[2 * u + 1], B1[u]));
+                }
+            }
+            float sum = 0.f;
+#pragma unroll
+            for (int u = 0; u < NP; ++u) {
+                const float A = (A2[u].x + A2[u].y) + A1[u];
+                const float B = ((B2[u].x + B2[u].y) - (C2[u].x + C2[u].y)) + B1[u];
+                sum = fmaf(cs[u].x, A, fmaf(cs[u].y, B, sum));
             }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (lane == 0 && j < n_src) {
-                float r = s * scale;
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (lane == 0) {
+                float r = sum * scale;
                 if (valid && !valid[j]) r = -INFINITY;
                 scores[j] = r;
             }
         }
+        __syncwarp();
+        if (lane == 0) pc_mbar_arrive(empty(s));
     }
 }
 
@@ -168,7 +297,9 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 }
 
 constexpr int SEL_THREADS = 512;
+constexpr int SEL_CACHE = 4096;   // keys of a frame kept in shared memory; longer frames re-read the rest from global
 
+// Exclusive block scan of a small per-thread value; total = sum over the block.
 __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int &total) {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     int inc = v;
@@ -193,6 +324,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int &
 
 __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict__ scores, const __grid_constant__ FrameTab tab,
                                                        int32_t *__restrict__ sel_idx, int32_t *status) {
+    __shared__ uint32_t keys[SEL_CACHE];
     __shared__ int hist[256];
     __shared__ int warp_sums[SEL_THREADS / 32];
     __shared__ uint32_t sh_prefix;
@@ -201,88 +333,132 @@ __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict_
     const int first = fr.x, n = fr.y, budget = fr.z, out0 = fr.w;
     if (budget <= 0 || n <= 0) return;
     const float *s = scores + first;
+    const int lane = threadIdx.x & 31;
+
+    for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
+        const float v = s[j];
+        if (v != v) pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_SELECT_NAN);
+        if (j < SEL_CACHE) keys[j] = score_key(v);
+    }
+    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+    __syncthreads();
+    auto key_at = [&](int j) { return j < SEL_CACHE ? keys[j] : score_key(s[j]); };
 
     uint32_t prefix = 0, mask = 0;
     int want = budget;                               // rank, among keys matching the prefix, of the threshold key
     for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int b = threadIdx.x; b < 256; b += SEL_THREADS) hist[b] = 0;
-        __syncthreads();
         for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
-            const float v = s[j];
-            if (v != v) pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_SELECT_NAN);
-            const uint32_t key = score_key(v);
+            const uint32_t key = key_at(j);
             if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            int w = want, b = 255;
-            for (; b > 0; --b) {
-                if (hist[b] >= w) break;
-                w -= hist[b];
+        if (threadIdx.x < 32) {
+            // lane l owns digits 255 - 8l down to 248 - 8l; an inclusive scan over lanes counts keys from the top digit down
+            int c[8], mine = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { c[i] = hist[255 - 8 * lane - i]; mine += c[i]; }
+            int inc = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int v = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += v;
             }
-            sh_prefix = prefix | ((uint32_t)b << shift);
-            sh_want = w;
+            const int before = inc - mine;
+            if (before < want && want <= inc) {      // exactly one lane: the threshold digit is among its eight
+                int w = want - before, digit = 255 - 8 * lane;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (c[i] >= w) { digit = 255 - 8 * lane - i; break; }
+                    w -= c[i];
+                }
+                sh_prefix = prefix | ((uint32_t)digit << shift);
+                sh_want = w;
+            }
         }
         __syncthreads();
         prefix = sh_prefix;
         want = sh_want;
         mask |= 255u << shift;
+        if (threadIdx.x < 256) hist[threadIdx.x] = 0;
         __syncthreads();
     }
-    // prefix is now the threshold key T; `want` of the keys equal to T are kept, lowest indices first
+    // prefix is now the threshold key T: every key above it is kept, and the `want` lowest-index keys equal to it.
+    // One scan per 512 keys carries both counts (keys above T in the low half, keys equal to T in the high half).
     const uint32_t T = prefix;
-    int eq_seen = 0, written = 0;
+    int gt_seen = 0, eq_seen = 0;
     for (int j0 = 0; j0 < n; j0 += SEL_THREADS) {
         const int j = j0 + threadIdx.x;
-        uint32_t key = 0;
         const bool in = j < n;
-        if (in) key = score_key(s[j]);
-        const int is_eq = in && key == T;
-        int eq_total, keep_total;
-        const int eq_rank = eq_seen + block_exclusive_scan(is_eq, warp_sums, eq_total);
-        const int keep = in && (key > T || (is_eq && eq_rank < want));
-        const int at = written + block_exclusive_scan(keep, warp_sums, keep_total);
-        if (keep && at < budget) sel_idx[out0 + at] = first + j;
-        eq_seen += eq_total;
-        written += keep_total;
+        const uint32_t key = in ? key_at(j) : 0u;
+        const int is_gt = in && key > T, is_eq = in && key == T;
+        int total;
+        const int ex = block_exclusive_scan(is_gt | (is_eq << 16), warp_sums, total);
+        const int gt_before = gt_seen + (ex & 0xFFFF), eq_before = eq_seen + (ex >> 16);
+        if (is_gt || (is_eq && eq_before < want)) {
+            const int at = gt_before + min(eq_before, want);
+            if (at < budget) sel_idx[out0 + at] = first + j;
+        }
+        gt_seen += total & 0xFFFF;
+        eq_seen += total >> 16;
     }
 }
 
+// Enqueue pooling and scoring on caller-given scratch (a context's, or the library's fixed array).
 template <typename T>
-pc_status launch_score(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q,
-                       const uint8_t *valid, float *scores, cudaStream_t stream) {
-    const pc_layer_desc &D = ctx->desc;
+pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev &rope, float *partial, float *pooled,
+                        unsigned int *ticket, int32_t *status, const void *hist_k, const int32_t *hist_pos, int n_src,
+                        const void *q, const int32_t *q_pos, int32_t n_q, const uint8_t *valid, float *scores,
+                        cudaStream_t stream, pc_ctx *marks) {
     const int row = D.n_kv_heads * D.head_dim;
-    const int n_src = src->history.n_tokens;
-    const int pool_blocks = std::min<int>(PC_QPOOL_BLOCKS, n_q);
-    const size_t smem = (size_t)D.n_q_heads * D.head_dim * sizeof(float);
-    if (smem > 48 * 1024)
-        PC_CUDA_TRY(cudaFuncSetAttribute(k_qpool<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    pc_mark(ctx, PC_MARK_SCORE0, stream);
-    k_qpool<T><<<pool_blocks, 256, smem, stream>>>(static_cast<const T *>(q), q_pos, n_q, D.n_q_heads, ctx->group,
-                                                   D.head_dim, ctx->rope, ctx->qpool_partial, ctx->qpool, ctx->ticket,
-                                                   ctx->status);
+    const int group = D.n_q_heads / D.n_kv_heads;
+    const int pool_blocks = std::min<int>(PC_QPOOL_BLOCKS, (n_q + 15) / 16);
+    if (marks) pc_mark(marks, PC_MARK_SCORE0, stream);
+#define PC_QPOOL_ARGS static_cast<const T *>(q), q_pos, n_q, D.n_q_heads, group, D.head_dim, rope, partial, pooled, ticket, status
+    switch (group) {
+    case 1: k_qpool<T, 1><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
+    case 2: k_qpool<T, 2><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
+    case 3: k_qpool<T, 3><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
+    case 4: k_qpool<T, 4><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
+    default: k_qpool<T, 0><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
+    }
+#undef PC_QPOOL_ARGS
     PC_CUDA_TRY(cudaGetLastError());
-    pc_mark(ctx, PC_MARK_QPOOL, stream);
+    if (marks) pc_mark(marks, PC_MARK_QPOOL, stream);
     const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
     const int chunks = row / Elem<T>::PER16;          // 16-byte chunks per token row
-    const int warps_needed = (n_src + 1) / 2;
-    const int blocks = std::max(1, std::min((warps_needed + 7) / 8, ctx->sm_count * 6));
-    const T *k = static_cast<const T *>(src->history.k);
-#define PC_SCORE_CASE(CPL)                                                                                          \
-    case CPL:                                                                                                       \
-        k_score<T, CPL><<<blocks, 256, 0, stream>>>(k, src->history.pos, valid, n_src, D.head_dim, scale, ctx->rope, \
-                                                    ctx->qpool, scores, ctx->status);                              \
-        break;
     if (chunks % 32) return PC_ERR_UNSUPPORTED;
+    const int n_tiles = (n_src + SCORE_TOK - 1) / SCORE_TOK;
+    const T *k = static_cast<const T *>(hist_k);
+#define PC_SCORE_CASE(CPL)                                                                                          \
+    case CPL: {                                                                                                     \
+        const int smem = SCORE_STAGES * (SCORE_TOK * CPL * 512 + SCORE_TOK * 16);                                   \
+        static int per_sm = 0; /* resident blocks per SM of this instance: the grid is persistent */              \
+        if (per_sm == 0) {                                                                                          \
+            PC_CUDA_TRY(cudaFuncSetAttribute(k_score<T, CPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));  \
+            int occ = 0;                                                                                            \
+            PC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_score<T, CPL>, SCORE_THREADS, smem)); \
+            per_sm = std::max(1, occ);                                                                              \
+        }                                                                                                           \
+        const int blocks = std::max(1, std::min(n_tiles, sm_count * per_sm));                                       \
+        k_score<T, CPL><<<blocks, SCORE_THREADS, smem, stream>>>(k, hist_pos, valid, n_src, D.head_dim, scale, rope, \
+                                                                 pooled, scores, status);                          \
+    } break;
     switch (chunks / 32) {
         PC_SCORE_CASE(1) PC_SCORE_CASE(2) PC_SCORE_CASE(3) PC_SCORE_CASE(4) PC_SCORE_CASE(6) PC_SCORE_CASE(8)
     default: return PC_ERR_UNSUPPORTED;
     }
 #undef PC_SCORE_CASE
     PC_CUDA_TRY(cudaGetLastError());
-    pc_mark(ctx, PC_MARK_SCORE, stream);
+    if (marks) pc_mark(marks, PC_MARK_SCORE, stream);
     return PC_OK;
+}
+
+template <typename T>
+pc_status launch_score(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q,
+                       const uint8_t *valid, float *scores, cudaStream_t stream) {
+    return enqueue_score<T>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_partial, ctx->qpool, ctx->ticket, ctx->status,
+                            src->history.k, src->history.pos, src->history.n_tokens, q, q_pos, n_q, valid, scores, stream,
+                            ctx);
 }
 
 }  // namespace
@@ -414,33 +590,11 @@ pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const
     k_rope_table<<<(total + 255) / 256, 256, 0, stream>>>(tab, rope, D.rope_base, total);
     PC_CUDA_TRY(cudaGetLastError());
 
-    const int row = D.n_kv_heads * D.head_dim;
-    const int pool_blocks = std::min<int>(PC_QPOOL_BLOCKS, n_q);
-    const size_t smem = (size_t)D.n_q_heads * D.head_dim * sizeof(float);
-    k_qpool<T><<<pool_blocks, 256, smem, stream>>>(static_cast<const T *>(q), q_pos, n_q, D.n_q_heads,
-                                                   D.n_q_heads / D.n_kv_heads, D.head_dim, rope, partial, pooled, ticket,
-                                                   status);
-    PC_CUDA_TRY(cudaGetLastError());
-    const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
-    const int chunks = row / Elem<T>::PER16;
-    const int warps_needed = (n_src + 1) / 2;
     int sm_count = 0, dev = 0;
     PC_CUDA_TRY(cudaGetDevice(&dev));
     PC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    const int blocks = std::max(1, std::min((warps_needed + 7) / 8, sm_count * 6));
-    const T *k = static_cast<const T *>(hist_k);
-#define PC_SCORE_CASE(CPL)                                                                                         \
-    case CPL:                                                                                                      \
-        k_score<T, CPL><<<blocks, 256, 0, stream>>>(k, hist_pos, valid, n_src, D.head_dim, scale, rope, pooled, scores, \
-                                                    status);                                                      \
-        break;
-    switch (chunks / 32) {
-        PC_SCORE_CASE(1) PC_SCORE_CASE(2) PC_SCORE_CASE(3) PC_SCORE_CASE(4) PC_SCORE_CASE(6) PC_SCORE_CASE(8)
-    default: return PC_ERR_UNSUPPORTED;
-    }
-#undef PC_SCORE_CASE
-    PC_CUDA_TRY(cudaGetLastError());
-    return PC_OK;
+    return enqueue_score<T>(D, sm_count, rope, partial, pooled, ticket, status, hist_k, hist_pos, n_src, q, q_pos, n_q,
+                            valid, scores, stream, nullptr);
 }
 
 }  // namespace
