@@ -8,7 +8,8 @@
 //                 tcgen05.mma: S_t = Q_t K^T (both operands K-major in shared memory) into TMEM, and
 //                 O_t += P_t V with P_t read from TMEM and V MN-major in shared memory.  Warps 4-7 / 8-11 are the
 //                 softmax groups of tile 0 / 1: tcgen05.ld the S row, running max and sum in fp32 (base 2), write
-//                 bf16 P over S in TMEM, and rescale O in TMEM only when the running max moved by more than 2^8.
+//                 bf16 P over S in TMEM (handed over in two halves of 64 keys), and rescale O in TMEM only when
+//                 the running max moved by more than 2^8.
 //                 While one tile's softmax runs, the tensor core works on the other tile.
 //   k_combine     merges the KV ranges' (max, sum, O) partials when the keys were split across CTAs.
 //
@@ -39,8 +40,8 @@ constexpr int SM_BAR = SM_V + KV_STAGES * TILE_BYTES;     // barriers etc.
 constexpr int SM_TOTAL = SM_BAR + 256;
 constexpr int SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
 
-enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PFULL = 11,
-       BAR_DONE = 13, N_BARS = 14 };
+enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PHALF = 11 /* [tile][half] */,
+       BAR_DONE = 15, N_BARS = 16 };
 
 struct TcParams {
     int n_q, n_q_heads, group, n_tb, tiles_per_g, pairs_per_g, n_splits, n_kv_tiles;
@@ -91,6 +92,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             return false;
         }
     }
+}
+
+// True in exactly one lane of a converged warp.  The compiler turns work predicated on elect.sync into single-issue
+// code with operands in uniform registers; the same work under `lane == 0` costs about five times the issue time.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
@@ -255,7 +264,8 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar(BAR_SFULL + t), 1);
-            mbar_init(bar(BAR_PFULL + t), 128);
+            mbar_init(bar(BAR_PHALF + 2 * t), 128);
+            mbar_init(bar(BAR_PHALF + 2 * t + 1), 128);
         }
         mbar_init(bar(BAR_DONE), 1);
         *abort_flag = 0;
@@ -307,52 +317,61 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
+        // The warp stays converged (every lane takes the waits) and only the tcgen05 instructions are predicated on
+        // one elected lane: issuing a multiply-add then costs about 12 cycles instead of about 60.
         reg_dealloc<72>();
-        if (lane == 0) {
-            bool alive = mbar_wait(bar(BAR_Q), 0, abort_flag, P.status);
-            auto issue_qk = [&](int t, int st) {
-                const uint32_t qa = base + SM_Q + t * TILE_BYTES, ka = base + SM_K + st * TILE_BYTES;
+        const bool lead = elect_one();
+        const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+        bool alive = mbar_wait(bar(BAR_Q), 0, abort_flag, P.status);
+        auto issue_qk = [&](int t, int st) {
+            const uint32_t qa = base + SM_Q + t * TILE_BYTES, ka = base + SM_K + st * TILE_BYTES;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                    mma_ss(tmem + t * TILE, desc_kmajor(qa + off), desc_kmajor(ka + off), IDESC_QK, ks > 0);
-                }
-            };
-            if (alive && n_j > 0) alive = mbar_wait(bar(BAR_KFULL + 0), 0, abort_flag, P.status);
-            if (alive && n_j > 0) {
-                tc_fence_after();
-                for (int t = 0; t < n_tiles_q; ++t) {
-                    issue_qk(t, 0);
-                    tc_commit(bar(BAR_SFULL + t));
-                }
-                tc_commit(bar(BAR_KEMPTY + 0));
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                if (lead) mma_ss(tm + t * TILE, desc_kmajor(qa + off), desc_kmajor(ka + off), IDESC_QK, ks > 0);
             }
-            for (int j = 0; j < n_j && alive; ++j) {
-                const int st = j % KV_STAGES, use = j / KV_STAGES;
-                const int nst = (j + 1) % KV_STAGES, nuse = (j + 1) / KV_STAGES;
-                alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status);
-                if (alive && j + 1 < n_j) alive = mbar_wait(bar(BAR_KFULL + nst), nuse & 1, abort_flag, P.status);
-                for (int t = 0; t < n_tiles_q && alive; ++t) {
-                    alive = mbar_wait(bar(BAR_PFULL + t), j & 1, abort_flag, P.status);
+        };
+        if (alive && n_j > 0) alive = mbar_wait(bar(BAR_KFULL + 0), 0, abort_flag, P.status);
+        if (alive && n_j > 0) {
+            tc_fence_after();
+            for (int t = 0; t < n_tiles_q; ++t) {
+                issue_qk(t, 0);
+                if (lead) tc_commit(bar(BAR_SFULL + t));
+            }
+            if (lead) tc_commit(bar(BAR_KEMPTY + 0));
+        }
+        for (int j = 0; j < n_j && alive; ++j) {
+            const int st = j % KV_STAGES, use = j / KV_STAGES;
+            const int nst = (j + 1) % KV_STAGES, nuse = (j + 1) / KV_STAGES;
+            alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status);
+            if (alive && j + 1 < n_j) alive = mbar_wait(bar(BAR_KFULL + nst), nuse & 1, abort_flag, P.status);
+            for (int t = 0; t < n_tiles_q && alive; ++t) {
+                const uint32_t va = base + SM_V + st * TILE_BYTES;
+                // P arrives in two halves of 64 keys: the first PV steps run while the rest is exponentiated
+                for (int hf = 0; hf < 2 && alive; ++hf) {
+                    alive = mbar_wait(bar(BAR_PHALF + 2 * t + hf), j & 1, abort_flag, P.status);
                     if (!alive) break;
                     tc_fence_after();
-                    const uint32_t va = base + SM_V + st * TILE_BYTES;
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)   // 16 keys per step: P columns advance by 8 (two bf16 per column)
-                        mma_ts(tmem + 256 + t * TILE, tmem + t * TILE + ks * 8, desc_mnmajor(va + ks * 2048), IDESC_PV,
-                               (j > 0 || ks > 0));
-                    if (j + 1 < n_j) issue_qk(t, nst);
-                    tc_commit(bar(BAR_SFULL + t));          // S_t(j+1) ready, or after the last tile: O_t final
+                    for (int k4 = 0; k4 < 4; ++k4) {   // 16 keys per step: P columns advance by 8 (two bf16 per column)
+                        const int ks = hf * 4 + k4;
+                        if (lead)
+                            mma_ts(tm + 256 + t * TILE, tm + t * TILE + ks * 8, desc_mnmajor(va + ks * 2048), IDESC_PV, (j > 0 || ks > 0));
+                    }
                 }
-                if (alive) {
-                    tc_commit(bar(BAR_VEMPTY + st));
-                    if (j + 1 < n_j) tc_commit(bar(BAR_KEMPTY + nst));
-                }
+                if (!alive) break;
+                if (j + 1 < n_j) issue_qk(t, nst);
+                if (lead) tc_commit(bar(BAR_SFULL + t));          // S_t(j+1) ready, or after the last tile: O_t final
             }
-            // make sure nothing of ours is still running on the tensor core before TMEM is freed
-            tc_commit(bar(BAR_DONE));
-            mbar_wait(bar(BAR_DONE), 0, abort_flag, P.status);
+            if (alive && lead) {
+                tc_commit(bar(BAR_VEMPTY + st));
+                if (j + 1 < n_j) tc_commit(bar(BAR_KEMPTY + nst));
+            }
         }
+        // make sure nothing of ours is still running on the tensor core before TMEM is freed
+        if (lead) tc_commit(bar(BAR_DONE));
+        __syncwarp();
+        mbar_wait(bar(BAR_DONE), 0, abort_flag, P.status);
     } else if (warp < 4) {
         reg_dealloc<72>();
     } else {
@@ -430,11 +449,13 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                     pk[i + 1] = pc_pack_bf16(y.x, y.y);
                 }
                 tmem_st16(s_addr + c * 16, pk);
+                if (c & 1) {                               // keys 0-63, then 64-127, handed to the tensor core
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bar(BAR_PHALF + 2 * t + (c >> 1)));
+                }
             }
             l += (la.x + la.y) + (lb.x + lb.y);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(BAR_PFULL + t));
         }
         // epilogue: O_t is final once the last PV has committed
         if (alive && n_j > 0) alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), n_j & 1, abort_flag, P.status));
