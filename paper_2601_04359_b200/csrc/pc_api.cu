@@ -86,8 +86,6 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
     PC_CUDA_TRY(cudaMallocHost(&c->host_status, 2 * sizeof(int32_t)));
     PC_CUDA_TRY(cudaMalloc(&c->qpool_partial, (size_t)PC_QPOOL_BLOCKS * row * sizeof(float)));
     PC_CUDA_TRY(cudaMalloc(&c->qpool, (size_t)row * sizeof(float)));
-    PC_CUDA_TRY(cudaMalloc(&c->ticket, sizeof(unsigned int)));
-    PC_CUDA_TRY(cudaMemset(c->ticket, 0, sizeof(unsigned int)));
     if (desc->dtype == PC_BF16) {
         pc_status st = pc_attend_tc_scratch(desc, c->sm_count, &c->k_rot_rows, &c->part_o_floats, &c->part_ml_floats);
         if (st != PC_OK) return st;
@@ -108,7 +106,6 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
     cudaFreeHost(c->host_status);
     cudaFree(c->qpool_partial);
     cudaFree(c->qpool);
-    cudaFree(c->ticket);
     for (int i = 0; i < PC_N_MARKS; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     cudaFree(c->k_rot);

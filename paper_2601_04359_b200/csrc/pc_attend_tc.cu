@@ -189,10 +189,33 @@ struct RopeJob {
     const __nv_bfloat16 *src;
     const int32_t *pos;
     __nv_bfloat16 *dst;
-    int n_rows, chunks_per_row /* 16-byte chunks */, first_warp;
+    int n_rows, chunks_per_row /* 16-byte chunks, a multiple of 32 */, first_warp;
     float scale;
 };
 struct RopeJobs { RopeJob job[PC_MAX_SEGMENTS + 1]; int n_jobs, total_warps; };
+
+// One warp per row.  32 lanes x 8 elements = 256 is a multiple of d, so all of a lane's chunks (lane, lane + 32, ...)
+// hold the same four rotary pairs: four table entries per lane per row, with the output scale folded in, serve every
+// chunk.  All of a row's chunks are loaded before any is used.
+template <int CPL /* chunks per lane */>
+__device__ __forceinline__ void rope_row(const RopeJob &J, int row, int lane, const float2 (&cs)[4]) {
+    const uint4 *src = reinterpret_cast<const uint4 *>(J.src) + (size_t)row * (CPL * 32) + lane;
+    uint4 *dst = reinterpret_cast<uint4 *>(J.dst) + (size_t)row * (CPL * 32) + lane;
+    uint4 v[CPL];
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) v[c] = pc_ldg_stream(src + c * 32);
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) {
+        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+        uint32_t o[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float x0 = pc_bf16_lo(w[u]), x1 = pc_bf16_hi(w[u]);
+            o[u] = pc_pack_bf16(x0 * cs[u].x - x1 * cs[u].y, x0 * cs[u].y + x1 * cs[u].x);
+        }
+        dst[c * 32] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
 
 __global__ void __launch_bounds__(256) k_rope_rows(const __grid_constant__ RopeJobs jobs, pc_rope_dev rope, int d,
                                                    int32_t *status) {
@@ -204,23 +227,35 @@ __global__ void __launch_bounds__(256) k_rope_rows(const __grid_constant__ RopeJ
     const RopeJob &J = jobs.job[ji];
     const int row = warp - J.first_warp;
     const int4 pp = __ldg(reinterpret_cast<const int4 *>(J.pos) + row);
-    // 32 lanes x 8 elements = 256 is a multiple of d: all of a lane's chunks hold the same four rotary pairs
     const int pair0 = ((lane * 8) % d) / 2;
     float2 cs[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_ROPE_POS);
-    const uint4 *src = reinterpret_cast<const uint4 *>(J.src) + (size_t)row * J.chunks_per_row;
-    uint4 *dst = reinterpret_cast<uint4 *>(J.dst) + (size_t)row * J.chunks_per_row;
-    for (int c = lane; c < J.chunks_per_row; c += 32) {
-        const uint4 v = pc_ldg_stream(src + c);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t o[4];
+    for (int u = 0; u < 4; ++u) {
+        cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_ROPE_POS);
+        cs[u].x *= J.scale;
+        cs[u].y *= J.scale;
+    }
+    switch (J.chunks_per_row >> 5) {
+    case 4: rope_row<4>(J, row, lane, cs); break;        // 8 KV heads x 128
+    case 12: rope_row<12>(J, row, lane, cs); break;      // 24 query heads x 128
+    case 1: rope_row<1>(J, row, lane, cs); break;
+    case 2: rope_row<2>(J, row, lane, cs); break;
+    case 8: rope_row<8>(J, row, lane, cs); break;
+    case 16: rope_row<16>(J, row, lane, cs); break;
+    default:
+        for (int c = 0; c < (J.chunks_per_row >> 5); ++c) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(J.src) + (size_t)row * J.chunks_per_row + c * 32 + lane;
+            uint4 *dst = reinterpret_cast<uint4 *>(J.dst) + (size_t)row * J.chunks_per_row + c * 32 + lane;
+            const uint4 v = pc_ldg_stream(src);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            uint32_t o[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const float x0 = pc_bf16_lo(w[u]), x1 = pc_bf16_hi(w[u]);
-            o[u] = pc_pack_bf16((x0 * cs[u].x - x1 * cs[u].y) * J.scale, (x0 * cs[u].y + x1 * cs[u].x) * J.scale);
+            for (int u = 0; u < 4; ++u) {
+                const float x0 = pc_bf16_lo(w[u]), x1 = pc_bf16_hi(w[u]);
+                o[u] = pc_pack_bf16(x0 * cs[u].x - x1 * cs[u].y, x0 * cs[u].y + x1 * cs[u].x);
+            }
+            *dst = make_uint4(o[0], o[1], o[2], o[3]);
         }
-        dst[c] = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
 
@@ -605,10 +640,12 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
 
     TcParams P{};
     RopeJobs jobs{};
+    const int k_chunks = row_elems / 8, q_chunks = D.n_q_heads * D.head_dim / 8;
+    if (k_chunks % 32 || q_chunks % 32) return PC_ERR_UNSUPPORTED;
     int tiles = 0, warps = 0;
     for (int s = 0; s < n_seg; ++s) {
         jobs.job[s] = RopeJob{static_cast<const __nv_bfloat16 *>(segs[s].k), segs[s].pos,
-                              k_rot + (size_t)tiles * TILE * row_elems, segs[s].n_tokens, row_elems / 8, warps, 1.0f};
+                              k_rot + (size_t)tiles * TILE * row_elems, segs[s].n_tokens, k_chunks, warps, 1.0f};
         warps += segs[s].n_tokens;
         tiles += div_up(segs[s].n_tokens, TILE);
         P.seg_tile_end[s] = tiles;
@@ -616,7 +653,7 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     }
     if ((size_t)tiles * TILE > ctx->k_rot_rows) return PC_ERR_CAPACITY;
     __nv_bfloat16 *q_rot = static_cast<__nv_bfloat16 *>(ctx->q_rot);
-    jobs.job[n_seg] = RopeJob{static_cast<const __nv_bfloat16 *>(q), q_pos, q_rot, n_q, D.n_q_heads * D.head_dim / 8, warps,
+    jobs.job[n_seg] = RopeJob{static_cast<const __nv_bfloat16 *>(q), q_pos, q_rot, n_q, q_chunks, warps,
                               (float)(1.4426950408889634 / std::sqrt((double)D.head_dim))};
     warps += n_q;
     jobs.n_jobs = n_seg + 1;

@@ -33,7 +33,7 @@ enum {
 enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT = 3, PC_MARK_PACK0 = 4, PC_MARK_PACK = 5,
        PC_MARK_ATT0 = 6, PC_MARK_ROPE = 7, PC_MARK_ATTEND = 8, PC_MARK_COMBINE = 9, PC_N_MARKS = 10 };
 
-constexpr int PC_QPOOL_BLOCKS = 64;
+constexpr int PC_QPOOL_BLOCKS = 128;
 constexpr int PC_MAX_SEGMENTS = 3;
 
 // Rotary tables: for axis a (t, h, w) a [max_pos[a]][n_axis[a]] array of (cos, sin) of pos * base^(-m/n_axis[a]).
@@ -58,7 +58,6 @@ struct pc_ctx {
     int32_t *host_status;      // pinned [2]
     float *qpool_partial;      // device [PC_QPOOL_BLOCKS][Hkv*d]
     float *qpool;              // device [Hkv*d]
-    unsigned int *ticket;      // device, zero between calls
     // attention scratch (tensor-core path)
     void *k_rot;               // rotated keys, bf16 [rows][Hkv][d]
     size_t k_rot_rows;

@@ -31,22 +31,20 @@ template <> struct Elem<__nv_bfloat16> {
 // ---------------------------------------------------------------------------------------------------------
 // Pooled query.  The rotation is the same for every head at a given token and rotary pair, so the heads of a group
 // are added first and the sum is rotated once:  q~[g] = (1/n_q) sum_i R(p_i) (sum_{h in g} q_ih).
-// A block owns a contiguous run of query tokens.  Its 1024 threads form `slices` token slices x n_cols pair-columns
+// A block owns a contiguous run of query tokens.  Its 512 threads form `slices` token slices x n_cols pair-columns
 // of the [Hkv][d/2] pooled grid (a warp reads 128 contiguous bytes of each head); a thread walks its slice's tokens
 // eight at a time with all loads of a batch issued before any is used.  Slices are added in slice order through
-// shared memory, and the last block to finish adds the per-block partials in block order, so the result does not
-// depend on scheduling.
+// shared memory; a second small kernel adds the per-block partials in a fixed order, so the result does not depend
+// on scheduling.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int QPOOL_THREADS = 1024;
+constexpr int QPOOL_THREADS = 512;
 constexpr int QPOOL_BATCH = 8;
 
 template <typename T, int GROUP /* query heads per KV head; 0 = any */>
 __global__ void __launch_bounds__(QPOOL_THREADS) k_qpool(const T *__restrict__ q, const int32_t *__restrict__ q_pos, int n_q,
                                                          int n_q_heads, int group_rt, int d, pc_rope_dev rope,
-                                                         float *__restrict__ partial, float *__restrict__ pooled,
-                                                         unsigned int *ticket, int32_t *status) {
+                                                         float *__restrict__ partial, int32_t *status) {
     __shared__ float2 slice_sum[QPOOL_THREADS];
-    __shared__ bool last;
     const int group = GROUP > 0 ? GROUP : group_rt;
     const int half = d / 2, n_kv = n_q_heads / group, n_cols = n_kv * half, row_len = n_kv * d;
     const size_t q_row = (size_t)n_q_heads * d;
@@ -113,20 +111,25 @@ __global__ void __launch_bounds__(QPOOL_THREADS) k_qpool(const T *__restrict__ q
         }
         __syncthreads();
     }
-    __threadfence();
+}
+
+// pooled[e] = (1/n_q) * sum over blocks of partial[b][e].  32 columns per block; eight threads per column each add
+// every eighth partial (in block order), and the eight sums are added in slice order.
+__global__ void __launch_bounds__(256) k_qpool_reduce(const float *__restrict__ partial, int n_partials, int row_len, float inv_n,
+                                                      float *__restrict__ pooled) {
+    __shared__ float part[8][32];
+    const int c = threadIdx.x & 31, sl = threadIdx.x >> 5, e = blockIdx.x * 32 + c;
+    float acc = 0.f;
+    if (e < row_len)
+        for (int b = sl; b < n_partials; b += 8) acc += __ldcg(partial + (size_t)b * row_len + e);
+    part[sl][c] = acc;
     __syncthreads();
-    if (threadIdx.x == 0) last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
-    const float inv_n = 1.f / (float)n_q;
-    for (int e = threadIdx.x; e < row_len; e += QPOOL_THREADS) {
-        float s = 0.f;
-#pragma unroll 16
-        for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(partial + (size_t)b * row_len + e);
-        pooled[e] = s * inv_n;
+    if (sl == 0 && e < row_len) {
+        float tot = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) tot += part[k][c];
+        pooled[e] = tot * inv_n;
     }
-    if (threadIdx.x == 0) *ticket = 0u;   // ready for the next call
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -406,14 +409,14 @@ __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict_
 // Enqueue pooling and scoring on caller-given scratch (a context's, or the library's fixed array).
 template <typename T>
 pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev &rope, float *partial, float *pooled,
-                        unsigned int *ticket, int32_t *status, const void *hist_k, const int32_t *hist_pos, int n_src,
+                        int32_t *status, const void *hist_k, const int32_t *hist_pos, int n_src,
                         const void *q, const int32_t *q_pos, int32_t n_q, const uint8_t *valid, float *scores,
                         cudaStream_t stream, pc_ctx *marks) {
     const int row = D.n_kv_heads * D.head_dim;
     const int group = D.n_q_heads / D.n_kv_heads;
-    const int pool_blocks = std::min<int>(PC_QPOOL_BLOCKS, (n_q + 15) / 16);
+    const int pool_blocks = std::min<int>(PC_QPOOL_BLOCKS, (n_q + QPOOL_BATCH - 1) / QPOOL_BATCH);
     if (marks) pc_mark(marks, PC_MARK_SCORE0, stream);
-#define PC_QPOOL_ARGS static_cast<const T *>(q), q_pos, n_q, D.n_q_heads, group, D.head_dim, rope, partial, pooled, ticket, status
+#define PC_QPOOL_ARGS static_cast<const T *>(q), q_pos, n_q, D.n_q_heads, group, D.head_dim, rope, partial, status
     switch (group) {
     case 1: k_qpool<T, 1><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
     case 2: k_qpool<T, 2><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
@@ -422,6 +425,8 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
     default: k_qpool<T, 0><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
     }
 #undef PC_QPOOL_ARGS
+    PC_CUDA_TRY(cudaGetLastError());
+    k_qpool_reduce<<<(row + 31) / 32, 256, 0, stream>>>(partial, pool_blocks, row, 1.f / (float)n_q, pooled);
     PC_CUDA_TRY(cudaGetLastError());
     if (marks) pc_mark(marks, PC_MARK_QPOOL, stream);
     const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
@@ -456,7 +461,7 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
 template <typename T>
 pc_status launch_score(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q,
                        const uint8_t *valid, float *scores, cudaStream_t stream) {
-    return enqueue_score<T>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_partial, ctx->qpool, ctx->ticket, ctx->status,
+    return enqueue_score<T>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_partial, ctx->qpool, ctx->status,
                             src->history.k, src->history.pos, src->history.n_tokens, q, q_pos, n_q, valid, scores, stream,
                             ctx);
 }
@@ -518,7 +523,7 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
 // was handed to its own arena at start-up and whose policy forbids driver allocations afterwards, or a
 // latency-critical thread that cannot take the device-wide synchronisation a cudaMalloc / cudaFree implies.  Such
 // callers cannot create a pc_ctx (pc_create allocates), so everything a context would hold for scoring — the rotary
-// table, the pooled query and its per-block partials, the completion ticket — lives in one file-scope device array
+// table, the pooled query and its per-block partials — lives in one file-scope device array
 // of fixed size that every GPU loading this library carries until the process exits.
 //
 // In host code the array's name is only a handle; the device address is obtained once per device with
@@ -530,11 +535,10 @@ constexpr int STATIC_MAX_ROW = 1024;          // n_kv_heads * head_dim
 constexpr int STATIC_MAX_ROPE = 32768;        // rotary table entries: sum over axes of max_pos * pairs on that axis
 constexpr int STATIC_MAX_DEVICES = 64;
 
-constexpr size_t STATIC_OFF_TICKET = 0;                                                    // unsigned, 256-byte slot
-constexpr size_t STATIC_OFF_POOLED = 256;                                                  // float [STATIC_MAX_ROW]
-constexpr size_t STATIC_OFF_PARTIAL = STATIC_OFF_POOLED + STATIC_MAX_ROW * sizeof(float);  // float [64][STATIC_MAX_ROW]
+constexpr size_t STATIC_OFF_POOLED = 256;  /* first 256 bytes unused */                                                  // float [STATIC_MAX_ROW]
+constexpr size_t STATIC_OFF_PARTIAL = STATIC_OFF_POOLED + STATIC_MAX_ROW * sizeof(float);  // float [PC_QPOOL_BLOCKS][STATIC_MAX_ROW]
 constexpr size_t STATIC_OFF_ROPE = STATIC_OFF_PARTIAL + (size_t)PC_QPOOL_BLOCKS * STATIC_MAX_ROW * sizeof(float);
-constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);   // 528,640 bytes
+constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);   // 790,784 bytes
 
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
 
@@ -571,7 +575,6 @@ template <typename T>
 pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const void *hist_k, const int32_t *hist_pos,
                               int32_t n_src, const void *q, const int32_t *q_pos, int32_t n_q, const uint8_t *valid,
                               float *scores, int32_t *status, cudaStream_t stream) {
-    unsigned int *ticket = reinterpret_cast<unsigned int *>(base + STATIC_OFF_TICKET);
     float *pooled = reinterpret_cast<float *>(base + STATIC_OFF_POOLED);
     float *partial = reinterpret_cast<float *>(base + STATIC_OFF_PARTIAL);
     float2 *tab = reinterpret_cast<float2 *>(base + STATIC_OFF_ROPE);
@@ -585,15 +588,15 @@ pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const
         total += D.max_pos[a] * rope.n_axis[a];
     }
     rope.tab = tab;
-    // the array keeps whatever the last call left: the ticket must start at zero, the table is rewritten
-    PC_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), stream));
+    // the array keeps whatever the last call left; the table, the partials and the pooled query are all rewritten before
+    // they are read, and nothing has to start at zero
     k_rope_table<<<(total + 255) / 256, 256, 0, stream>>>(tab, rope, D.rope_base, total);
     PC_CUDA_TRY(cudaGetLastError());
 
     int sm_count = 0, dev = 0;
     PC_CUDA_TRY(cudaGetDevice(&dev));
     PC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    return enqueue_score<T>(D, sm_count, rope, partial, pooled, ticket, status, hist_k, hist_pos, n_src, q, q_pos, n_q,
+    return enqueue_score<T>(D, sm_count, rope, partial, pooled, status, hist_k, hist_pos, n_src, q, q_pos, n_q,
                             valid, scores, stream, nullptr);
 }
 
