@@ -228,6 +228,13 @@ pc_status pc_set_attend_impl(pc_ctx *ctx, int32_t impl);
  * choose the count that fills the GPU's SMs best.  Results agree up to fp32 rounding order. */
 pc_status pc_set_kv_splits(pc_ctx *ctx, int32_t n);
 
+/* How the key ranges of the tensor-core attention kernel are merged: 0 (default) = each range writes fp32 partials to
+ * context scratch and a second kernel merges them; 1 = the ranges of one work item run as a thread-block cluster and
+ * merge inside the kernel through distributed shared memory (no partials in global memory, one launch less).  On a
+ * B200 only 45 clusters of three CTAs are resident at a time (135 of 148 SMs), so the cluster form pays only when the
+ * number of work items fits that; results agree up to fp32 rounding order. */
+pc_status pc_set_cluster_merge(pc_ctx *ctx, int32_t on);
+
 /* Per-kernel timing for benchmarks.  With timing on, each call records CUDA events on its stream at the boundaries
  * of its kernels (a few microseconds of overhead per call); pc_get_timing waits for the last recorded events and
  * writes the duration in milliseconds of each kernel of the most recent calls, -1 for a kernel that did not run.

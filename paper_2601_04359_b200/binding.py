@@ -23,7 +23,7 @@ PC_MAX_FRAMES = 256
 
 EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact", "pc_attend_frame",
            "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_set_timing", "pc_get_timing",
-           "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static"]
+           "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge"]
 
 
 class pc_layer_desc(C.Structure):
@@ -94,6 +94,7 @@ def load() -> C.CDLL:
     lib.pc_poll_status.argtypes = [C.c_void_p, C.c_void_p]
     lib.pc_set_attend_impl.argtypes = [C.c_void_p, C.c_int32]
     lib.pc_set_kv_splits.argtypes = [C.c_void_p, C.c_int32]
+    lib.pc_set_cluster_merge.argtypes = [C.c_void_p, C.c_int32]
     lib.pc_set_timing.argtypes = [C.c_void_p, C.c_int32]
     lib.pc_get_timing.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
     lib.pc_frame_step_host.argtypes = [C.c_void_p, C.POINTER(pc_host_frame), C.POINTER(pc_device_workspace),
@@ -246,6 +247,10 @@ def pc_set_attend_impl(ctx: Context, impl: int) -> None:
 
 def pc_set_kv_splits(ctx: Context, n: int) -> None:
     _check(load().pc_set_kv_splits(ctx.handle, n), "pc_set_kv_splits")
+
+
+def pc_set_cluster_merge(ctx: Context, on: bool) -> None:
+    _check(load().pc_set_cluster_merge(ctx.handle, 1 if on else 0), "pc_set_cluster_merge")
 
 
 def pc_set_timing(ctx: Context, on: bool) -> None:

@@ -51,6 +51,7 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
     c->elem_size = desc->dtype == PC_BF16 ? 2 : 4;
     c->attend_impl = 0;
     c->kv_splits = 0;
+    c->cluster_merge = 0;
     c->timing_on = 0;
     c->ev_mask = 0;
     for (int i = 0; i < PC_N_MARKS; ++i) c->ev[i] = nullptr;
@@ -125,6 +126,12 @@ extern "C" pc_status pc_set_attend_impl(pc_ctx *c, int32_t impl) {
 extern "C" pc_status pc_set_kv_splits(pc_ctx *c, int32_t n) {
     if (!c || n < 0 || n > 4) return PC_ERR_INVALID_ARG;
     c->kv_splits = n;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_set_cluster_merge(pc_ctx *c, int32_t on) {
+    if (!c || on < 0 || on > 1) return PC_ERR_INVALID_ARG;
+    c->cluster_merge = on;
     return PC_OK;
 }
 

@@ -11,7 +11,9 @@
 //                 bf16 P over S in TMEM (handed over in two halves of 64 keys), and rescale O in TMEM only when
 //                 the running max moved by more than 2^8.
 //                 While one tile's softmax runs, the tensor core works on the other tile.
-//   k_combine     merges the KV ranges' (max, sum, O) partials when the keys were split across CTAs.
+//   Key ranges of one work item are launched as a thread-block cluster and merge their (max, sum, O) through
+//   distributed shared memory at the end of the kernel; k_combine does the same from global partials when the
+//   cluster merge is switched off.
 //
 // TMEM columns: S0/P0 0-127, S1/P1 128-255, O0 256-383, O1 384-511 (fp32, 128 lanes = the tile's rows).
 // Every wait is bounded: a wait that runs out records PC_ERR_TIMEOUT, raises a CTA-wide abort flag that makes every
@@ -37,7 +39,8 @@ constexpr int SM_Q = 0;                                   // 2 tiles
 constexpr int SM_K = SM_Q + 2 * TILE_BYTES;               // KV_STAGES tiles
 constexpr int SM_V = SM_K + KV_STAGES * TILE_BYTES;       // KV_STAGES tiles
 constexpr int SM_BAR = SM_V + KV_STAGES * TILE_BYTES;     // barriers etc.
-constexpr int SM_TOTAL = SM_BAR + 256;
+constexpr int SM_ML = SM_BAR + 256;                       // (max, sum) of both tiles' rows for the cluster merge: 2 KB
+constexpr int SM_TOTAL = SM_ML + 2 * TILE * 8;
 constexpr int SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
 
 enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PHALF = 11 /* [tile][half] */,
@@ -46,6 +49,7 @@ enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, 
 struct TcParams {
     int n_q, n_q_heads, group, n_tb, tiles_per_g, pairs_per_g, n_splits, n_kv_tiles;
     int n_seg;
+    int cluster;      // 1: the KV ranges of one item form a thread-block cluster and merge through shared memory
     int seg_tile_end[PC_MAX_SEGMENTS];
     int seg_n[PC_MAX_SEGMENTS];
     __nv_bfloat16 *out;
@@ -160,6 +164,38 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b) {
 }
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// thread-block cluster: rank, barrier, and reads of a peer CTA's shared memory
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t rank) {
+    uint32_t a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local), "r"(rank));
+    return a;
+}
+__device__ __forceinline__ float4 peer_ld128(uint32_t a) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 peer_ld64(uint32_t a) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+// Staging layout of one tile's fp32 O for the merge: 16-byte unit (c4, r) = columns 4*c4..4*c4+3 of row r sits at unit
+// c4*128 + ((r + c4) & 127): a warp writing 32 rows of one c4 and a half-warp reading 16 c4 of one row both spread
+// over the banks.
+__device__ __forceinline__ uint32_t stage_off(int c4, int r) { return (uint32_t)(c4 * TILE + ((r + c4) & (TILE - 1))) * 16u; }
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -519,6 +555,19 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                     }
                 }
                 if (P.lse && row < P.n_q) P.lse[(size_t)row * P.n_q_heads + h] = (m_used + log2f(l)) * 0.6931471805599453f;
+            } else if (P.cluster) {
+                // Stage O (un-normalised, fp32) and (max, sum) in shared memory that no multiply-add reads any more:
+                // tile 0 over both query tiles (every QK^T has completed once this tile's last PV has), tile 1 over the
+                // key stages (its own last PV is the last multiply-add of the CTA).
+                const uint32_t stage = base + (t == 0 ? SM_Q : SM_K);
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    tmem_ld32(o_addr + c * 32, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) sts128(stage + stage_off(c * 8 + i, r), v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                }
+                *reinterpret_cast<float2 *>(gen + SM_ML + (t * TILE + r) * 8) = make_float2(m_used, l);
             } else {
                 const size_t slot = ((size_t)blockIdx.x * 2 + t) * TILE + r;
                 float *prow = P.part_o + slot * TILE;
@@ -540,10 +589,57 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
     }
+    if (P.cluster && P.n_splits > 1) {
+        // Merge the KV ranges of this item across the cluster: CTA `rank` finishes every n_splits-th row of the two
+        // tiles, reading each peer's staged O and (max, sum) through distributed shared memory.  Sixteen threads share
+        // a row (two 16-byte units each), so a row's 256 output bytes leave as two 128-byte runs.
+        cluster_sync_all();                        // every CTA's staging is complete and visible
+        if (warp >= 4) {
+            const int S = P.n_splits, my = (int)cluster_rank();
+            const int id = threadIdx.x - 128, sub = id & 15, slot = id >> 4;
+            uint32_t peer_base[MAX_SPLITS];
+#pragma unroll
+            for (int k = 0; k < MAX_SPLITS; ++k) peer_base[k] = peer_addr(base, k < S ? k : 0);
+            for (int R = my + slot * S; R < 2 * TILE; R += 16 * S) {
+                const int t = R >> 7, r = R & (TILE - 1);
+                if (t >= n_tiles_q) break;
+                const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
+                const int row = tb * TILE + r;
+                if (row >= P.n_q) continue;
+                float mk[MAX_SPLITS], lk[MAX_SPLITS], m = -INFINITY;
+#pragma unroll
+                for (int k = 0; k < MAX_SPLITS; ++k)
+                    if (k < S) {
+                        const float2 ml = peer_ld64(peer_base[k] + SM_ML + (t * TILE + r) * 8);
+                        mk[k] = ml.x; lk[k] = ml.y;
+                        m = fmaxf(m, ml.x);
+                    }
+                float lsum = 0.f;
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+                const uint32_t stage = (t == 0 ? SM_Q : SM_K);
+#pragma unroll
+                for (int k = 0; k < MAX_SPLITS; ++k)
+                    if (k < S) {
+                        const float sc = exp2f(mk[k] - m);
+                        lsum = fmaf(lk[k], sc, lsum);
+                        const float4 x = peer_ld128(peer_base[k] + stage + stage_off(sub, r));
+                        const float4 y = peer_ld128(peer_base[k] + stage + stage_off(sub + 16, r));
+                        a.x = fmaf(x.x, sc, a.x); a.y = fmaf(x.y, sc, a.y); a.z = fmaf(x.z, sc, a.z); a.w = fmaf(x.w, sc, a.w);
+                        b.x = fmaf(y.x, sc, b.x); b.y = fmaf(y.y, sc, b.y); b.z = fmaf(y.z, sc, b.z); b.w = fmaf(y.w, sc, b.w);
+                    }
+                const float inv = 1.f / lsum;
+                __nv_bfloat16 *orow = P.out + ((size_t)row * P.n_q_heads + h) * TILE;
+                *reinterpret_cast<uint2 *>(orow + 4 * sub) = make_uint2(pc_pack_bf16(a.x * inv, a.y * inv), pc_pack_bf16(a.z * inv, a.w * inv));
+                *reinterpret_cast<uint2 *>(orow + 64 + 4 * sub) = make_uint2(pc_pack_bf16(b.x * inv, b.y * inv), pc_pack_bf16(b.z * inv, b.w * inv));
+                if (P.lse && sub == 0) P.lse[(size_t)row * P.n_q_heads + h] = (m + log2f(lsum)) * 0.6931471805599453f;
+            }
+        }
+        cluster_sync_all();                        // nobody leaves while a peer may still read its shared memory
+    }
 }
 
 // ------------------------------------------------------------------------------------------------ combine
-// One warp per (query row, head): merges the KV ranges' partials in range order.
+// One warp per (query row, head): merges the KV ranges' partials in range order.  Every load is issued before any is used.
 __global__ void __launch_bounds__(256) k_combine(const TcParams P) {
     const int lane = threadIdx.x & 31;
     const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -551,21 +647,28 @@ __global__ void __launch_bounds__(256) k_combine(const TcParams P) {
     const int row = w / P.n_q_heads, h = w % P.n_q_heads;
     const int g = h / P.group, T = (row / TILE) * P.group + h % P.group;
     const int item = g * P.pairs_per_g + T / 2, t = T & 1, r = row % TILE;
+    float2 ml[MAX_SPLITS];
+    float4 o[MAX_SPLITS];
+#pragma unroll
+    for (int s = 0; s < MAX_SPLITS; ++s)
+        if (s < P.n_splits) {
+            const size_t slot = ((size_t)(item * P.n_splits + s) * 2 + t) * TILE + r;
+            ml[s] = __ldcg(reinterpret_cast<const float2 *>(P.part_ml + slot * 2));
+            o[s] = __ldcg(reinterpret_cast<const float4 *>(P.part_o + slot * TILE) + lane);
+        }
     float m = -INFINITY;
-    for (int s = 0; s < P.n_splits; ++s) {
-        const size_t slot = ((size_t)(item * P.n_splits + s) * 2 + t) * TILE + r;
-        m = fmaxf(m, __ldcg(P.part_ml + slot * 2));
-    }
+#pragma unroll
+    for (int s = 0; s < MAX_SPLITS; ++s)
+        if (s < P.n_splits) m = fmaxf(m, ml[s].x);
     float l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < P.n_splits; ++s) {
-        const size_t slot = ((size_t)(item * P.n_splits + s) * 2 + t) * TILE + r;
-        const float2 ml = __ldcg(reinterpret_cast<const float2 *>(P.part_ml + slot * 2));
-        const float sc = exp2f(ml.x - m);
-        const float4 o = __ldcg(reinterpret_cast<const float4 *>(P.part_o + slot * TILE) + lane);
-        l = fmaf(ml.y, sc, l);
-        acc.x = fmaf(o.x, sc, acc.x); acc.y = fmaf(o.y, sc, acc.y); acc.z = fmaf(o.z, sc, acc.z); acc.w = fmaf(o.w, sc, acc.w);
-    }
+#pragma unroll
+    for (int s = 0; s < MAX_SPLITS; ++s)
+        if (s < P.n_splits) {
+            const float sc = exp2f(ml[s].x - m);
+            l = fmaf(ml[s].y, sc, l);
+            acc.x = fmaf(o[s].x, sc, acc.x); acc.y = fmaf(o[s].y, sc, acc.y); acc.z = fmaf(o[s].z, sc, acc.z); acc.w = fmaf(o[s].w, sc, acc.w);
+        }
     const float inv = 1.f / l;
     uint2 out = make_uint2(pc_pack_bf16(acc.x * inv, acc.y * inv), pc_pack_bf16(acc.z * inv, acc.w * inv));
     *reinterpret_cast<uint2 *>(P.out + ((size_t)row * P.n_q_heads + h) * TILE + lane * 4) = out;
@@ -678,7 +781,7 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     P.part_o = ctx->part_o;
     P.part_ml = ctx->part_ml;
     P.status = ctx->status;
-    if (P.n_splits > 1 && (size_t)n_items * P.n_splits * 2 * TILE * TILE > ctx->part_o_floats) return PC_ERR_CAPACITY;
+    if (P.n_splits > 1 && !ctx->cluster_merge && (size_t)n_items * P.n_splits * 2 * TILE * TILE > ctx->part_o_floats) return PC_ERR_CAPACITY;
 
     CUtensorMap mq, mk, mv[PC_MAX_SEGMENTS];
     bool ok = make_map(&mq, q_rot, (uint64_t)n_q, (uint64_t)D.n_q_heads * D.head_dim) &&
@@ -696,10 +799,27 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
         PC_CUDA_TRY(cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
         attr_set = true;
     }
-    k_attend_tc<<<n_items * P.n_splits, TC_THREADS, SM_ALLOC, stream>>>(mq, mk, mv[0], mv[1], mv[2], P);
+    P.cluster = (P.n_splits > 1 && ctx->cluster_merge) ? 1 : 0;
+    if (P.cluster) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(n_items * P.n_splits);
+        cfg.blockDim = dim3(TC_THREADS);
+        cfg.dynamicSmemBytes = SM_ALLOC;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = P.n_splits;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        PC_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_attend_tc, mq, mk, mv[0], mv[1], mv[2], P));
+    } else {
+        k_attend_tc<<<n_items * P.n_splits, TC_THREADS, SM_ALLOC, stream>>>(mq, mk, mv[0], mv[1], mv[2], P);
+    }
     PC_CUDA_TRY(cudaGetLastError());
     pc_mark(ctx, PC_MARK_ATTEND, stream);
-    if (P.n_splits > 1) {
+    if (P.n_splits > 1 && !P.cluster) {
         k_combine<<<div_up(n_q * D.n_q_heads, 8), 256, 0, stream>>>(P);
         PC_CUDA_TRY(cudaGetLastError());
         pc_mark(ctx, PC_MARK_COMBINE, stream);

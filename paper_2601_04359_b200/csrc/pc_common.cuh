@@ -63,6 +63,7 @@ struct pc_ctx {
     size_t k_rot_rows;
     void *q_rot;               // rotated, pre-scaled queries, bf16 [max_q][Hq][d]
     int kv_splits;             // 0 = chosen per call
+    int cluster_merge;         // 1 = KV ranges merge inside the kernel through cluster shared memory (default 0)
     // optional per-kernel timing (benchmarks): events at the boundaries of the kernels of each call
     int timing_on;
     unsigned ev_mask;

@@ -149,6 +149,31 @@ def test_unlimited_budget_equals_full_cache_attention():
     assert np.abs(host(a) - full).max() <= BF16_ATOL
 
 
+# ------------------------------------------------------------------------------------------- split-KV merge
+@pytest.mark.parametrize("cluster", [True, False])
+def test_attention_key_ranges_merge_like_one_range(cluster):
+    """Every split count (1-4 key ranges), merged inside the kernel through cluster shared memory or by the separate
+    merge kernel, against the oracle; anchors and history of ragged length, with and without the current frame."""
+    cfg = wl.small_bf16(n_frames=4, grid=(12, 21), n_text=130, total=700, keep_full=1, seed=11)
+    L = wl.make_layer(cfg, with_current=True)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    pc.pc_set_cluster_merge(ctx, cluster)
+    segs = [(L.anchor_k, L.anchor_v, L.anchor_pos), (L.hist_k, L.hist_v, L.hist_pos), (L.cur_k, L.cur_v, L.q_pos)]
+    want, want_lse = oracle.attend(L.q, L.q_pos, segs, cfg.rope_base, want_lse=True)
+    outs = []
+    for n in (1, 2, 3, 4):
+        pc.pc_set_kv_splits(ctx, n)
+        out, lse = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos, want_lse=True)
+        _ok(ctx)
+        assert np.abs(host(out).astype(np.float64) - want).max() <= BF16_ATOL
+        assert np.abs(host(lse) - want_lse).max() <= 2e-2
+        outs.append(host(out))
+    for o in outs[1:]:                       # the split only changes fp32 rounding order: at most a bf16 ulp or two
+        assert (np.abs(o - outs[0]) <= 2.0 ** -6 * np.maximum(np.abs(outs[0]), 0.5)).all()
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------------- select
 def _select_case(frame_count, budget, scores, cfg=None):
     cfg = cfg or wl.CONFIGS["tiny"]

@@ -12,6 +12,7 @@ This file sorts last on purpose: a run that stops at the first failure has alrea
 from __future__ import annotations
 
 import ctypes as C
+import gc
 
 import numpy as np
 import pytest
@@ -40,11 +41,12 @@ def _both(cfg, layer):
     # buffers exist before the call; the call itself must not need any more memory
     scores = torch.full((cfg.n_src,), float("nan"), dtype=torch.float32, device="cuda")
     status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    gc.collect()                       # tensors of earlier tests must not be freed in the middle of the measurement
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
     pc.pc_score_tokens_static(_desc(cfg), D.cache.history.k, D.cache.history.pos, cfg.n_src, D.q, D.q_pos, scores, status)
     torch.cuda.synchronize()
-    assert torch.cuda.memory_allocated() == before
+    assert torch.cuda.memory_allocated() <= before          # the call took no device memory from torch's allocator
     assert status.cpu().tolist() == [0, 0]
     ctx.close()
     return host(want)[:cfg.n_src].astype(np.float64), host(scores).astype(np.float64), L.frame_count
