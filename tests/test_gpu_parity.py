@@ -313,7 +313,7 @@ def test_device_side_checks_record_instead_of_faulting():
 
 
 # ------------------------------------------------------------------------------------------- full size
-@pytest.mark.parametrize("name", ["lumos12", "lumos47"])
+@pytest.mark.parametrize("name", ["lumos12", "lumos24", "lumos47"])
 def test_full_size_sampled_against_oracle(name):
     """The benchmark's launch configuration at full size: scores against the pooled fp64 oracle on every token and
     the mean-logit oracle on a sample; selection and packing bit-exact; attention on sampled (query, head) rows."""
@@ -355,4 +355,58 @@ def test_full_size_sampled_against_oracle(name):
     assert np.abs(o[rows[:, 0], rows[:, 1]] - want).max() <= BF16_ATOL
     assert np.abs(host(lse)[rows[:, 0], rows[:, 1]] - want_lse).max() <= 2e-2
     assert np.isfinite(o).all()
+    ctx.close()
+
+
+def test_full_cache_comparator_at_24_frames():
+    """Attention over the uncompacted cache (anchors ++ all 24 history frames, 25,328 keys): the comparator the
+    24-frame configuration is measured against, on sampled (query, head) rows."""
+    cfg = wl.CONFIGS["lumos24"]
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    out, lse = pc.pc_attend_frame(ctx, D.cache, None, D.q, D.q_pos, want_lse=True)
+    _ok(ctx)
+    rng = np.random.default_rng(2)
+    rows = np.stack([rng.integers(0, cfg.n_q, size=48), rng.integers(0, cfg.n_q_heads, size=48)], axis=1).astype(np.int32)
+    rows[0] = (0, 0); rows[1] = (cfg.n_q - 1, cfg.n_q_heads - 1)
+    want, want_lse = oracle.attend(L.q, L.q_pos, [(L.anchor_k, L.anchor_v, L.anchor_pos), (L.hist_k, L.hist_v, L.hist_pos)],
+                                   rows=rows, want_lse=True)
+    o = host(out)
+    assert np.abs(o[rows[:, 0], rows[:, 1]] - want).max() <= BF16_ATOL
+    assert np.abs(host(lse)[rows[:, 0], rows[:, 1]] - want_lse).max() <= 2e-2
+    assert np.isfinite(o).all()
+    ctx.close()
+
+
+@pytest.mark.parametrize("layer,frac,kind,param", [(3, 0.10, wl.HALFLIFE, 2.0), (17, 0.50, wl.LINEAR, 0.0),
+                                                   (27, 1.00, wl.HALFLIFE, 8.0)])
+def test_layer_stack_cells_sampled(layer, frac, kind, param):
+    """Cells of the 28-layer sweep (layer, budget fraction, decay): each layer has its own seeded tensors; budgets
+    bit-exact, selection and packing bit-exact on the oracle's scores, attention on sampled rows."""
+    base = wl.CONFIGS["stack28"]
+    cfg = wl.with_budget(base, kind=kind, param=param, total=int(frac * base.n_src), keep_full=0)
+    L = wl.make_layer(cfg, layer=layer)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    budget = _plan(cfg)
+    assert budget.sum() == min(cfg.budget.total, cfg.n_src)
+    scores, sel = pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget)
+    ref = oracle.score_pooled(L.hist_k, L.hist_pos, L.q, L.q_pos)
+    assert (np.abs(host(scores).astype(np.float64) - ref) <= score_tolerance(ref, L.frame_count)).all()
+    _valid_topk(host(scores), sel.cpu().numpy(), L.frame_count, budget)
+    ref32 = ref.astype(np.float32)
+    _, sel2 = pc.pc_score(ctx, D.cache, None, None, budget, scores_override=torch.from_numpy(ref32).cuda())
+    want_sel = oracle.select(ref32, L.frame_count, budget)
+    assert np.array_equal(sel2.cpu().numpy()[:len(want_sel)], want_sel)
+    dst = D.empty_packed(int(budget.sum()))
+    pc.pc_compact(ctx, D.cache, sel2, budget, 0, dst)
+    wk, wv, wp = oracle.pack(L.hist_k, L.hist_v, L.hist_pos, want_sel, 0)
+    assert np.array_equal(host(dst.history.k), wk) and np.array_equal(dst.history.pos.cpu().numpy(), wp)
+    out = pc.pc_attend_frame(ctx, dst, None, D.q, D.q_pos)
+    _ok(ctx)
+    rng = np.random.default_rng(layer)
+    rows = np.stack([rng.integers(0, cfg.n_q, size=32), rng.integers(0, cfg.n_q_heads, size=32)], axis=1).astype(np.int32)
+    want = oracle.attend(L.q, L.q_pos, [(L.anchor_k, L.anchor_v, L.anchor_pos), (wk, wv, wp)], rows=rows)
+    assert np.abs(host(out)[rows[:, 0], rows[:, 1]] - want).max() <= BF16_ATOL
     ctx.close()
