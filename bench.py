@@ -31,6 +31,10 @@ METRIC = "late_frame_attn_plus_compaction_latency"
 UNIT = "ms/frame"
 WORKLOAD = "lumos47"
 N_LAYERS = 4          # rotated input sets; 4 x ~0.2 GB > L2 (--layers changes it for small profiler captures)
+KERNELS_PER_STEP = 8  # k_qpool, k_qpool_reduce, k_score, k_select, k_pack, k_rope_rows, k_attend_tc, k_combine
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_attend_tc launch at this workload, from the ncu capture
+# summarised in profiles/ncu_kernels_lumos47_small_case.md (same launch shape); None when the kernel has changed since
+ATTEND_DRAM_TRAFFIC = 43_997_696 + 2_566_656
 
 
 def _peaks():
@@ -311,9 +315,9 @@ def run_cuda(args):
         "clocks": clocks,
         "e2e": {"value": (e2e_ms / world) if n_e2e else None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": n_e2e},
-        "gpu_launches": 7 * args.steps,
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"kernel": "k_attend_tc", "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
-                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": ATTEND_DRAM_TRAFFIC,
                      "peak_source": f"{peaks['source']} (burst; sustained {peaks['bf16_tflops_sustained']})",
                      "flops_per_launch": flops, "ms_per_launch": att_ms},
         "kernels_ms": stages,
