@@ -39,6 +39,8 @@ __global__ void __launch_bounds__(AT_THREADS) k_attend_simt(const T *__restrict_
                                                             int n_q, int n_q_heads, int n_kv_heads, SegTable seg,
                                                             pc_rope_dev rope, T *__restrict__ out,
                                                             float *__restrict__ lse, int32_t *status) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
     constexpr int NC = D / 16;                       // 4-element groups per thread
     __shared__ __align__(16) float sk[AT_KEYS][D];
     __shared__ __align__(16) float sv[AT_KEYS][D];
@@ -160,7 +162,7 @@ pc_status pc_launch_attend_simt(pc_ctx *ctx, int n_seg, const pc_segment *segs, 
     dim3 grid((n_q + AT_ROWS - 1) / AT_ROWS, D.n_q_heads);
     pc_mark(ctx, PC_MARK_ROPE, stream);
 #define PC_AT_LAUNCH(T, DIM)                                                                                          \
-    k_attend_simt<T, DIM><<<grid, AT_THREADS, 0, stream>>>(static_cast<const T *>(q), q_pos, n_q, D.n_q_heads,         \
+    PC_LAUNCH((k_attend_simt<T, DIM>), dim3(grid), dim3(AT_THREADS), 0, stream, static_cast<const T *>(q), q_pos, n_q, D.n_q_heads,         \
                                                           D.n_kv_heads, t, ctx->rope, static_cast<T *>(out), lse,    \
                                                           ctx->status)
     if (D.dtype == PC_F32) {

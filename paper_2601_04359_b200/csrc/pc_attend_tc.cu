@@ -255,6 +255,8 @@ __device__ __forceinline__ void rope_row(const RopeJob &J, int row, int lane, co
 
 __global__ void __launch_bounds__(256) k_rope_rows(const __grid_constant__ RopeJobs jobs, pc_rope_dev rope, int d,
                                                    int32_t *status) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (warp >= jobs.total_warps) return;
@@ -308,6 +310,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
             const __grid_constant__ CUtensorMap map_v0, const __grid_constant__ CUtensorMap map_v1,
             const __grid_constant__ CUtensorMap map_v2, const __grid_constant__ TcParams P) {
+    pc_grid_dep_launch();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
@@ -351,6 +354,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    pc_grid_dep_wait();   // barriers and TMEM are set up; from here on the rotated K / Q of the pre-pass are read
 
     // the softmax warps hold a whole 128-column score row per thread: registers move from warps 0-3 to warps 4-11
     if (warp == 0) {
@@ -641,6 +645,8 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
 // ------------------------------------------------------------------------------------------------ combine
 // One warp per (query row, head): merges the KV ranges' partials in range order.  Every load is issued before any is used.
 __global__ void __launch_bounds__(256) k_combine(const TcParams P) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
     const int lane = threadIdx.x & 31;
     const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (w >= P.n_q * P.n_q_heads) return;
@@ -762,7 +768,7 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     jobs.n_jobs = n_seg + 1;
     jobs.total_warps = warps;
     pc_mark(ctx, PC_MARK_ATT0, stream);
-    k_rope_rows<<<div_up(warps, 8), 256, 0, stream>>>(jobs, ctx->rope, D.head_dim, ctx->status);
+    PC_LAUNCH(k_rope_rows, dim3(div_up(warps, 8)), dim3(256), 0, stream, jobs, ctx->rope, D.head_dim, ctx->status);
     PC_CUDA_TRY(cudaGetLastError());
     pc_mark(ctx, PC_MARK_ROPE, stream);
 
@@ -815,12 +821,12 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
         cfg.numAttrs = 1;
         PC_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_attend_tc, mq, mk, mv[0], mv[1], mv[2], P));
     } else {
-        k_attend_tc<<<n_items * P.n_splits, TC_THREADS, SM_ALLOC, stream>>>(mq, mk, mv[0], mv[1], mv[2], P);
+        PC_LAUNCH(k_attend_tc, dim3(n_items * P.n_splits), dim3(TC_THREADS), SM_ALLOC, stream, mq, mk, mv[0], mv[1], mv[2], P);
     }
     PC_CUDA_TRY(cudaGetLastError());
     pc_mark(ctx, PC_MARK_ATTEND, stream);
     if (P.n_splits > 1 && !P.cluster) {
-        k_combine<<<div_up(n_q * D.n_q_heads, 8), 256, 0, stream>>>(P);
+        PC_LAUNCH(k_combine, dim3(div_up(n_q * D.n_q_heads, 8)), dim3(256), 0, stream, P);
         PC_CUDA_TRY(cudaGetLastError());
         pc_mark(ctx, PC_MARK_COMBINE, stream);
     }

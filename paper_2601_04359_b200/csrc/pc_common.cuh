@@ -166,6 +166,32 @@ __device__ __forceinline__ void pc_fma2(float2 &d, float2 a, float2 b) {
         : "+f"(d.x), "+f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
 }
 
+// ---- programmatic dependent launch
+// Every kernel of the library is launched with programmatic stream serialisation: it may start while the kernel before
+// it in the stream is still draining.  A kernel lets its own dependents go at its very start (pc_grid_dep_launch) and
+// must not touch global memory before pc_grid_dep_wait, which returns once the preceding kernel has completed and its
+// writes are visible; only set-up that needs no global data (barrier initialisation, TMEM allocation) goes before it.
+__device__ __forceinline__ void pc_grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pc_grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t pc_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// launch + error check in one statement (returns PC_ERR_CUDA from the calling function on failure)
+#define PC_LAUNCH(kernel, grid, block, smem, stream, ...) PC_CUDA_TRY(pc_launch(kernel, grid, block, smem, stream, __VA_ARGS__))
+
 inline void pc_mark(pc_ctx *c, int idx, cudaStream_t s) {
     if (c->timing_on && c->ev[idx] && cudaEventRecord(c->ev[idx], s) == cudaSuccess) c->ev_mask |= 1u << idx;
 }

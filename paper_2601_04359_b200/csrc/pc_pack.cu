@@ -16,6 +16,8 @@ __global__ void __launch_bounds__(PACK_THREADS) k_pack(const char *__restrict__ 
                                                        int row_bytes, int delta_t, char *__restrict__ dst_k,
                                                        char *__restrict__ dst_v, int32_t *__restrict__ dst_pos,
                                                        int32_t *status) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
     const int lane = threadIdx.x & 31;
     const int r = (blockIdx.x * PACK_THREADS + threadIdx.x) >> 5;
     if (r >= n_sel) return;
@@ -90,10 +92,10 @@ extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t 
 #define PC_PACK_ARGS sk, sv, src->history.pos, sel_idx, (int)n_sel, (int)n_src, row_bytes, delta_t, dk, dv, D.pos, ctx->status
     pc_mark(ctx, PC_MARK_PACK0, stream);
     switch (row_bytes) {
-    case 512: k_pack<1><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
-    case 1024: k_pack<2><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
-    case 2048: k_pack<4><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
-    default: k_pack<0><<<blocks, PACK_THREADS, 0, stream>>>(PC_PACK_ARGS); break;
+    case 512: PC_LAUNCH((k_pack<1>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+    case 1024: PC_LAUNCH((k_pack<2>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+    case 2048: PC_LAUNCH((k_pack<4>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+    default: PC_LAUNCH((k_pack<0>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
     }
 #undef PC_PACK_ARGS
     PC_CUDA_TRY(cudaGetLastError());

@@ -44,6 +44,8 @@ template <typename T, int GROUP /* query heads per KV head; 0 = any */>
 __global__ void __launch_bounds__(QPOOL_THREADS) k_qpool(const T *__restrict__ q, const int32_t *__restrict__ q_pos, int n_q,
                                                          int n_q_heads, int group_rt, int d, pc_rope_dev rope,
                                                          float *__restrict__ partial, int32_t *status) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
     __shared__ float2 slice_sum[QPOOL_THREADS];
     const int group = GROUP > 0 ? GROUP : group_rt;
     const int half = d / 2, n_kv = n_q_heads / group, n_cols = n_kv * half, row_len = n_kv * d;
@@ -117,6 +119,8 @@ __global__ void __launch_bounds__(QPOOL_THREADS) k_qpool(const T *__restrict__ q
 // every eighth partial (in block order), and the eight sums are added in slice order.
 __global__ void __launch_bounds__(256) k_qpool_reduce(const float *__restrict__ partial, int n_partials, int row_len, float inv_n,
                                                       float *__restrict__ pooled) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
     __shared__ float part[8][32];
     const int c = threadIdx.x & 31, sl = threadIdx.x >> 5, e = blockIdx.x * 32 + c;
     float acc = 0.f;
@@ -150,6 +154,7 @@ __global__ void __launch_bounds__(SCORE_THREADS) k_score(const T *__restrict__ k
                                                          const uint8_t *__restrict__ valid, int n_src, int d, float scale,
                                                          pc_rope_dev rope, const float *__restrict__ pooled,
                                                          float *__restrict__ scores, int32_t *status) {
+    pc_grid_dep_launch();
     constexpr int PER = Elem<T>::PER16, NP = PER / 2;
     constexpr uint32_t ROW_BYTES = CPL * 32 * 16;
     constexpr uint32_t STAGE_BYTES = SCORE_TOK * ROW_BYTES + SCORE_TOK * 16;
@@ -167,6 +172,7 @@ __global__ void __launch_bounds__(SCORE_THREADS) k_score(const T *__restrict__ k
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    pc_grid_dep_wait();   // the pooled query comes from the kernel before
     const int n_tiles = (n_src + SCORE_TOK - 1) / SCORE_TOK;
 
     if (warp == SCORE_TOK) {
@@ -327,6 +333,8 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int &
 
 __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict__ scores, const __grid_constant__ FrameTab tab,
                                                        int32_t *__restrict__ sel_idx, int32_t *status) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
     __shared__ uint32_t keys[SEL_CACHE];
     __shared__ int hist[256];
     __shared__ int warp_sums[SEL_THREADS / 32];
@@ -418,15 +426,15 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
     if (marks) pc_mark(marks, PC_MARK_SCORE0, stream);
 #define PC_QPOOL_ARGS static_cast<const T *>(q), q_pos, n_q, D.n_q_heads, group, D.head_dim, rope, partial, status
     switch (group) {
-    case 1: k_qpool<T, 1><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
-    case 2: k_qpool<T, 2><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
-    case 3: k_qpool<T, 3><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
-    case 4: k_qpool<T, 4><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
-    default: k_qpool<T, 0><<<pool_blocks, QPOOL_THREADS, 0, stream>>>(PC_QPOOL_ARGS); break;
+    case 1: PC_LAUNCH((k_qpool<T, 1>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
+    case 2: PC_LAUNCH((k_qpool<T, 2>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
+    case 3: PC_LAUNCH((k_qpool<T, 3>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
+    case 4: PC_LAUNCH((k_qpool<T, 4>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
+    default: PC_LAUNCH((k_qpool<T, 0>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
     }
 #undef PC_QPOOL_ARGS
     PC_CUDA_TRY(cudaGetLastError());
-    k_qpool_reduce<<<(row + 31) / 32, 256, 0, stream>>>(partial, pool_blocks, row, 1.f / (float)n_q, pooled);
+    PC_LAUNCH(k_qpool_reduce, dim3((row + 31) / 32), dim3(256), 0, stream, partial, pool_blocks, row, 1.f / (float)n_q, pooled);
     PC_CUDA_TRY(cudaGetLastError());
     if (marks) pc_mark(marks, PC_MARK_QPOOL, stream);
     const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
@@ -445,7 +453,7 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
             per_sm = std::max(1, occ);                                                                              \
         }                                                                                                           \
         const int blocks = std::max(1, std::min(n_tiles, sm_count * per_sm));                                       \
-        k_score<T, CPL><<<blocks, SCORE_THREADS, smem, stream>>>(k, hist_pos, valid, n_src, D.head_dim, scale, rope, \
+        PC_LAUNCH((k_score<T, CPL>), dim3(blocks), dim3(SCORE_THREADS), smem, stream, k, hist_pos, valid, n_src, D.head_dim, scale, rope, \
                                                                  pooled, scores, status);                          \
     } break;
     switch (chunks / 32) {
@@ -509,7 +517,7 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
     }
     if (n_frames > 0 && out > 0) {
         if (scores_override) pc_mark(ctx, PC_MARK_SCORE, stream);
-        k_select<<<n_frames, SEL_THREADS, 0, stream>>>(select_on, tab, sel_idx, ctx->status);
+        PC_LAUNCH(k_select, dim3(n_frames), dim3(SEL_THREADS), 0, stream, select_on, tab, sel_idx, ctx->status);
         PC_CUDA_TRY(cudaGetLastError());
         pc_mark(ctx, PC_MARK_SELECT, stream);
     }
@@ -544,6 +552,8 @@ static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
 
 // Rotary table in fp64, stored as fp32 (cos, sin): entry (axis a, position p, column m) = p * base^(-m / n_axis[a]).
 __global__ void __launch_bounds__(256) k_rope_table(float2 *__restrict__ tab, pc_rope_dev rope, double base, int total) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= total) return;
     const int a = e >= rope.off[2] ? 2 : (e >= rope.off[1] ? 1 : 0);
@@ -590,7 +600,7 @@ pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const
     rope.tab = tab;
     // the array keeps whatever the last call left; the table, the partials and the pooled query are all rewritten before
     // they are read, and nothing has to start at zero
-    k_rope_table<<<(total + 255) / 256, 256, 0, stream>>>(tab, rope, D.rope_base, total);
+    PC_LAUNCH(k_rope_table, dim3((total + 255) / 256), dim3(256), 0, stream, tab, rope, D.rope_base, total);
     PC_CUDA_TRY(cudaGetLastError());
 
     int sm_count = 0, dev = 0;
