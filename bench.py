@@ -46,6 +46,29 @@ def _peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+# --------------------------------------------------------------------------------------------- ranks
+def rank_layer_ids(rank: int, n_layers: int):
+    """Layers a rank draws: disjoint seeded layers per rank (weak scaling by replication, nothing exchanged on the data
+    path)."""
+    return [rank * n_layers + i for i in range(n_layers)]
+
+
+def max_over_ranks(value: float, dist, device="cpu") -> float:
+    """The slowest rank's time: a job of N replicas takes as long as its slowest member."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_ms_per_frame(ms_step_max: float, world: int) -> float:
+    """Whole-job latency per frame: every rank finishes one frame per step, so the job finishes `world` frames in the time
+    of the slowest rank's step."""
+    return ms_step_max / world
+
+
 # --------------------------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) while the timed regions run."""
@@ -187,7 +210,7 @@ def run_cuda(args):
     cfg = wl.CONFIGS[WORKLOAD]
     b = cfg.budget
     # every rank draws its own layers (weak scaling: independent layers, no exchange on the data path)
-    host_layers = [wl.make_layer(cfg, layer=rank * N_LAYERS + i) for i in range(N_LAYERS)]
+    host_layers = [wl.make_layer(cfg, layer=i) for i in rank_layer_ids(rank, N_LAYERS)]
     layers = [DeviceLayer(L) for L in host_layers]
     ctx = make_ctx(cfg)
     n_sel = b.total
@@ -226,10 +249,7 @@ def run_cuda(args):
     e1.record(stream)
     barrier()
     ms_total = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, "cuda")
     ms_step = ms_total / args.steps
     assert pc.pc_poll_status(ctx) == pc.PC_OK, "device-side error in the timed region"
 
@@ -279,10 +299,7 @@ def run_cuda(args):
     e1.record(stream)
     barrier()
     e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(n_e2e, 1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
     clocks = sampler.stop()
     status = pc.pc_poll_status(ctx)
     assert status == pc.PC_OK, f"device-side status {status}"
@@ -304,7 +321,7 @@ def run_cuda(args):
     hbm = lambda nbytes, ms: (nbytes / (ms * 1e-3) / 1e9) if ms else None
     stages = {k: (round(v, 5) if v is not None else None) for k, v in kern_ms.items()}
     line = {
-        "metric": METRIC, "value": ms_step / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": job_ms_per_frame(ms_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "n_frames": cfg.n_frames, "frame_tokens": cfg.frame_tokens,
@@ -313,7 +330,7 @@ def run_cuda(args):
                    "budget": "2 newest frames whole + 6048 at half-life 4", "mode": "one-shot compaction every frame",
                    "l2": f"inputs rotate over {N_LAYERS} layers (~{0.2 * N_LAYERS:.1f} GB; L2 is 126 MB)", "parallelism": f"replicas x{world}"},
         "clocks": clocks,
-        "e2e": {"value": (e2e_ms / world) if n_e2e else None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        "e2e": {"value": job_ms_per_frame(e2e_ms, world) if n_e2e else None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": n_e2e},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"kernel": "k_attend_tc", "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],

@@ -1,0 +1,70 @@
+"""The multi-rank path of the benchmark on CPU: two `gloo` ranks.  The path shards by replication (each rank its own
+seeded layers, no collective on the data path), so what has to hold is: ranks draw disjoint layers, the job time is the
+maximum over ranks, the job metric divides by the number of replicas, and under a two-rank launch of the reference arm
+only rank 0 works and prints."""
+from __future__ import annotations
+
+import json
+import os
+import socket
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+import bench  # noqa: E402
+
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank: int, world: int, port: int, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    mine = bench.rank_layer_ids(rank, 4)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, mine)
+    slowest = bench.max_over_ranks(10.0 + 5.0 * rank, dist)          # rank 1 is the slow one
+    dist.barrier()
+    out.put((rank, gathered, slowest))
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_layers_and_take_the_slowest_time():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, gathered, slowest in got:
+        assert gathered == [[0, 1, 2, 3], [4, 5, 6, 7]]                # disjoint, seeded per rank
+        assert slowest == 15.0                                         # every rank reports the maximum
+    assert bench.job_ms_per_frame(15.0, world) == 7.5                  # two replicas finish two frames per step
+    assert bench.max_over_ranks(3.0, None) == 3.0
+
+
+def test_reference_arm_under_two_ranks_prints_once():
+    env = dict(os.environ, WORLD_SIZE="2", OMP_NUM_THREADS="2")
+    outs = []
+    for rank in (0, 1):
+        env["RANK"] = env["LOCAL_RANK"] = str(rank)
+        r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                            "--warmup", "0"], env=env, capture_output=True, text=True, timeout=600)
+        assert r.returncode == 0, r.stderr[-500:]
+        outs.append(r.stdout.strip())
+    assert outs[1] == ""                                               # rank 1 exits without work
+    line = json.loads(outs[0].splitlines()[-1])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["cpu_baseline"]["kind"] == "oracle"
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
