@@ -216,6 +216,56 @@ pc_status pc_score_tokens_static(const pc_layer_desc *desc, const void *hist_k, 
                                  int32_t n_src, const void *q, const int32_t *q_pos, int32_t n_q,
                                  const uint8_t *valid, float *scores, int32_t *status, void *stream);
 
+/* ---- Cache window: the Fill / Pack / Slide regimes of Sec. 3.4 (Fig. 6) around the calls above.
+ *
+ * The window keeps at most `window` history frames (W of Eq. 3) in one of two caller-owned history buffers.
+ *   Fill : appended frames are kept whole while they fit the token budget (budget.total) and the window.
+ *   Pack : once they do not, every retained frame is cut to its quota (pc_plan_budget over the frames' current token
+ *          counts), keeping the tokens that score best against the current frame's queries, and the survivors are packed
+ *          into the other buffer, which becomes the active one.
+ *   Slide: a frame beyond the window is dropped first (first in, first out), the rest is re-packed under the same rule, and
+ *          with `rebase` set the temporal coordinate of every retained history token drops by t_step per dropped frame
+ *          (Eq. 9: only t moves; h, w and the tag are carried).  Anchors are never touched.  The caller builds the next
+ *          frames' positions in the shifted frame of reference: pc_window_state reports the accumulated shift.
+ * Re-selection is incremental: the source of a pack is what the last pack kept plus the frames appended since.
+ * All device memory is the caller's: the two history buffers (each must hold budget.total tokens plus the frames
+ * appended between two packs), a score buffer and an index buffer of the same token capacity. */
+typedef struct pc_window pc_window;
+
+typedef struct {
+    int32_t window;          /* W: most history frames kept */
+    pc_budget_params budget; /* decay kernel and token budget of the history (anchors not counted) */
+    int32_t rebase;          /* 1: apply the temporal rebase of Eq. 9 when frames are dropped */
+    int32_t t_step;          /* temporal coordinate units per frame (4 under MM-RoPE's scaling) */
+} pc_window_params;
+
+enum { PC_WINDOW_FILL = 0, PC_WINDOW_PACK = 1, PC_WINDOW_SLIDE = 2 };
+
+/* scores device [capacity] fp32 and sel_idx device [capacity] int32, capacity = the smaller history buffer's.
+ * Errors: PC_ERR_INVALID_ARG (null, window < 1, t_step < 0, empty buffers, misaligned). */
+pc_status pc_window_create(pc_ctx *ctx, const pc_window_params *params, const pc_segment *anchors,
+                           const pc_segment *hist_a, const pc_segment *hist_b, float *scores, int32_t *sel_idx,
+                           pc_window **out);
+pc_status pc_window_destroy(pc_window *w);
+
+/* Append a finished frame (device K, V, pos; positions already in the shifted frame of reference) as the newest
+ * history frame: device-to-device copies on the stream.  Errors: PC_ERR_CAPACITY (active buffer full). */
+pc_status pc_window_append(pc_window *w, const pc_segment *frame, void *stream);
+
+/* Bring the cache back inside window and budget for the frame whose queries are q (see the regimes above); regime
+ * (host out, may be NULL) receives PC_WINDOW_FILL / PACK / SLIDE.  scores_override: device fp32 scores of the source
+ * tokens (after dropped frames) to select on instead of scoring, or NULL.  Errors as pc_score / pc_compact. */
+pc_status pc_window_update(pc_window *w, const void *q, const int32_t *q_pos, int32_t n_q, const float *scores_override,
+                           int32_t *regime, void *stream);
+
+/* The current cache as a pc_cache for pc_attend_frame (frame_count points into the window: valid until the next
+ * append / update / destroy). */
+pc_status pc_window_cache(pc_window *w, pc_cache *out);
+
+/* Host-side state: frames kept, their token counts oldest -> newest (counts may be NULL, else room for window + 1),
+ * the accumulated temporal shift, and which buffer (0 = hist_a, 1 = hist_b) is active. */
+pc_status pc_window_state(pc_window *w, int32_t *n_frames, int32_t *counts, int64_t *t_shift, int32_t *active);
+
 /* Wait for the stream, then return and clear the first device-side event
  * recorded since the last poll (PC_OK if none). */
 pc_status pc_poll_status(pc_ctx *ctx, void *stream);

@@ -23,7 +23,9 @@ PC_MAX_FRAMES = 256
 
 EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact", "pc_attend_frame",
            "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_set_timing", "pc_get_timing",
-           "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge"]
+           "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge",
+           "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_update", "pc_window_cache",
+           "pc_window_state"]
 
 
 class pc_layer_desc(C.Structure):
@@ -44,6 +46,10 @@ class pc_cache(C.Structure):
 class pc_budget_params(C.Structure):
     _fields_ = [("kind", C.c_int32), ("param", C.c_double), ("total", C.c_int64), ("keep_full", C.c_int32),
                 ("min_quota", C.c_int32)]
+
+
+class pc_window_params(C.Structure):
+    _fields_ = [("window", C.c_int32), ("budget", pc_budget_params), ("rebase", C.c_int32), ("t_step", C.c_int32)]
 
 
 class pc_host_frame(C.Structure):
@@ -101,6 +107,14 @@ def load() -> C.CDLL:
                                        C.POINTER(pc_budget_params), C.c_int32, C.c_void_p]
     lib.pc_score_tokens_static.argtypes = [C.POINTER(pc_layer_desc), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                            C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.pc_window_create.argtypes = [C.c_void_p, C.POINTER(pc_window_params), C.POINTER(pc_segment), C.POINTER(pc_segment),
+                                     C.POINTER(pc_segment), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p)]
+    lib.pc_window_destroy.argtypes = [C.c_void_p]
+    lib.pc_window_append.argtypes = [C.c_void_p, C.POINTER(pc_segment), C.c_void_p]
+    lib.pc_window_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int32), C.c_void_p]
+    lib.pc_window_cache.argtypes = [C.c_void_p, C.POINTER(pc_cache)]
+    lib.pc_window_state.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int64),
+                                    C.POINTER(C.c_int32)]
     _lib = lib
     return lib
 
@@ -289,3 +303,60 @@ def pc_score_tokens_static(desc: pc_layer_desc, hist_k: torch.Tensor, hist_pos: 
                                          q.shape[0], _ptr(valid), _ptr(scores), _ptr(status), _stream(stream)),
            "pc_score_tokens_static")
     return scores
+
+
+PC_WINDOW_FILL, PC_WINDOW_PACK, PC_WINDOW_SLIDE = 0, 1, 2
+
+
+class Window:
+    """The Fill / Pack / Slide cache window over two caller-owned history buffers (Segments with capacity; their n_tokens
+    is managed by the library).  Argument marshalling only: plan, score, select, pack run in the library."""
+
+    def __init__(self, ctx: Context, window: int, kind: int, param: float, total: int, keep_full: int, anchors: Segment,
+                 hist_a: Segment, hist_b: Segment, rebase: bool = False, t_step: int = 4):
+        self.ctx, self.anchors, self.bufs = ctx, anchors, (hist_a, hist_b)
+        cap = min(hist_a.capacity, hist_b.capacity)
+        dev = hist_a.k.device
+        self.scores = torch.empty(cap, dtype=torch.float32, device=dev)
+        self.sel_idx = torch.empty(cap, dtype=torch.int32, device=dev)
+        self.window = window
+        p = pc_window_params(window, pc_budget_params(kind, param, total, keep_full, 0), 1 if rebase else 0, t_step)
+        a, ha, hb = anchors.c(), hist_a.c(), hist_b.c()
+        h = C.c_void_p()
+        _check(load().pc_window_create(ctx.handle, C.byref(p), C.byref(a), C.byref(ha), C.byref(hb), _ptr(self.scores),
+                                       _ptr(self.sel_idx), C.byref(h)), "pc_window_create")
+        self.handle = h
+
+    def append(self, frame: Segment, stream=None) -> None:
+        f = frame.c()
+        _check(load().pc_window_append(self.handle, C.byref(f), _stream(stream)), "pc_window_append")
+
+    def update(self, q: Optional[torch.Tensor], q_pos: Optional[torch.Tensor], scores_override: Optional[torch.Tensor] = None,
+               stream=None) -> int:
+        regime = C.c_int32(-1)
+        _check(load().pc_window_update(self.handle, _ptr(q), _ptr(q_pos), 0 if q is None else q.shape[0],
+                                       _ptr(scores_override), C.byref(regime), _stream(stream)), "pc_window_update")
+        return regime.value
+
+    def state(self):
+        """(token counts oldest -> newest, accumulated temporal shift, index of the active buffer)"""
+        n, shift, active = C.c_int32(), C.c_int64(), C.c_int32()
+        counts = (C.c_int32 * (self.window + 1))()
+        _check(load().pc_window_state(self.handle, C.byref(n), counts, C.byref(shift), C.byref(active)), "pc_window_state")
+        return np.array(counts[:n.value], dtype=np.int32), int(shift.value), int(active.value)
+
+    def cache(self) -> Cache:
+        counts, _, active = self.state()
+        b = self.bufs[active]
+        return Cache(self.anchors, Segment(b.k, b.v, b.pos, int(counts.sum())), counts)
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            load().pc_window_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

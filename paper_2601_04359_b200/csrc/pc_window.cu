@@ -1,0 +1,144 @@
+// Cache window: the Fill / Pack / Slide regimes (Sec. 3.4, Fig. 6) and the temporal rebase (Eq. 9) as a host-side state
+// machine around pc_plan_budget, pc_score and pc_compact.  No kernels of its own.
+#include <vector>
+
+#include "pc_common.cuh"
+
+struct pc_window {
+    pc_ctx *ctx;
+    pc_window_params p;
+    pc_segment anchors;
+    pc_segment buf[2];
+    int active;
+    std::vector<int32_t> count;      // tokens per retained frame, oldest -> newest
+    std::vector<int32_t> budget;     // scratch of the last plan
+    int64_t t_shift;
+    float *scores;
+    int32_t *sel_idx;
+    int32_t scratch_capacity;
+};
+
+extern "C" pc_status pc_window_create(pc_ctx *ctx, const pc_window_params *params, const pc_segment *anchors,
+                                      const pc_segment *hist_a, const pc_segment *hist_b, float *scores, int32_t *sel_idx,
+                                      pc_window **out) {
+    if (!ctx || !params || !anchors || !hist_a || !hist_b || !scores || !sel_idx || !out) return PC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (params->window < 1 || params->window >= PC_MAX_FRAMES || params->t_step < 0 || params->budget.total < 0)
+        return PC_ERR_INVALID_ARG;
+    if (!pc_aligned16(scores) || !pc_aligned16(sel_idx)) return PC_ERR_INVALID_ARG;
+    pc_status st = pc_check_segment(anchors, true);
+    if (st != PC_OK) return st;
+    const pc_segment *hb[2] = {hist_a, hist_b};
+    for (int i = 0; i < 2; ++i) {
+        if (hb[i]->capacity <= 0 || !hb[i]->k || !hb[i]->v || !hb[i]->pos) return PC_ERR_INVALID_ARG;
+        if (!pc_aligned16(hb[i]->k) || !pc_aligned16(hb[i]->v) || !pc_aligned16(hb[i]->pos)) return PC_ERR_INVALID_ARG;
+    }
+    pc_window *w = new (std::nothrow) pc_window();
+    if (!w) return PC_ERR_CUDA;
+    w->ctx = ctx;
+    w->p = *params;
+    w->anchors = *anchors;
+    w->buf[0] = *hist_a;
+    w->buf[1] = *hist_b;
+    w->buf[0].n_tokens = w->buf[1].n_tokens = 0;
+    w->active = 0;
+    w->t_shift = 0;
+    w->scores = scores;
+    w->sel_idx = sel_idx;
+    w->scratch_capacity = std::min(hist_a->capacity, hist_b->capacity);
+    *out = w;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_window_destroy(pc_window *w) {
+    if (!w) return PC_ERR_INVALID_ARG;
+    delete w;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_window_append(pc_window *w, const pc_segment *frame, void *stream_) {
+    if (!w || !frame) return PC_ERR_INVALID_ARG;
+    pc_status st = pc_check_segment(frame, false);
+    if (st != PC_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    pc_segment &A = w->buf[w->active];
+    const int n = frame->n_tokens;
+    if ((int64_t)A.n_tokens + n > A.capacity || (int64_t)A.n_tokens + n > w->scratch_capacity) return PC_ERR_CAPACITY;
+    if ((int)w->count.size() + 1 > PC_MAX_FRAMES) return PC_ERR_CAPACITY;
+    const size_t row = (size_t)w->ctx->desc.n_kv_heads * w->ctx->desc.head_dim * w->ctx->elem_size;
+    char *k = static_cast<char *>(A.k) + (size_t)A.n_tokens * row, *v = static_cast<char *>(A.v) + (size_t)A.n_tokens * row;
+    PC_CUDA_TRY(cudaMemcpyAsync(k, frame->k, (size_t)n * row, cudaMemcpyDeviceToDevice, stream));
+    PC_CUDA_TRY(cudaMemcpyAsync(v, frame->v, (size_t)n * row, cudaMemcpyDeviceToDevice, stream));
+    PC_CUDA_TRY(cudaMemcpyAsync(A.pos + 4 * (size_t)A.n_tokens, frame->pos, (size_t)n * 16, cudaMemcpyDeviceToDevice, stream));
+    A.n_tokens += n;
+    w->count.push_back(n);
+    return PC_OK;
+}
+
+extern "C" pc_status pc_window_update(pc_window *w, const void *q, const int32_t *q_pos, int32_t n_q,
+                                      const float *scores_override, int32_t *regime, void *stream) {
+    if (!w) return PC_ERR_INVALID_ARG;
+    const int n_frames = (int)w->count.size();
+    const int drop = std::max(0, n_frames - w->p.window);          // frames beyond the window leave first (FIFO)
+    int64_t dropped_tokens = 0, kept_tokens = 0;
+    for (int f = 0; f < n_frames; ++f) (f < drop ? dropped_tokens : kept_tokens) += w->count[f];
+    if (drop == 0 && kept_tokens <= w->p.budget.total) {           // Fill: everything still fits
+        if (regime) *regime = PC_WINDOW_FILL;
+        return PC_OK;
+    }
+    const int kept = n_frames - drop;
+    pc_segment &A = w->buf[w->active], &B = w->buf[w->active ^ 1];
+    const size_t row = (size_t)w->ctx->desc.n_kv_heads * w->ctx->desc.head_dim * w->ctx->elem_size;
+    // source: the active buffer past the dropped frames
+    pc_cache src;
+    src.anchors = w->anchors;
+    src.history.k = static_cast<char *>(A.k) + (size_t)dropped_tokens * row;
+    src.history.v = static_cast<char *>(A.v) + (size_t)dropped_tokens * row;
+    src.history.pos = A.pos + 4 * (size_t)dropped_tokens;
+    src.history.n_tokens = (int32_t)kept_tokens;
+    src.history.capacity = (int32_t)(A.capacity - dropped_tokens);
+    src.n_frames = kept;
+    src.frame_count = w->count.data() + drop;
+    w->budget.assign((size_t)std::max(kept, 1), 0);
+    pc_status st = pc_plan_budget(&w->p.budget, kept, src.frame_count, w->budget.data());
+    if (st != PC_OK) return st;
+    int64_t n_sel = 0;
+    for (int f = 0; f < kept; ++f) n_sel += w->budget[f];
+    if (n_sel > B.capacity) return PC_ERR_CAPACITY;
+    st = pc_score(w->ctx, &src, q, q_pos, n_q, w->budget.data(), nullptr, scores_override, w->scores, w->sel_idx, stream);
+    if (st != PC_OK) return st;
+    pc_cache dst;
+    dst.anchors = w->anchors;
+    dst.history = B;
+    dst.n_frames = kept;
+    dst.frame_count = w->budget.data();
+    const int32_t delta_t = w->p.rebase ? drop * w->p.t_step : 0;  // Eq. 9: t falls by the number of dropped frames
+    st = pc_compact(w->ctx, &src, w->sel_idx, w->budget.data(), delta_t, &dst, stream);
+    if (st != PC_OK) return st;
+    B.n_tokens = (int32_t)n_sel;
+    A.n_tokens = 0;
+    w->active ^= 1;
+    w->count.assign(w->budget.begin(), w->budget.begin() + kept);
+    w->t_shift += delta_t;
+    if (regime) *regime = drop ? PC_WINDOW_SLIDE : PC_WINDOW_PACK;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_window_cache(pc_window *w, pc_cache *out) {
+    if (!w || !out) return PC_ERR_INVALID_ARG;
+    out->anchors = w->anchors;
+    out->history = w->buf[w->active];
+    out->n_frames = (int32_t)w->count.size();
+    out->frame_count = w->count.data();
+    return PC_OK;
+}
+
+extern "C" pc_status pc_window_state(pc_window *w, int32_t *n_frames, int32_t *counts, int64_t *t_shift, int32_t *active) {
+    if (!w) return PC_ERR_INVALID_ARG;
+    if (n_frames) *n_frames = (int32_t)w->count.size();
+    if (counts)
+        for (size_t f = 0; f < w->count.size(); ++f) counts[f] = w->count[f];
+    if (t_shift) *t_shift = w->t_shift;
+    if (active) *active = w->active;
+    return PC_OK;
+}

@@ -1,0 +1,184 @@
+"""The cache window (Fill / Pack / Slide, Sec. 3.4 and Fig. 6; rebase, Eq. 9).
+
+CPU part: the reference state machine in oracle/window.py against what the paper fixes — the allocation pattern printed
+after Eq. 7 row by row as the window fills, first-in-first-out eviction, the rebase moving t only — and against
+structural invariants.  GPU part: the library's window against the reference, frame by frame, bit for bit on counts,
+packed rows and positions when both select on the same fp32 scores, and attention over the window's cache against the
+oracle's attention over the reference's cache."""
+from __future__ import annotations
+
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import window as ow
+from paper_2601_04359_b200 import workload as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "allocation_pattern.txt")
+
+
+def _frames(cfg, n_frames, seed=0):
+    """K, V, positions of frames 1..n_frames and the queries of each following frame (tags = global token ids)."""
+    rng = np.random.Generator(np.random.Philox(key=[seed, 77]))
+    n, hkv, hq, d = cfg.frame_tokens, cfg.n_kv_heads, cfg.n_q_heads, cfg.head_dim
+    st = lambda x: wl.to_storage(x.astype(np.float32), cfg.dtype)
+    out = []
+    for f in range(1, n_frames + 2):
+        pos = wl.frame_positions(cfg, f, cfg.n_anchor + (f - 1) * n)
+        out.append(dict(k=st(rng.standard_normal((n, hkv, d))), v=st(rng.standard_normal((n, hkv, d))), pos=pos,
+                        q=st(rng.standard_normal((n, hq, d)))))
+    return out
+
+
+def _printed_pattern():
+    rows = {}
+    for line in open(GOLDEN):
+        if line.strip() and not line.startswith("#"):
+            w, vals = line.split(":")
+            rows[int(w)] = [Fraction(x) for x in vals.split()]
+    return rows
+
+
+def test_window_fills_by_the_printed_allocation_pattern():
+    """With a budget of one frame (B_one = N) and the closed-form decay, the cache after 1, 2, 3, 4 frames holds
+    N x [1], [1/2, 1/2], [1/2, 1/4, 1/4], [1/2, 1/4, 1/8, 1/8] tokens, newest first: the pattern printed after Eq. 7."""
+    cfg = wl.CONFIGS["tiny"]
+    n = cfg.frame_tokens
+    fr = _frames(cfg, 6)
+    ref = ow.WindowRef(4, oracle.CLOSED_HALF, 0.5, n, 0)
+    rows = _printed_pattern()
+    for f in range(4):
+        ref.append(fr[f]["k"], fr[f]["v"], fr[f]["pos"])
+        regime = ref.update(fr[f + 1]["q"], fr[f + 1]["pos"])
+        assert regime == (ow.FILL if f == 0 else ow.PACK)
+        assert ref.count[::-1] == [int(n * b) for b in rows[f + 1]]
+        assert sum(ref.count) == n
+    # sliding: the window stays at four frames under the W = 4 row, the oldest frame leaves
+    for f in range(4, 6):
+        ref.append(fr[f]["k"], fr[f]["v"], fr[f]["pos"])
+        assert ref.update(fr[f + 1]["q"], fr[f + 1]["pos"]) == ow.SLIDE
+        assert ref.count[::-1] == [int(n * b) for b in rows[4]]
+        frames_present = sorted(set(((ref.pos[:, 3] - cfg.n_anchor) // n).tolist()))
+        assert frames_present == list(range(f - 3, f + 1))                 # tags prove which frames survive (FIFO)
+
+
+def test_window_rebase_moves_t_only_and_kept_sets_shrink():
+    cfg = wl.CONFIGS["tiny"]
+    n = cfg.frame_tokens
+    fr = _frames(cfg, 7, seed=3)
+    plain = ow.WindowRef(3, oracle.HALFLIFE, 1.0, 96, 1)
+    moved = ow.WindowRef(3, oracle.HALFLIFE, 1.0, 96, 1, rebase=True, t_step=4)
+    kept_before = {}
+    for f in range(7):
+        for w in (plain, moved):
+            pos = fr[f]["pos"].copy()
+            pos[:, 0] -= w.t_shift                                          # the caller builds positions in the shifted frame
+            qpos = fr[f + 1]["pos"].copy()
+            qpos[:, 0] -= w.t_shift
+            w.append(fr[f]["k"], fr[f]["v"], pos)
+            w.update(fr[f + 1]["q"], qpos)
+        assert plain.count == moved.count and moved.t_shift == 4 * max(0, f + 1 - 3)
+        # same tokens either way (rotary logits depend on position differences only), t lower by the shift, h / w / tag equal
+        assert np.array_equal(plain.pos[:, 1:], moved.pos[:, 1:])
+        assert np.array_equal(plain.pos[:, 0] - moved.t_shift, moved.pos[:, 0])
+        assert np.array_equal(plain.k, moved.k)
+        # a frame's kept tokens only ever shrink: re-selection is from what the last pack kept
+        tags = set(plain.pos[:, 3].tolist())
+        for g, old in kept_before.items():
+            now = {t for t in tags if (t - cfg.n_anchor) // n == g}
+            assert now <= old
+        kept_before = {g: {t for t in tags if (t - cfg.n_anchor) // n == g} for g in range(f + 1)}
+        assert sum(plain.count) <= 96 and len(plain.count) <= 3
+
+
+# ------------------------------------------------------------------------------------------------ GPU
+@pytest.mark.gpu
+@pytest.mark.parametrize("rebase", [False, True])
+def test_window_matches_reference_frame_by_frame(rebase):
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200.device import dev, host, idev, make_ctx, segment
+
+    cfg = wl.small_bf16(n_frames=8, grid=(9, 15), n_text=37, total=300, kind=wl.HALFLIFE, param=2.0, keep_full=1, seed=9)
+    n, W, total = cfg.frame_tokens, 5, 300
+    L = wl.make_layer(cfg)                                                  # anchors only
+    fr = _frames(cfg, 8, seed=5)
+    ctx = make_ctx(cfg, max_keys=cfg.n_anchor + total + 3 * n)
+    cap = total + 2 * n
+    td = torch.bfloat16
+    mk = lambda: pc.Segment(torch.full((cap, cfg.n_kv_heads, cfg.head_dim), 7.0, dtype=td, device="cuda"),
+                            torch.full((cap, cfg.n_kv_heads, cfg.head_dim), 7.0, dtype=td, device="cuda"),
+                            torch.full((cap, 4), -9, dtype=torch.int32, device="cuda"), 0)
+    anchors = segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype)
+    win = pc.Window(ctx, W, pc.PC_HALFLIFE, 2.0, total, 1, anchors, mk(), mk(), rebase=rebase, t_step=4)
+    ref = ow.WindowRef(W, oracle.HALFLIFE, 2.0, total, 1, rebase=rebase, t_step=4)
+    regimes = []
+    for f in range(8):
+        pos = fr[f]["pos"].copy(); pos[:, 0] -= ref.t_shift
+        qpos = fr[f + 1]["pos"].copy(); qpos[:, 0] -= ref.t_shift
+        ref.append(fr[f]["k"], fr[f]["v"], pos)
+        win.append(segment(fr[f]["k"], fr[f]["v"], pos, cfg.dtype))
+        # both sides select on the same fp32 scores (the oracle's); the GPU's own scores are checked separately below
+        sk, _, spos, scounts, _ = ref.source_after_drop()
+        s32 = oracle.score_pooled(sk, spos, fr[f + 1]["q"], qpos, cfg.rope_base).astype(np.float32)
+        want_regime = ref.update(fr[f + 1]["q"], qpos, scores32=s32)
+        got_regime = win.update(dev(fr[f + 1]["q"], cfg.dtype), idev(qpos), scores_override=torch.from_numpy(s32).cuda())
+        assert got_regime == want_regime
+        regimes.append(got_regime)
+        counts, shift, _ = win.state()
+        assert counts.tolist() == ref.count and shift == ref.t_shift
+        cache = win.cache()
+        m = int(counts.sum())
+        assert np.array_equal(host(cache.history.k)[:m], ref.k) and np.array_equal(host(cache.history.v)[:m], ref.v)
+        assert np.array_equal(cache.history.pos.cpu().numpy()[:m], ref.pos)
+        # attention of the next frame's queries over the window's cache
+        out = pc.pc_attend_frame(ctx, cache, None, dev(fr[f + 1]["q"], cfg.dtype), idev(qpos))
+        assert pc.pc_poll_status(ctx) == pc.PC_OK
+        want = oracle.attend(fr[f + 1]["q"], qpos, [(L.anchor_k, L.anchor_v, L.anchor_pos), (ref.k, ref.v, ref.pos)], cfg.rope_base)
+        assert np.abs(host(out).astype(np.float64) - want).max() <= 2e-2
+    assert regimes[0] == pc.PC_WINDOW_FILL and pc.PC_WINDOW_PACK in regimes and regimes[-1] == pc.PC_WINDOW_SLIDE
+    win.close(); ctx.close()
+
+
+@pytest.mark.gpu
+def test_window_on_its_own_scores_keeps_valid_state():
+    """Without an override the window scores on the GPU: counts follow the plan, every kept token is a token of the
+    frame it is filed under, and each frame's kept set only shrinks."""
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200.device import dev, idev, make_ctx, segment
+
+    cfg = wl.small_bf16(n_frames=8, grid=(9, 15), n_text=37, total=300, kind=wl.LINEAR, param=0.0, keep_full=0, seed=2)
+    n, W, total = cfg.frame_tokens, 4, 260
+    L = wl.make_layer(cfg)
+    fr = _frames(cfg, 7, seed=8)
+    ctx = make_ctx(cfg, max_keys=cfg.n_anchor + total + 3 * n)
+    cap = total + 2 * n
+    mk = lambda: pc.Segment(torch.zeros((cap, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((cap, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((cap, 4), dtype=torch.int32, device="cuda"), 0)
+    win = pc.Window(ctx, W, pc.PC_LINEAR, 0.0, total, 0, segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype), mk(), mk())
+    kept = {}
+    counts_before = []
+    for f in range(7):
+        win.append(segment(fr[f]["k"], fr[f]["v"], fr[f]["pos"], cfg.dtype))
+        regime = win.update(dev(fr[f + 1]["q"], cfg.dtype), idev(fr[f + 1]["pos"]))
+        assert pc.pc_poll_status(ctx) == pc.PC_OK
+        counts, shift, _ = win.state()
+        avail = (counts_before + [n])[-W:] if regime != pc.PC_WINDOW_FILL else None
+        if avail is not None:
+            assert counts.tolist() == oracle.plan_budget(oracle.LINEAR, 0.0, total, 0, avail).tolist()
+        tags = win.cache().history.pos.cpu().numpy()[:int(counts.sum()), 3]
+        frames_of = (tags - cfg.n_anchor) // n
+        first = f + 1 - len(counts)
+        want_frames = np.repeat(np.arange(first, first + len(counts)), counts)
+        assert np.array_equal(frames_of, want_frames) and len(set(tags.tolist())) == len(tags)
+        now = {g: set(tags[frames_of == g].tolist()) for g in range(first, f + 1)}
+        for g, s in now.items():
+            assert g not in kept or s <= kept[g]
+        kept = now
+        counts_before = counts.tolist()
+    win.close(); ctx.close()
