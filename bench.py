@@ -264,6 +264,45 @@ def run_cuda(args):
     pc.pc_set_timing(ctx, False)
     kern_ms = {k: (float(np.mean(v)) if v else None) for k, v in acc.items()}
 
+    # ---- the same frame step in the Slide regime of the cache window (incremental re-selection: the source of each pack is
+    # what the last pack kept plus the newest frame, about 9 k tokens instead of the whole 47-frame history)
+    N = cfg.frame_tokens
+    cap = n_sel + 2 * N
+    mkbuf = lambda: pc.Segment(torch.empty((cap, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                               torch.empty((cap, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                               torch.empty((cap, 4), dtype=torch.int32, device="cuda"), 0)
+    win = pc.Window(ctx, cfg.n_frames, b.kind, b.param, b.total, b.keep_full, layers[0].cache.anchors, mkbuf(), mkbuf())
+
+    def frame_of(i):
+        D = layers[i % N_LAYERS]
+        f = i % cfg.n_frames
+        h = D.cache.history
+        return D, pc.Segment(h.k[f * N:(f + 1) * N], h.v[f * N:(f + 1) * N], h.pos[f * N:(f + 1) * N], N)
+
+    def inc_step(i):
+        D, fr = frame_of(i)
+        win.append(fr, stream=stream)
+        regime = win.update(D.q, D.q_pos, stream=stream)
+        pc.pc_attend_frame(ctx, win.cache(), None, D.q, D.q_pos, out=out, stream=stream)
+        return regime
+
+    inc_ms, inc_src = None, None
+    if not args.no_incremental:
+        for i in range(cfg.n_frames + 3):                       # fill the window, then a few sliding steps
+            regime = inc_step(i)
+        barrier()
+        assert regime == pc.PC_WINDOW_SLIDE and pc.pc_poll_status(ctx) == pc.PC_OK
+        inc_src = int(win.state()[0].sum()) + N
+        n_inc = min(args.steps, 200)
+        e0.record(stream)
+        for i in range(n_inc):
+            inc_step(cfg.n_frames + 3 + i)
+        e1.record(stream)
+        barrier()
+        inc_ms = max_over_ranks(e0.elapsed_time(e1) / n_inc, dist, "cuda")
+        assert pc.pc_poll_status(ctx) == pc.PC_OK
+    win.close()
+
     # ---- end to end from pinned host memory through the host-buffer entry point
     L0 = host_layers[0]
     td = torch.bfloat16
@@ -338,6 +377,9 @@ def run_cuda(args):
                      "peak_source": f"{peaks['source']} (burst; sustained {peaks['bf16_tflops_sustained']})",
                      "flops_per_launch": flops, "ms_per_launch": att_ms},
         "kernels_ms": stages,
+        "incremental": {"ms_per_frame": job_ms_per_frame(inc_ms, world) if inc_ms else None, "source_tokens": inc_src,
+                        "mode": "cache window in the Slide regime: append the newest frame, drop the oldest, re-plan, "
+                                "score and re-select from packed + new, pack, attend (same keys attended)"},
         "hbm_kernels": {
             "score": {"GBps": hbm(score_bytes, kern_ms["score"]), "bytes": score_bytes,
                       "frac": (hbm(score_bytes, kern_ms["score"]) or 0) / peaks["hbm_gbs"]},
@@ -364,6 +406,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--no-incremental", action="store_true", help="skip the cache-window leg (profiler captures)")
     ap.add_argument("--layers", type=int, default=N_LAYERS, help="rotated input sets (default 4, > L2)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
