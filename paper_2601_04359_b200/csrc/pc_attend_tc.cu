@@ -54,7 +54,7 @@ struct TcParams {
     int seg_n[PC_MAX_SEGMENTS];
     __nv_bfloat16 *out;
     float *lse;
-    float *part_o;    // [item*S + s][2][128][128]
+    float *part_o;    // [item*S + s][2] tiles of 128 x 128 fp32, 16-byte unit (c4, r) at c4*128 + r
     float *part_ml;   // [item*S + s][2][128][2]
     int32_t *status;
 };
@@ -573,17 +573,19 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 }
                 *reinterpret_cast<float2 *>(gen + SM_ML + (t * TILE + r) * 8) = make_float2(m_used, l);
             } else {
-                const size_t slot = ((size_t)blockIdx.x * 2 + t) * TILE + r;
-                float *prow = P.part_o + slot * TILE;
+                // Partial tile layout: 16-byte unit (c4, r) = columns 4*c4..4*c4+3 of row r at unit c4*128 + r, so the 32 rows
+                // of a warp store 512 contiguous bytes per instruction (a row-major tile would touch 32 lines per store).
+                const size_t tile_slot = (size_t)blockIdx.x * 2 + t;
+                uint4 *ptile = reinterpret_cast<uint4 *>(P.part_o) + tile_slot * (TILE * TILE / 4) + r;
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
                     tmem_ld32(o_addr + c * 32, v);
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        *reinterpret_cast<uint4 *>(prow + c * 32 + i * 4) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        ptile[(c * 8 + i) * TILE] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                 }
-                *reinterpret_cast<float2 *>(P.part_ml + slot * 2) = make_float2(m_used, l);
+                *reinterpret_cast<float2 *>(P.part_ml + (tile_slot * TILE + r) * 2) = make_float2(m_used, l);
             }
         }
     }
@@ -643,42 +645,60 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
 }
 
 // ------------------------------------------------------------------------------------------------ combine
-// One warp per (query row, head): merges the KV ranges' partials in range order.  Every load is issued before any is used.
+// Merge of the KV ranges' partials.  One block per (query tile of one head, 32-row quadrant); its eight warps take four
+// 16-byte column units each, lanes are consecutive rows, so every load of the partial tiles is a 512-byte run.  Every
+// load of a thread is issued before any is used.
 __global__ void __launch_bounds__(256) k_combine(const TcParams P) {
     pc_grid_dep_launch();
     pc_grid_dep_wait();
-    const int lane = threadIdx.x & 31;
-    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (w >= P.n_q * P.n_q_heads) return;
-    const int row = w / P.n_q_heads, h = w % P.n_q_heads;
-    const int g = h / P.group, T = (row / TILE) * P.group + h % P.group;
-    const int item = g * P.pairs_per_g + T / 2, t = T & 1, r = row % TILE;
+    const int lane = threadIdx.x & 31, cg = threadIdx.x >> 5;                   // cg: units 4*cg .. 4*cg+3
+    const int quad = blockIdx.x & 3, tile = blockIdx.x >> 2;
+    const int h = tile % P.n_q_heads, tb = tile / P.n_q_heads;
+    const int g = h / P.group, T = tb * P.group + h % P.group;
+    const int item = g * P.pairs_per_g + (T >> 1), t = T & 1;
+    const int r = quad * 32 + lane, row = tb * TILE + r;
+    if (row >= P.n_q) return;
     float2 ml[MAX_SPLITS];
-    float4 o[MAX_SPLITS];
+    float4 o[MAX_SPLITS][4];
 #pragma unroll
     for (int s = 0; s < MAX_SPLITS; ++s)
         if (s < P.n_splits) {
-            const size_t slot = ((size_t)(item * P.n_splits + s) * 2 + t) * TILE + r;
-            ml[s] = __ldcg(reinterpret_cast<const float2 *>(P.part_ml + slot * 2));
-            o[s] = __ldcg(reinterpret_cast<const float4 *>(P.part_o + slot * TILE) + lane);
+            const size_t tile_slot = ((size_t)item * P.n_splits + s) * 2 + t;
+            ml[s] = __ldcg(reinterpret_cast<const float2 *>(P.part_ml) + tile_slot * TILE + r);
+            const float4 *pt = reinterpret_cast<const float4 *>(P.part_o) + tile_slot * (TILE * TILE / 4) + r;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) o[s][u] = __ldcg(pt + (cg * 4 + u) * TILE);
         }
     float m = -INFINITY;
 #pragma unroll
     for (int s = 0; s < MAX_SPLITS; ++s)
         if (s < P.n_splits) m = fmaxf(m, ml[s].x);
     float l = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int s = 0; s < MAX_SPLITS; ++s)
         if (s < P.n_splits) {
             const float sc = exp2f(ml[s].x - m);
             l = fmaf(ml[s].y, sc, l);
-            acc.x = fmaf(o[s].x, sc, acc.x); acc.y = fmaf(o[s].y, sc, acc.y); acc.z = fmaf(o[s].z, sc, acc.z); acc.w = fmaf(o[s].w, sc, acc.w);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                acc[u].x = fmaf(o[s][u].x, sc, acc[u].x); acc[u].y = fmaf(o[s][u].y, sc, acc[u].y);
+                acc[u].z = fmaf(o[s][u].z, sc, acc[u].z); acc[u].w = fmaf(o[s][u].w, sc, acc[u].w);
+            }
         }
     const float inv = 1.f / l;
-    uint2 out = make_uint2(pc_pack_bf16(acc.x * inv, acc.y * inv), pc_pack_bf16(acc.z * inv, acc.w * inv));
-    *reinterpret_cast<uint2 *>(P.out + ((size_t)row * P.n_q_heads + h) * TILE + lane * 4) = out;
-    if (P.lse && lane == 0) P.lse[(size_t)row * P.n_q_heads + h] = (m + log2f(l)) * 0.6931471805599453f;
+    // this thread's 16 columns of its row: 32 contiguous bytes
+    uint4 w0, w1;
+    w0.x = pc_pack_bf16(acc[0].x * inv, acc[0].y * inv); w0.y = pc_pack_bf16(acc[0].z * inv, acc[0].w * inv);
+    w0.z = pc_pack_bf16(acc[1].x * inv, acc[1].y * inv); w0.w = pc_pack_bf16(acc[1].z * inv, acc[1].w * inv);
+    w1.x = pc_pack_bf16(acc[2].x * inv, acc[2].y * inv); w1.y = pc_pack_bf16(acc[2].z * inv, acc[2].w * inv);
+    w1.z = pc_pack_bf16(acc[3].x * inv, acc[3].y * inv); w1.w = pc_pack_bf16(acc[3].z * inv, acc[3].w * inv);
+    uint4 *orow = reinterpret_cast<uint4 *>(P.out + ((size_t)row * P.n_q_heads + h) * TILE + cg * 16);
+    orow[0] = w0;
+    orow[1] = w1;
+    if (P.lse && cg == 0) P.lse[(size_t)row * P.n_q_heads + h] = (m + log2f(l)) * 0.6931471805599453f;
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -826,7 +846,7 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     PC_CUDA_TRY(cudaGetLastError());
     pc_mark(ctx, PC_MARK_ATTEND, stream);
     if (P.n_splits > 1 && !P.cluster) {
-        PC_LAUNCH(k_combine, dim3(div_up(n_q * D.n_q_heads, 8)), dim3(256), 0, stream, P);
+        PC_LAUNCH(k_combine, dim3(P.n_tb * D.n_q_heads * 4), dim3(256), 0, stream, P);
         PC_CUDA_TRY(cudaGetLastError());
         pc_mark(ctx, PC_MARK_COMBINE, stream);
     }
