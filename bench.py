@@ -34,7 +34,7 @@ N_LAYERS = 4          # rotated input sets; 4 x ~0.2 GB > L2 (--layers changes i
 KERNELS_PER_STEP = 8  # k_qpool, k_qpool_reduce, k_score, k_select, k_pack, k_rope_rows, k_attend_tc, k_combine
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_attend_tc launch at this workload, from the ncu capture
 # summarised in profiles/ncu_kernels_lumos47_small_case.md (same launch shape); None when the kernel has changed since
-ATTEND_DRAM_TRAFFIC = 43_997_696 + 2_566_656
+ATTEND_DRAM_TRAFFIC = 43_983_616 + 3_283_968
 
 
 def _peaks():
