@@ -115,23 +115,28 @@ __global__ void __launch_bounds__(QPOOL_THREADS) k_qpool(const T *__restrict__ q
     }
 }
 
-// pooled[e] = (1/n_q) * sum over blocks of partial[b][e].  32 columns per block; eight threads per column each add
-// every eighth partial (in block order), and the eight sums are added in slice order.
-__global__ void __launch_bounds__(256) k_qpool_reduce(const float *__restrict__ partial, int n_partials, int row_len, float inv_n,
-                                                      float *__restrict__ pooled) {
+// pooled[e] = (1/n_q) * sum over blocks of partial[b][e].  32 columns per block; 32 threads per column each add every
+// 32nd partial (in block order, at most four loads, all in flight together), and the 32 sums are added in slice order.
+__global__ void __launch_bounds__(1024) k_qpool_reduce(const float *__restrict__ partial, int n_partials, int row_len, float inv_n,
+                                                       float *__restrict__ pooled) {
     pc_grid_dep_launch();
     pc_grid_dep_wait();
-    __shared__ float part[8][32];
+    __shared__ float part[32][33];
     const int c = threadIdx.x & 31, sl = threadIdx.x >> 5, e = blockIdx.x * 32 + c;
-    float acc = 0.f;
-    if (e < row_len)
-        for (int b = sl; b < n_partials; b += 8) acc += __ldcg(partial + (size_t)b * row_len + e);
-    part[sl][c] = acc;
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    if (e < row_len) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int b = sl + 32 * i;
+            if (b < n_partials) v[i] = __ldcg(partial + (size_t)b * row_len + e);
+        }
+    }
+    part[sl][c] = (v[0] + v[1]) + (v[2] + v[3]);
     __syncthreads();
     if (sl == 0 && e < row_len) {
         float tot = 0.f;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) tot += part[k][c];
+        for (int k = 0; k < 32; ++k) tot += part[k][c];
         pooled[e] = tot * inv_n;
     }
 }
@@ -434,7 +439,7 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
     }
 #undef PC_QPOOL_ARGS
     PC_CUDA_TRY(cudaGetLastError());
-    PC_LAUNCH(k_qpool_reduce, dim3((row + 31) / 32), dim3(256), 0, stream, partial, pool_blocks, row, 1.f / (float)n_q, pooled);
+    PC_LAUNCH(k_qpool_reduce, dim3((row + 31) / 32), dim3(1024), 0, stream, partial, pool_blocks, row, 1.f / (float)n_q, pooled);
     PC_CUDA_TRY(cudaGetLastError());
     if (marks) pc_mark(marks, PC_MARK_QPOOL, stream);
     const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
