@@ -97,7 +97,7 @@ typedef struct {
     double param;      /* rho or half-life, see the enum */
     int64_t total;     /* history tokens to retain in all, anchors not counted (B_one of Eq. 8) */
     int32_t keep_full; /* most recent frames kept whole (counted inside total) */
-    int32_t min_quota; /* reserved (minimum per-frame quota b_min); must be 0 */
+    int32_t min_quota; /* b_min of Sec. 3.4 in tokens: every frame that takes part keeps at least this many; 0 = none */
 } pc_budget_params;
 
 /* Create / destroy a context on the current CUDA device.  Builds the rotary
@@ -112,9 +112,11 @@ pc_status pc_destroy(pc_ctx *ctx);
  * weights to 2^-32: the keep_full newest frames keep everything; the rest of
  * `total` is shared in proportion to g(dist) by largest remainder (ties to the
  * nearer frame); a frame granted more than avail keeps avail and the surplus is
- * re-shared.  avail and budget are host arrays [n_frames], oldest -> newest.
- * The result sums to min(total, sum(avail)).
- * Errors: PC_ERR_INVALID_ARG (null, negative, bad param, min_quota != 0),
+ * re-shared.  With min_quota > 0 every frame that takes part is first guaranteed min(min_quota, avail) tokens and the
+ * decay kernel shares out the rest on top; if the guarantees of all frames exceed the budget, the oldest frames leave
+ * the window first (first in, first out) and get nothing.  avail and budget are host arrays [n_frames], oldest -> newest.
+ * The result sums to min(total, sum(avail)) (over the frames that take part).
+ * Errors: PC_ERR_INVALID_ARG (null, negative, bad param),
  * PC_ERR_BUDGET (kept-whole frames exceed total). */
 pc_status pc_plan_budget(const pc_budget_params *params, int32_t n_frames, const int32_t *avail,
                          int32_t *budget);

@@ -81,11 +81,11 @@ def rope(x: np.ndarray, pos: Sequence[int], base: float = 10000.0) -> np.ndarray
     return out
 
 
-def plan_budget(kind: int, param: float, total: int, keep_full: int, avail: Sequence[int]) -> np.ndarray:
+def plan_budget(kind: int, param: float, total: int, keep_full: int, avail: Sequence[int], min_quota: int = 0) -> np.ndarray:
     avail = _i32(avail)
     out = np.zeros(len(avail), dtype=np.int32)
-    _check(lib().po_plan_budget(C.c_int(kind), C.c_double(param), C.c_int64(total), C.c_int(keep_full),
-                                C.c_int(len(avail)), _p(avail, C.c_int32), _p(out, C.c_int32)))
+    _check(lib().po_plan_budget_min(C.c_int(kind), C.c_double(param), C.c_int64(total), C.c_int(keep_full),
+                                    C.c_int(min_quota), C.c_int(len(avail)), _p(avail, C.c_int32), _p(out, C.c_int32)))
     return out
 
 

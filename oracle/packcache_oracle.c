@@ -108,9 +108,9 @@ static double *rope_all(const float *x, const int32_t *pos, int64_t n, int heads
  * ------------------------------------------------------------------------ */
 typedef unsigned __int128 u128;
 
-int po_plan_budget(int kind, double param, int64_t total, int keep_full, int n_frames,
-                   const int32_t *avail, int32_t *budget) {
-    if (n_frames < 0 || total < 0 || keep_full < 0) return PO_ERR_ARG;
+int po_plan_budget_min(int kind, double param, int64_t total, int keep_full, int min_quota, int n_frames,
+                       const int32_t *avail_in, int32_t *budget) {
+    if (n_frames < 0 || total < 0 || keep_full < 0 || min_quota < 0) return PO_ERR_ARG;
     if (kind == PO_GEOMETRIC && !(param > 0.0 && param < 1.0)) return PO_ERR_ARG;
     if (kind == PO_HALFLIFE && !(param > 0.0)) return PO_ERR_ARG;
     if (kind < 0 || kind > 3) return PO_ERR_ARG;
@@ -118,11 +118,14 @@ int po_plan_budget(int kind, double param, int64_t total, int keep_full, int n_f
     if (W == 0) return PO_OK;
     uint64_t *w = (uint64_t *)calloc((size_t)W, sizeof(uint64_t));
     char *active = (char *)calloc((size_t)W, 1);
-    if (!w || !active) { free(w); free(active); return PO_ERR_ARG; }
+    int32_t *avail = (int32_t *)calloc((size_t)W, sizeof(int32_t));   /* room left in a frame above its guaranteed part */
+    int32_t *floor_q = (int32_t *)calloc((size_t)W, sizeof(int32_t)); /* guaranteed part (minimum quota) */
+    if (!w || !active || !avail || !floor_q) { free(w); free(active); free(avail); free(floor_q); return PO_ERR_ARG; }
     int64_t B = total;
     for (int f = 0; f < W; ++f) {
         int dist = W - f;
-        if (avail[f] < 0) { free(w); free(active); return PO_ERR_ARG; }
+        if (avail_in[f] < 0) { free(w); free(active); free(avail); free(floor_q); return PO_ERR_ARG; }
+        avail[f] = avail_in[f];
         budget[f] = 0;
         if (dist <= keep_full) {
             budget[f] = avail[f];
@@ -139,7 +142,22 @@ int po_plan_budget(int kind, double param, int64_t total, int keep_full, int n_f
         w[f] = (uint64_t)floor(g * 4294967296.0 + 0.5);
         active[f] = 1;
     }
-    if (B < 0) { free(w); free(active); return PO_ERR_BUDGET; }
+    if (B < 0) { free(w); free(active); free(avail); free(floor_q); return PO_ERR_BUDGET; }
+    /* Minimum quota b_min (Sec. 3.4): a frame that takes part is guaranteed min_quota tokens (or all it holds, if
+     * fewer).  When the guarantees of all frames would exceed the budget, the window shrinks first in, first out: only
+     * the nearest floor(B / min_quota) frames take part, the farther ones get nothing.  The guarantees are set aside
+     * and the decay kernel shares out what is left, on top of them. */
+    if (min_quota > 0) {
+        int64_t can_hold = B / min_quota, taking_part = 0;
+        for (int f = W - 1; f >= 0; --f) {              /* nearest frame first */
+            if (!active[f]) continue;
+            if (taking_part >= can_hold) { active[f] = 0; continue; }
+            ++taking_part;
+            floor_q[f] = avail[f] < min_quota ? avail[f] : min_quota;
+            avail[f] -= floor_q[f];
+            B -= floor_q[f];
+        }
+    }
     for (;;) {
         u128 S = 0;
         int64_t room = 0;
@@ -183,9 +201,17 @@ int po_plan_budget(int kind, double param, int64_t total, int keep_full, int n_f
         for (int f = 0; f < W; ++f)
             if (active[f]) budget[f] = 0;
     }
+    for (int f = 0; f < W; ++f) budget[f] += floor_q[f];
     free(w);
     free(active);
+    free(avail);
+    free(floor_q);
     return PO_OK;
+}
+
+int po_plan_budget(int kind, double param, int64_t total, int keep_full, int n_frames,
+                   const int32_t *avail, int32_t *budget) {
+    return po_plan_budget_min(kind, param, total, keep_full, 0, n_frames, avail, budget);
 }
 
 /* ------------------------------------------------------------------------

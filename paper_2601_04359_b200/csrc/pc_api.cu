@@ -201,7 +201,7 @@ uint64_t decay_weight_q32(int kind, double param, int dist, int W, int keep_full
 
 extern "C" pc_status pc_plan_budget(const pc_budget_params *p, int32_t n_frames, const int32_t *avail, int32_t *budget) {
     if (!p || n_frames < 0 || (n_frames > 0 && (!avail || !budget))) return PC_ERR_INVALID_ARG;
-    if (p->total < 0 || p->keep_full < 0 || p->min_quota != 0) return PC_ERR_INVALID_ARG;
+    if (p->total < 0 || p->keep_full < 0 || p->min_quota < 0) return PC_ERR_INVALID_ARG;
     if (p->kind < PC_GEOMETRIC || p->kind > PC_HALFLIFE) return PC_ERR_INVALID_ARG;
     if (p->kind == PC_GEOMETRIC && !(p->param > 0.0 && p->param < 1.0)) return PC_ERR_INVALID_ARG;
     if (p->kind == PC_HALFLIFE && !(p->param > 0.0)) return PC_ERR_INVALID_ARG;
@@ -222,6 +222,23 @@ extern "C" pc_status pc_plan_budget(const pc_budget_params *p, int32_t n_frames,
         }
     }
     if (remaining < 0) return PC_ERR_BUDGET;
+
+    // Minimum quota (b_min of Sec. 3.4).  `live` runs oldest -> newest.  If every live frame's guarantee does not fit the
+    // budget, the oldest frames leave the window (first in, first out) until the guarantees of the rest do; each frame
+    // that stays is granted min(min_quota, what it holds) up front, and only its remaining room competes for the rest.
+    std::vector<int32_t> granted((size_t)W, 0), room_of((size_t)W, 0);
+    for (int f = 0; f < W; ++f) room_of[f] = avail[f];
+    if (p->min_quota > 0) {
+        const int64_t fits = remaining / p->min_quota;
+        if ((int64_t)live.size() > fits) live.erase(live.begin(), live.end() - (size_t)fits);
+        for (const Share &s : live) {
+            granted[s.frame] = std::min<int32_t>(p->min_quota, avail[s.frame]);
+            room_of[s.frame] -= granted[s.frame];
+            remaining -= granted[s.frame];
+        }
+    }
+    const int32_t *avail_all = avail;
+    avail = room_of.data();          // from here on a frame's capacity is what is left above its guarantee
 
     while (!live.empty() && remaining > 0) {
         u128 weight_sum = 0;
@@ -270,5 +287,7 @@ extern "C" pc_status pc_plan_budget(const pc_budget_params *p, int32_t n_frames,
         for (const Share &s : next) budget[s.frame] = 0;
         live.swap(next);
     }
+    (void)avail_all;
+    for (int f = 0; f < W; ++f) budget[f] += granted[f];
     return PC_OK;
 }

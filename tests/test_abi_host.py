@@ -90,5 +90,25 @@ def test_plan_budget_errors():
     with pytest.raises(pc.PackCacheError):
         pc.pc_plan_budget(pc.PC_LINEAR, 0.0, -1, 0, [5])
     with pytest.raises(pc.PackCacheError):
-        pc.pc_plan_budget(pc.PC_LINEAR, 0.0, 5, 0, [5], min_quota=1)
+        pc.pc_plan_budget(pc.PC_LINEAR, 0.0, 5, 0, [5], min_quota=-1)
     assert pc.pc_plan_budget(pc.PC_LINEAR, 0.0, 5, 0, []).tolist() == []
+
+
+@pytest.mark.parametrize("kind,param", KINDS)
+def test_plan_budget_with_minimum_quota_bit_exact_with_oracle(kind, param):
+    rng = np.random.default_rng(7)
+    for _ in range(60):
+        W = int(rng.integers(1, 20))
+        avail = rng.integers(0, 1200, size=W)
+        keep = int(rng.integers(0, 3))
+        m = int(rng.integers(0, 200))
+        total = int(rng.integers(0, int(avail.sum()) + 300))
+        try:
+            want = oracle.plan_budget(kind, param, total, keep, avail, min_quota=m).tolist()
+        except oracle.OracleError as e:
+            assert e.code == oracle.ERR_BUDGET
+            with pytest.raises(pc.PackCacheError) as g:
+                pc.pc_plan_budget(kind, param, total, keep, avail, min_quota=m)
+            assert g.value.status == pc.PC_ERR_BUDGET
+            continue
+        assert pc.pc_plan_budget(kind, param, total, keep, avail, min_quota=m).tolist() == want

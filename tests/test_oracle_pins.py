@@ -361,3 +361,72 @@ def test_anchors_survive_and_rebase_leaves_history_logits_unchanged():
     a = oracle.attend(L.q, L.q_pos, [(pk, pv, pp)])
     b = oracle.attend(L.q, qp2, [(pk2, pv2, pp2)])
     np.testing.assert_allclose(a, b, rtol=0, atol=1e-11)
+
+
+# ------------------------------------------------------------------------------------------- minimum quota (b_min)
+def _exact_plan_with_floor(weights, avail, total, m):
+    """Exact-rational statement of the minimum-quota rule for frames listed nearest first: the nearest floor(B/m) frames
+    take part, each is guaranteed min(m, avail), the rest is shared in proportion to the weights by largest remainder
+    (ties to the nearer frame), capping at what a frame holds and re-sharing the surplus."""
+    n = len(weights)
+    part = list(range(n)) if m == 0 else list(range(min(n, total // m)))
+    floor_q = [min(m, avail[i]) if i in part else 0 for i in range(n)]
+    room = [avail[i] - floor_q[i] for i in range(n)]
+    B = total - sum(floor_q)
+    extra = [0] * n
+    live = [i for i in part]
+    while live and B > 0:
+        if B >= sum(room[i] for i in live):
+            for i in live:
+                extra[i] = room[i]
+            break
+        S = sum(weights[i] for i in live)
+        if S == 0:
+            break
+        share = {i: Fraction(B * weights[i], S) for i in live}
+        for i in live:
+            extra[i] = share[i].numerator // share[i].denominator
+        left = B - sum(extra[i] for i in live)
+        order = sorted(live, key=lambda i: (-(share[i] - extra[i]), i))      # largest remainder, then nearer frame
+        for i in order[:left]:
+            extra[i] += 1
+        over = [i for i in live if extra[i] > room[i]]
+        if not over:
+            break
+        for i in over:
+            extra[i] = room[i]
+            B -= room[i]
+        live = [i for i in live if i not in over]
+        for i in live:
+            extra[i] = 0
+    return [floor_q[i] + extra[i] for i in range(n)]
+
+
+def test_plan_minimum_quota_against_exact_rationals():
+    rng = np.random.default_rng(11)
+    for _ in range(200):
+        W = int(rng.integers(1, 9))
+        avail = [int(x) for x in rng.integers(0, 90, size=W)]
+        m = int(rng.integers(0, 40))
+        total = int(rng.integers(0, sum(avail) + 40))
+        got = oracle.plan_budget(oracle.LINEAR, 0.0, total, 0, avail, min_quota=m).tolist()
+        near_first_w = [(W + 1 - d) << 32 for d in range(1, W + 1)]                # linear weights are exact in Q32
+        want = _exact_plan_with_floor(near_first_w, avail[::-1], total, m)[::-1]
+        assert got == want
+
+
+def test_plan_minimum_quota_properties():
+    n, W = 64, 6
+    base = oracle.plan_budget(oracle.CLOSED_HALF, 0.5, 128, 0, [n] * W).tolist()
+    assert oracle.plan_budget(oracle.CLOSED_HALF, 0.5, 128, 0, [n] * W, min_quota=0).tolist() == base
+    # every frame that takes part keeps at least the quota; the total is unchanged; still non-increasing with distance
+    q = oracle.plan_budget(oracle.CLOSED_HALF, 0.5, 128, 0, [n] * W, min_quota=8).tolist()
+    assert q == [10, 11, 13, 18, 28, 48] and sum(q) == 128 and min(q) >= 8 and q == sorted(q)
+    # guarantees beyond the budget: the window shrinks first in, first out (6 x 3 > 10: the three nearest frames stay)
+    t = oracle.plan_budget(oracle.LINEAR, 0.0, 10, 0, [n] * W, min_quota=3).tolist()
+    assert t == [0, 0, 0, 3, 3, 4]
+    # a frame that holds less than the quota keeps what it holds; kept-whole frames are outside the rule
+    u = oracle.plan_budget(oracle.HALFLIFE, 1.0, 100, 1, [2, 64, 64, 64, 64, 64], min_quota=5).tolist()
+    assert u[0] == 2 and u[-1] == 64 and sum(u) == 100 and all(x >= 5 for x in u[1:-1])
+    with pytest.raises(oracle.OracleError):
+        oracle.plan_budget(oracle.LINEAR, 0.0, 10, 0, [5], min_quota=-1)
