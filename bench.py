@@ -264,6 +264,21 @@ def run_cuda(args):
     pc.pc_set_timing(ctx, False)
     kern_ms = {k: (float(np.mean(v)) if v else None) for k, v in acc.items()}
 
+    # ---- one further attention pass over an unchanged cache (a frame is generated over several diffusion steps that all
+    # attend to the same keys): keys rotated once by pc_attend_prepare, each pass rotates only its queries
+    pc.pc_attend_prepare(ctx, dsts[0], None, stream=stream)
+    for i in range(5):
+        pc.pc_attend_prepared(ctx, layers[i % N_LAYERS].q, layers[i % N_LAYERS].q_pos, out=out, stream=stream)
+    barrier()
+    n_pass = min(args.steps, 200)
+    e0.record(stream)
+    for i in range(n_pass):
+        pc.pc_attend_prepared(ctx, layers[i % N_LAYERS].q, layers[i % N_LAYERS].q_pos, out=out, stream=stream)
+    e1.record(stream)
+    barrier()
+    pass_ms = max_over_ranks(e0.elapsed_time(e1) / n_pass, dist, "cuda")
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+
     # ---- the same frame step in the Slide regime of the cache window (incremental re-selection: the source of each pack is
     # what the last pack kept plus the newest frame, about 9 k tokens instead of the whole 47-frame history)
     N = cfg.frame_tokens
@@ -377,6 +392,8 @@ def run_cuda(args):
                      "peak_source": f"{peaks['source']} (burst; sustained {peaks['bf16_tflops_sustained']})",
                      "flops_per_launch": flops, "ms_per_launch": att_ms},
         "kernels_ms": stages,
+        "extra_pass": {"ms_per_pass": pass_ms, "what": "one more attention pass of the frame over the unchanged packed cache "
+                       "(pc_attend_prepared: query rotation, attention, merge; keys were rotated once per frame)"},
         "incremental": {"ms_per_frame": job_ms_per_frame(inc_ms, world) if inc_ms else None, "source_tokens": inc_src,
                         "mode": "cache window in the Slide regime: append the newest frame, drop the oldest, re-plan, "
                                 "score and re-select from packed + new, pack, attend (same keys attended)"},

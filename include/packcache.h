@@ -162,6 +162,17 @@ pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, c
 pc_status pc_attend_frame(pc_ctx *ctx, const pc_cache *cache, const pc_segment *current, const void *q,
                           const int32_t *q_pos, int32_t n_q, void *out, float *lse, void *stream);
 
+/* The same attention in two parts, for a frame that is generated over several passes that all attend to one unchanged
+ * cache (the diffusion steps of Sec. 3.1 / Fig. 4): pc_attend_prepare fixes the key set (anchors ++ history ++ current)
+ * and applies the rotary embedding to its keys once; pc_attend_prepared then runs one pass for the given queries and
+ * only rotates those.  Results are identical to pc_attend_frame on the same inputs.  The caller must not change the
+ * segments' K, V or positions between the two calls; the prepared key set lives in the context's scratch and is
+ * dropped by the next pc_attend_prepare or pc_attend_frame on this context.
+ * Errors: as pc_attend_frame; pc_attend_prepared returns PC_ERR_INVALID_ARG when nothing is prepared. */
+pc_status pc_attend_prepare(pc_ctx *ctx, const pc_cache *cache, const pc_segment *current, void *stream);
+pc_status pc_attend_prepared(pc_ctx *ctx, const void *q, const int32_t *q_pos, int32_t n_q, void *out, float *lse,
+                             void *stream);
+
 /* One frame step with inputs and output in HOST memory (pinned memory keeps the copies asynchronous): copies Q,
  * positions, anchors and the history frames into the caller's device workspace, plans the budget, scores, selects,
  * packs and attends (anchors ++ packed history), copies the output back and waits for the stream.  Everything the

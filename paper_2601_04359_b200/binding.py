@@ -25,7 +25,7 @@ EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact"
            "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_set_timing", "pc_get_timing",
            "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge",
            "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_update", "pc_window_cache",
-           "pc_window_state"]
+           "pc_window_state", "pc_attend_prepare", "pc_attend_prepared"]
 
 
 class pc_layer_desc(C.Structure):
@@ -107,6 +107,8 @@ def load() -> C.CDLL:
                                        C.POINTER(pc_budget_params), C.c_int32, C.c_void_p]
     lib.pc_score_tokens_static.argtypes = [C.POINTER(pc_layer_desc), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                            C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.pc_attend_prepare.argtypes = [C.c_void_p, C.POINTER(pc_cache), C.POINTER(pc_segment), C.c_void_p]
+    lib.pc_attend_prepared.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.pc_window_create.argtypes = [C.c_void_p, C.POINTER(pc_window_params), C.POINTER(pc_segment), C.POINTER(pc_segment),
                                      C.POINTER(pc_segment), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p)]
     lib.pc_window_destroy.argtypes = [C.c_void_p]
@@ -248,6 +250,24 @@ def pc_attend_frame(ctx: Context, cache: Cache, current: Optional[Segment], q: t
     cur = current.c() if current is not None else None
     _check(load().pc_attend_frame(ctx.handle, C.byref(c), C.byref(cur) if cur is not None else None, _ptr(q),
                                   _ptr(q_pos), q.shape[0], _ptr(out), _ptr(lse), _stream(stream)), "pc_attend_frame")
+    return (out, lse) if want_lse else out
+
+
+def pc_attend_prepare(ctx: Context, cache: Cache, current: Optional[Segment] = None, stream=None) -> None:
+    c = cache.c()
+    cur = current.c() if current is not None else None
+    _check(load().pc_attend_prepare(ctx.handle, C.byref(c), C.byref(cur) if cur is not None else None, _stream(stream)),
+           "pc_attend_prepare")
+
+
+def pc_attend_prepared(ctx: Context, q: torch.Tensor, q_pos: torch.Tensor, out: Optional[torch.Tensor] = None,
+                       lse: Optional[torch.Tensor] = None, want_lse: bool = False, stream=None):
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None and want_lse:
+        lse = torch.empty(q.shape[0], q.shape[1], dtype=torch.float32, device=q.device)
+    _check(load().pc_attend_prepared(ctx.handle, _ptr(q), _ptr(q_pos), q.shape[0], _ptr(out), _ptr(lse), _stream(stream)),
+           "pc_attend_prepared")
     return (out, lse) if want_lse else out
 
 

@@ -52,6 +52,7 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
     c->attend_impl = 0;
     c->kv_splits = 0;
     c->cluster_merge = 0;
+    c->prepared_n_seg = 0;
     c->timing_on = 0;
     c->ev_mask = 0;
     for (int i = 0; i < PC_N_MARKS; ++i) c->ev[i] = nullptr;

@@ -760,8 +760,10 @@ pc_status pc_attend_tc_scratch(const pc_layer_desc *d, int sm_count, size_t *k_r
     return PC_OK;
 }
 
+// what: PC_TC_ROPE_K rotates the segments' keys into the context scratch, PC_TC_ROPE_Q rotates the queries,
+// PC_TC_ATTEND runs attention (and the merge) on the rotated data.
 pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
-                              int32_t n_q, void *out, float *lse, cudaStream_t stream) {
+                              int32_t n_q, void *out, float *lse, cudaStream_t stream, int what) {
     const pc_layer_desc &D = ctx->desc;
     if (D.head_dim != TILE || D.dtype != PC_BF16) return PC_ERR_UNSUPPORTED;
     const int row_elems = D.n_kv_heads * D.head_dim;
@@ -771,26 +773,33 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     RopeJobs jobs{};
     const int k_chunks = row_elems / 8, q_chunks = D.n_q_heads * D.head_dim / 8;
     if (k_chunks % 32 || q_chunks % 32) return PC_ERR_UNSUPPORTED;
-    int tiles = 0, warps = 0;
+    int tiles = 0, warps = 0, n_jobs = 0;
     for (int s = 0; s < n_seg; ++s) {
-        jobs.job[s] = RopeJob{static_cast<const __nv_bfloat16 *>(segs[s].k), segs[s].pos,
-                              k_rot + (size_t)tiles * TILE * row_elems, segs[s].n_tokens, k_chunks, warps, 1.0f};
-        warps += segs[s].n_tokens;
+        if (what & PC_TC_ROPE_K) {
+            jobs.job[n_jobs++] = RopeJob{static_cast<const __nv_bfloat16 *>(segs[s].k), segs[s].pos,
+                                         k_rot + (size_t)tiles * TILE * row_elems, segs[s].n_tokens, k_chunks, warps, 1.0f};
+            warps += segs[s].n_tokens;
+        }
         tiles += div_up(segs[s].n_tokens, TILE);
         P.seg_tile_end[s] = tiles;
         P.seg_n[s] = segs[s].n_tokens;
     }
     if ((size_t)tiles * TILE > ctx->k_rot_rows) return PC_ERR_CAPACITY;
     __nv_bfloat16 *q_rot = static_cast<__nv_bfloat16 *>(ctx->q_rot);
-    jobs.job[n_seg] = RopeJob{static_cast<const __nv_bfloat16 *>(q), q_pos, q_rot, n_q, q_chunks, warps,
-                              (float)(1.4426950408889634 / std::sqrt((double)D.head_dim))};
-    warps += n_q;
-    jobs.n_jobs = n_seg + 1;
+    if (what & PC_TC_ROPE_Q) {
+        jobs.job[n_jobs++] = RopeJob{static_cast<const __nv_bfloat16 *>(q), q_pos, q_rot, n_q, q_chunks, warps,
+                                     (float)(1.4426950408889634 / std::sqrt((double)D.head_dim))};
+        warps += n_q;
+    }
+    jobs.n_jobs = n_jobs;
     jobs.total_warps = warps;
     pc_mark(ctx, PC_MARK_ATT0, stream);
-    PC_LAUNCH(k_rope_rows, dim3(div_up(warps, 8)), dim3(256), 0, stream, jobs, ctx->rope, D.head_dim, ctx->status);
-    PC_CUDA_TRY(cudaGetLastError());
+    if (n_jobs > 0) {
+        PC_LAUNCH(k_rope_rows, dim3(div_up(warps, 8)), dim3(256), 0, stream, jobs, ctx->rope, D.head_dim, ctx->status);
+        PC_CUDA_TRY(cudaGetLastError());
+    }
     pc_mark(ctx, PC_MARK_ROPE, stream);
+    if (!(what & PC_TC_ATTEND)) return PC_OK;
 
     P.n_q = n_q;
     P.n_q_heads = D.n_q_heads;

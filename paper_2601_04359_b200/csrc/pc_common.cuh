@@ -64,6 +64,9 @@ struct pc_ctx {
     void *q_rot;               // rotated, pre-scaled queries, bf16 [max_q][Hq][d]
     int kv_splits;             // 0 = chosen per call
     int cluster_merge;         // 1 = KV ranges merge inside the kernel through cluster shared memory (default 0)
+    // key set fixed by pc_attend_prepare (its rotated keys sit in k_rot until the next prepare or pc_attend_frame)
+    int prepared_n_seg;        // 0 = nothing prepared
+    pc_segment prepared_seg[PC_MAX_SEGMENTS];
     // optional per-kernel timing (benchmarks): events at the boundaries of the kernels of each call
     int timing_on;
     unsigned ev_mask;
@@ -203,7 +206,8 @@ pc_status pc_check_segment(const pc_segment *s, bool allow_empty);
 // stage launchers (each validates nothing: the pc_* entry points did)
 pc_status pc_launch_attend_simt(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
                                 int32_t n_q, void *out, float *lse, cudaStream_t stream);
+enum { PC_TC_ROPE_K = 1, PC_TC_ROPE_Q = 2, PC_TC_ATTEND = 4, PC_TC_ALL = 7 };
 pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
-                              int32_t n_q, void *out, float *lse, cudaStream_t stream);
+                              int32_t n_q, void *out, float *lse, cudaStream_t stream, int what);
 pc_status pc_attend_tc_scratch(const pc_layer_desc *d, int sm_count, size_t *k_rot_rows, size_t *part_o_floats,
                                size_t *part_ml_floats);

@@ -174,6 +174,38 @@ def test_attention_key_ranges_merge_like_one_range(cluster):
     ctx.close()
 
 
+# ------------------------------------------------------------------------------------------- prepared key set
+@pytest.mark.parametrize("cfg_name", ["tiny", "small_bf16"])
+def test_prepared_attention_equals_attend_frame_over_several_passes(cfg_name):
+    """A frame generated over several passes: the key set is prepared once (keys rotated once), each pass brings its own
+    queries.  Every pass must reproduce pc_attend_frame on the same inputs bit for bit, and match the oracle."""
+    cfg = wl.CONFIGS["tiny"] if cfg_name == "tiny" else wl.small_bf16(n_frames=3, grid=(11, 13), n_text=130, total=260, seed=4)
+    L = wl.make_layer(cfg, with_current=True)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    with pytest.raises(pc.PackCacheError):
+        pc.pc_attend_prepared(ctx, D.q, D.q_pos)                       # nothing prepared yet
+    pc.pc_attend_prepare(ctx, D.cache, D.current)
+    rng = np.random.default_rng(3)
+    segs = [(L.anchor_k, L.anchor_v, L.anchor_pos), (L.hist_k, L.hist_v, L.hist_pos), (L.cur_k, L.cur_v, L.q_pos)]
+    passes = []
+    for step in range(3):
+        q = wl.to_storage(rng.standard_normal(L.q.shape).astype(np.float32), cfg.dtype)
+        qd = dev(q, cfg.dtype)
+        got, lse = pc.pc_attend_prepared(ctx, qd, D.q_pos, want_lse=True)
+        want = oracle.attend(q, L.q_pos, segs, cfg.rope_base)
+        _check_attention(cfg, host(got).astype(np.float64), want)
+        passes.append((qd, got.clone(), lse.clone()))
+    _ok(ctx)
+    for qd, got, lse in passes:                                        # the one-call form gives the same bits
+        ref, ref_lse = pc.pc_attend_frame(ctx, D.cache, D.current, qd, D.q_pos, want_lse=True)
+        assert torch.equal(ref, got) and torch.equal(ref_lse, lse)
+    if cfg.dtype == wl.BF16:
+        with pytest.raises(pc.PackCacheError):                         # pc_attend_frame reused the scratch: prepare again
+            pc.pc_attend_prepared(ctx, D.q, D.q_pos)
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------------- select
 def _select_case(frame_count, budget, scores, cfg=None):
     cfg = cfg or wl.CONFIGS["tiny"]
