@@ -40,6 +40,7 @@ def main():
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--layers", type=int, default=28)
     ap.add_argument("--depths", type=str, default="1,2,3,4,6,8,12,16,24,32,40,44,45,46,47")
+    ap.add_argument("--stack", type=int, default=0, help="also time one frame through this many distinct layers (5.6 GB at 28)")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise RuntimeError("the sweep needs a CUDA device; there is no CPU fallback")
@@ -93,6 +94,23 @@ def main():
             grid.append(cell)
             print(json.dumps(cell), flush=True)
     assert pc.pc_poll_status(ctx) == pc.PC_OK
+    if args.stack > 0:
+        # one frame of the whole stack: every layer has its own seeded K / V / Q (its own compaction, its own attention)
+        stack = [D] + [DeviceLayer(wl.make_layer(cfg, layer=i)) for i in range(1, args.stack)]
+        dsts = [x.empty_packed(2 * N + 6048) for x in stack]
+        avail = np.full(cfg.n_frames, N, np.int32)
+
+        def frame():
+            for x, d in zip(stack, dsts):
+                budget = pc.pc_plan_budget(pc.PC_HALFLIFE, 4.0, 2 * N + 6048, 2, avail)
+                pc.pc_score(ctx, x.cache, x.q, x.q_pos, budget, scores=scores, sel_idx=sel, stream=stream)
+                pc.pc_compact(ctx, x.cache, sel, budget, 0, d, stream=stream)
+                pc.pc_attend_frame(ctx, d, None, x.q, x.q_pos, out=out, stream=stream)
+
+        t = _time(frame, max(3, args.reps // 4), stream)
+        assert pc.pc_poll_status(ctx) == pc.PC_OK
+        print(json.dumps({"stack_layers": args.stack, "history_frames": cfg.n_frames, "ms_per_frame": round(t, 3),
+                          "ms_per_layer": round(t / args.stack, 4)}), flush=True)
     late = [r for r in rows if r["history_frames"] >= 44]
     print(json.dumps({"summary": "last four frames (44-47 history frames), one layer",
                       "ms_full": round(sum(r["ms_full"] for r in late), 4), "ms_packcache": round(sum(r["ms_packcache"] for r in late), 4),
