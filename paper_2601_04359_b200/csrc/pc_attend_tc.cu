@@ -829,10 +829,11 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
         fprintf(stderr, "packcache: cuTensorMapEncodeTiled failed\n");
         return PC_ERR_CUDA;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[PC_MAX_DEVICES] = {};      // the attribute belongs to the device, not to the process
+    if (ctx->device < 0 || ctx->device >= PC_MAX_DEVICES) return PC_ERR_UNSUPPORTED;
+    if (!attr_set[ctx->device]) {
         PC_CUDA_TRY(cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
-        attr_set = true;
+        attr_set[ctx->device] = true;
     }
     P.cluster = (P.n_splits > 1 && ctx->cluster_merge) ? 1 : 0;
     if (P.cluster) {

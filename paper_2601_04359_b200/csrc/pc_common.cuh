@@ -35,6 +35,7 @@ enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT 
 
 constexpr int PC_QPOOL_BLOCKS = 128;
 constexpr int PC_MAX_SEGMENTS = 3;
+constexpr int PC_MAX_DEVICES = 64;            // per-device launch state is kept in arrays of this size
 
 // Rotary tables: for axis a (t, h, w) a [max_pos[a]][n_axis[a]] array of (cos, sin) of pos * base^(-m/n_axis[a]).
 // Pair i of a head uses axis i % 3 and column m = i / 3.

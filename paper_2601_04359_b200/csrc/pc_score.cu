@@ -450,14 +450,18 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
 #define PC_SCORE_CASE(CPL)                                                                                          \
     case CPL: {                                                                                                     \
         const int smem = SCORE_STAGES * (SCORE_TOK * CPL * 512 + SCORE_TOK * 16);                                   \
-        static int per_sm = 0; /* resident blocks per SM of this instance: the grid is persistent */              \
-        if (per_sm == 0) {                                                                                          \
+        /* resident blocks per SM of this instance (the grid is persistent), looked up once per device */          \
+        static int per_sm_of[PC_MAX_DEVICES] = {};                                                                  \
+        int dev_id = 0;                                                                                             \
+        PC_CUDA_TRY(cudaGetDevice(&dev_id));                                                                        \
+        if (dev_id < 0 || dev_id >= PC_MAX_DEVICES) return PC_ERR_UNSUPPORTED;                                      \
+        if (per_sm_of[dev_id] == 0) {                                                                               \
             PC_CUDA_TRY(cudaFuncSetAttribute(k_score<T, CPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));  \
             int occ = 0;                                                                                            \
             PC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_score<T, CPL>, SCORE_THREADS, smem)); \
-            per_sm = std::max(1, occ);                                                                              \
+            per_sm_of[dev_id] = std::max(1, occ);                                                                   \
         }                                                                                                           \
-        const int blocks = std::max(1, std::min(n_tiles, sm_count * per_sm));                                       \
+        const int blocks = std::max(1, std::min(n_tiles, sm_count * per_sm_of[dev_id]));                            \
         PC_LAUNCH((k_score<T, CPL>), dim3(blocks), dim3(SCORE_THREADS), smem, stream, k, hist_pos, valid, n_src, D.head_dim, scale, rope, \
                                                                  pooled, scores, status);                          \
     } break;
@@ -546,7 +550,7 @@ namespace {
 
 constexpr int STATIC_MAX_ROW = 1024;          // n_kv_heads * head_dim
 constexpr int STATIC_MAX_ROPE = 32768;        // rotary table entries: sum over axes of max_pos * pairs on that axis
-constexpr int STATIC_MAX_DEVICES = 64;
+constexpr int STATIC_MAX_DEVICES = PC_MAX_DEVICES;
 
 constexpr size_t STATIC_OFF_POOLED = 256;  /* first 256 bytes unused */                                                  // float [STATIC_MAX_ROW]
 constexpr size_t STATIC_OFF_PARTIAL = STATIC_OFF_POOLED + STATIC_MAX_ROW * sizeof(float);  // float [PC_QPOOL_BLOCKS][STATIC_MAX_ROW]
