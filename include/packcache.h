@@ -265,6 +265,13 @@ pc_status pc_window_destroy(pc_window *w);
  * history frame: device-to-device copies on the stream.  Errors: PC_ERR_CAPACITY (active buffer full). */
 pc_status pc_window_append(pc_window *w, const pc_segment *frame, void *stream);
 
+/* Append only the unmasked positions of a finished frame (cache mask of Eq. 1; Fig. 6b: masked positions are removed,
+ * not stored): valid is a device array of frame->n_tokens bytes, non-zero = keep; n_valid (host) is how many are
+ * non-zero, which the caller knows from its masking schedule.  Kept rows keep their order and positions.  A mask
+ * whose count differs from n_valid is recorded in the context's status word (PC_ERR_INVALID_ARG).
+ * Errors: PC_ERR_INVALID_ARG, PC_ERR_CAPACITY. */
+pc_status pc_window_append_masked(pc_window *w, const pc_segment *frame, const uint8_t *valid, int32_t n_valid, void *stream);
+
 /* Bring the cache back inside window and budget for the frame whose queries are q (see the regimes above); regime
  * (host out, may be NULL) receives PC_WINDOW_FILL / PACK / SLIDE.  scores_override: device fp32 scores of the source
  * tokens (after dropped frames) to select on instead of scoring, or NULL.  Errors as pc_score / pc_compact. */

@@ -30,7 +30,10 @@ class WindowRef:
         self.count: List[int] = []
         self.t_shift = 0
 
-    def append(self, k: np.ndarray, v: np.ndarray, pos: np.ndarray) -> None:
+    def append(self, k: np.ndarray, v: np.ndarray, pos: np.ndarray, valid: Optional[np.ndarray] = None) -> None:
+        if valid is not None:                      # cache mask (Eq. 1): masked positions are removed, not stored
+            keep = np.asarray(valid) != 0
+            k, v, pos = k[keep], v[keep], pos[keep]
         cat = lambda a, b: b.copy() if a is None else np.concatenate([a, b], axis=0)
         self.k, self.v, self.pos = cat(self.k, k), cat(self.v, v), cat(self.pos, pos)
         self.count.append(len(k))

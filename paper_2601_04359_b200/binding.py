@@ -24,7 +24,7 @@ PC_MAX_FRAMES = 256
 EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact", "pc_attend_frame",
            "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_set_timing", "pc_get_timing",
            "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge",
-           "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_update", "pc_window_cache",
+           "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_append_masked", "pc_window_update", "pc_window_cache",
            "pc_window_state", "pc_attend_prepare", "pc_attend_prepared"]
 
 
@@ -113,6 +113,7 @@ def load() -> C.CDLL:
                                      C.POINTER(pc_segment), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p)]
     lib.pc_window_destroy.argtypes = [C.c_void_p]
     lib.pc_window_append.argtypes = [C.c_void_p, C.POINTER(pc_segment), C.c_void_p]
+    lib.pc_window_append_masked.argtypes = [C.c_void_p, C.POINTER(pc_segment), C.c_void_p, C.c_int32, C.c_void_p]
     lib.pc_window_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int32), C.c_void_p]
     lib.pc_window_cache.argtypes = [C.c_void_p, C.POINTER(pc_cache)]
     lib.pc_window_state.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int64),
@@ -350,6 +351,11 @@ class Window:
     def append(self, frame: Segment, stream=None) -> None:
         f = frame.c()
         _check(load().pc_window_append(self.handle, C.byref(f), _stream(stream)), "pc_window_append")
+
+    def append_masked(self, frame: Segment, valid: torch.Tensor, n_valid: int, stream=None) -> None:
+        f = frame.c()
+        _check(load().pc_window_append_masked(self.handle, C.byref(f), _ptr(valid), n_valid, _stream(stream)),
+               "pc_window_append_masked")
 
     def update(self, q: Optional[torch.Tensor], q_pos: Optional[torch.Tensor], scores_override: Optional[torch.Tensor] = None,
                stream=None) -> int:

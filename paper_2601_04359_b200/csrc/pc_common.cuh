@@ -27,6 +27,7 @@ enum {
     PC_WHERE_ATTN_WAIT = 6,
     PC_WHERE_ROPE_POS = 7,
     PC_WHERE_SCORE_WAIT = 8,
+    PC_WHERE_MASK_COUNT = 9,
 };
 
 // event marks: score call 0-3, pack 4-5, attend 6-9
@@ -205,6 +206,8 @@ bool pc_aligned16(const void *p);
 pc_status pc_check_segment(const pc_segment *s, bool allow_empty);
 
 // stage launchers (each validates nothing: the pc_* entry points did)
+pc_status pc_launch_pack(pc_ctx *ctx, const void *src_k, const void *src_v, const int32_t *src_pos, const int32_t *sel_idx,
+                         int n_sel, int n_src, int delta_t, void *dst_k, void *dst_v, int32_t *dst_pos, cudaStream_t stream);
 pc_status pc_launch_attend_simt(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
                                 int32_t n_q, void *out, float *lse, cudaStream_t stream);
 enum { PC_TC_ROPE_K = 1, PC_TC_ROPE_Q = 2, PC_TC_ATTEND = 4, PC_TC_ALL = 7 };

@@ -86,11 +86,22 @@ extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t 
         overlaps(src->history.k, src_bytes, D.v, dst_bytes) || overlaps(src->history.v, src_bytes, D.k, dst_bytes) ||
         overlaps(src->history.pos, (size_t)n_src * 16, D.pos, (size_t)n_sel * 16))
         return PC_ERR_INVALID_ARG;
-    const int blocks = (int)((n_sel * 32 + PACK_THREADS - 1) / PACK_THREADS);
-    const char *sk = static_cast<const char *>(src->history.k), *sv = static_cast<const char *>(src->history.v);
-    char *dk = static_cast<char *>(D.k), *dv = static_cast<char *>(D.v);
-#define PC_PACK_ARGS sk, sv, src->history.pos, sel_idx, (int)n_sel, (int)n_src, row_bytes, delta_t, dk, dv, D.pos, ctx->status
     pc_mark(ctx, PC_MARK_PACK0, stream);
+    st = pc_launch_pack(ctx, src->history.k, src->history.v, src->history.pos, sel_idx, (int)n_sel, (int)n_src, delta_t, D.k, D.v,
+                        D.pos, stream);
+    if (st != PC_OK) return st;
+    pc_mark(ctx, PC_MARK_PACK, stream);
+    return PC_OK;
+}
+
+// Gather n_sel rows (K, V, position records) of a source of n_src rows into a destination; arguments already checked.
+pc_status pc_launch_pack(pc_ctx *ctx, const void *src_k, const void *src_v, const int32_t *src_pos, const int32_t *sel_idx,
+                         int n_sel, int n_src, int delta_t, void *dst_k, void *dst_v, int32_t *dst_pos, cudaStream_t stream) {
+    const int row_bytes = ctx->desc.n_kv_heads * ctx->desc.head_dim * ctx->elem_size;
+    const int blocks = (int)(((int64_t)n_sel * 32 + PACK_THREADS - 1) / PACK_THREADS);
+    const char *sk = static_cast<const char *>(src_k), *sv = static_cast<const char *>(src_v);
+    char *dk = static_cast<char *>(dst_k), *dv = static_cast<char *>(dst_v);
+#define PC_PACK_ARGS sk, sv, src_pos, sel_idx, n_sel, n_src, row_bytes, delta_t, dk, dv, dst_pos, ctx->status
     switch (row_bytes) {
     case 512: PC_LAUNCH((k_pack<1>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
     case 1024: PC_LAUNCH((k_pack<2>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
@@ -99,6 +110,5 @@ extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t 
     }
 #undef PC_PACK_ARGS
     PC_CUDA_TRY(cudaGetLastError());
-    pc_mark(ctx, PC_MARK_PACK, stream);
     return PC_OK;
 }

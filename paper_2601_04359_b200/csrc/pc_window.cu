@@ -1,5 +1,5 @@
 // Cache window: the Fill / Pack / Slide regimes (Sec. 3.4, Fig. 6) and the temporal rebase (Eq. 9) as a host-side state
-// machine around pc_plan_budget, pc_score and pc_compact.  No kernels of its own.
+// machine around pc_plan_budget, pc_score and pc_compact; its one kernel turns a cache mask (Eq. 1) into row indices.
 #include <vector>
 
 #include "pc_common.cuh"
@@ -72,6 +72,67 @@ extern "C" pc_status pc_window_append(pc_window *w, const pc_segment *frame, voi
     PC_CUDA_TRY(cudaMemcpyAsync(A.pos + 4 * (size_t)A.n_tokens, frame->pos, (size_t)n * 16, cudaMemcpyDeviceToDevice, stream));
     A.n_tokens += n;
     w->count.push_back(n);
+    return PC_OK;
+}
+
+namespace {
+
+// Indices of the non-zero bytes of valid[0..n), ascending, into idx; one block, a scan per 1024 bytes.  The host states how
+// many there are (it sizes the frame table without a device round trip): a different count is recorded as an error.
+__global__ void __launch_bounds__(1024) k_mask_to_index(const uint8_t *__restrict__ valid, int n, int32_t *__restrict__ idx,
+                                                        int expected, int32_t *status) {
+    pc_grid_dep_launch();
+    pc_grid_dep_wait();
+    __shared__ int warp_sums[32];
+    __shared__ int carry;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int j0 = 0; j0 < n; j0 += 1024) {
+        const int j = j0 + threadIdx.x;
+        const int keep = j < n && valid[j] != 0;
+        int inc = keep;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
+        }
+        if (lane == 31) warp_sums[w] = inc;
+        __syncthreads();
+        int base = carry;
+        for (int i = 0; i < w; ++i) base += warp_sums[i];
+        const int at = base + inc - keep;
+        if (keep && at < expected) idx[at] = j;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = base + inc;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && carry != expected) pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_MASK_COUNT);
+}
+
+}  // namespace
+
+extern "C" pc_status pc_window_append_masked(pc_window *w, const pc_segment *frame, const uint8_t *valid, int32_t n_valid,
+                                             void *stream_) {
+    if (!w || !frame || !valid) return PC_ERR_INVALID_ARG;
+    pc_status st = pc_check_segment(frame, false);
+    if (st != PC_OK) return st;
+    if (n_valid < 0 || n_valid > frame->n_tokens) return PC_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    pc_segment &A = w->buf[w->active];
+    if ((int64_t)A.n_tokens + n_valid > A.capacity || frame->n_tokens > w->scratch_capacity) return PC_ERR_CAPACITY;
+    if ((int)w->count.size() + 1 > PC_MAX_FRAMES) return PC_ERR_CAPACITY;
+    if (n_valid > 0) {
+        const size_t row = (size_t)w->ctx->desc.n_kv_heads * w->ctx->desc.head_dim * w->ctx->elem_size;
+        PC_LAUNCH(k_mask_to_index, dim3(1), dim3(1024), 0, stream, valid, (int)frame->n_tokens, w->sel_idx, (int)n_valid,
+                  w->ctx->status);
+        st = pc_launch_pack(w->ctx, frame->k, frame->v, frame->pos, w->sel_idx, n_valid, frame->n_tokens, 0,
+                            static_cast<char *>(A.k) + (size_t)A.n_tokens * row, static_cast<char *>(A.v) + (size_t)A.n_tokens * row,
+                            A.pos + 4 * (size_t)A.n_tokens, stream);
+        if (st != PC_OK) return st;
+    }
+    A.n_tokens += n_valid;
+    w->count.push_back(n_valid);
     return PC_OK;
 }
 

@@ -182,3 +182,65 @@ def test_window_on_its_own_scores_keeps_valid_state():
         kept = now
         counts_before = counts.tolist()
     win.close(); ctx.close()
+
+
+def test_masked_append_removes_positions_in_the_reference():
+    """Cache mask of Eq. 1 at write time: masked positions never enter the cache (their tags never appear), the frame's
+    count is the number of unmasked positions, order and coordinates of the kept ones are untouched."""
+    cfg = wl.CONFIGS["tiny"]
+    n = cfg.frame_tokens
+    fr = _frames(cfg, 3, seed=6)
+    rng = np.random.default_rng(4)
+    ref = ow.WindowRef(4, oracle.CLOSED_HALF, 0.5, 10 ** 6, 0)             # budget never binds: only the mask removes
+    kept_tags = []
+    for f in range(3):
+        valid = (rng.random(n) < 0.6).astype(np.uint8)
+        ref.append(fr[f]["k"], fr[f]["v"], fr[f]["pos"], valid=valid)
+        assert ref.update(fr[f + 1]["q"], fr[f + 1]["pos"]) == ow.FILL
+        kept_tags += fr[f]["pos"][valid != 0, 3].tolist()
+        assert ref.count[-1] == int(valid.sum())
+    assert ref.pos[:, 3].tolist() == kept_tags
+    assert np.array_equal(ref.k, np.concatenate([fr[f]["k"] for f in range(3)])[np.isin(
+        np.concatenate([fr[f]["pos"][:, 3] for f in range(3)]), kept_tags)])
+
+
+@pytest.mark.gpu
+def test_window_masked_append_matches_reference():
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200.device import dev, host, idev, make_ctx, segment
+
+    cfg = wl.small_bf16(n_frames=6, grid=(33, 35), n_text=37, total=900, kind=wl.HALFLIFE, param=2.0, keep_full=1, seed=12)
+    n, W, total = cfg.frame_tokens, 3, 900                                   # 1155 tokens per frame: more than one scan chunk
+    L = wl.make_layer(cfg)
+    fr = _frames(cfg, 5, seed=13)
+    ctx = make_ctx(cfg, max_keys=cfg.n_anchor + total + 3 * n)
+    cap = total + 2 * n
+    mk = lambda: pc.Segment(torch.full((cap, cfg.n_kv_heads, cfg.head_dim), 5.0, dtype=torch.bfloat16, device="cuda"),
+                            torch.full((cap, cfg.n_kv_heads, cfg.head_dim), 5.0, dtype=torch.bfloat16, device="cuda"),
+                            torch.full((cap, 4), -3, dtype=torch.int32, device="cuda"), 0)
+    win = pc.Window(ctx, W, pc.PC_HALFLIFE, 2.0, total, 1, segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype), mk(), mk())
+    ref = ow.WindowRef(W, oracle.HALFLIFE, 2.0, total, 1)
+    rng = np.random.default_rng(1)
+    for f in range(5):
+        valid = (rng.random(n) < (0.7 if f % 2 else 0.35)).astype(np.uint8)
+        if f == 2:
+            valid[:] = 0; valid[[0, 511, 1024, n - 1]] = 1                   # nearly empty, with survivors at chunk edges
+        ref.append(fr[f]["k"], fr[f]["v"], fr[f]["pos"], valid=valid)
+        win.append_masked(segment(fr[f]["k"], fr[f]["v"], fr[f]["pos"], cfg.dtype), torch.from_numpy(valid).cuda(), int(valid.sum()))
+        sk, _, spos, _, _ = ref.source_after_drop()
+        s32 = oracle.score_pooled(sk, spos, fr[f + 1]["q"], fr[f + 1]["pos"], cfg.rope_base).astype(np.float32)
+        want = ref.update(fr[f + 1]["q"], fr[f + 1]["pos"], scores32=s32)
+        got = win.update(dev(fr[f + 1]["q"], cfg.dtype), idev(fr[f + 1]["pos"]), scores_override=torch.from_numpy(s32).cuda())
+        assert got == want and pc.pc_poll_status(ctx) == pc.PC_OK
+        counts, _, _ = win.state()
+        assert counts.tolist() == ref.count
+        cache = win.cache()
+        m = int(counts.sum())
+        assert np.array_equal(host(cache.history.k)[:m], ref.k) and np.array_equal(cache.history.pos.cpu().numpy()[:m], ref.pos)
+        assert np.array_equal(host(cache.history.v)[:m], ref.v)
+    # a count that does not match the mask is recorded, not trusted
+    valid = np.ones(n, np.uint8)
+    win.append_masked(segment(fr[0]["k"], fr[0]["v"], fr[0]["pos"], cfg.dtype), torch.from_numpy(valid).cuda(), n - 5)
+    assert pc.pc_poll_status(ctx) == pc.PC_ERR_INVALID_ARG
+    win.close(); ctx.close()
