@@ -238,7 +238,6 @@ extern "C" pc_status pc_plan_budget(const pc_budget_params *p, int32_t n_frames,
             remaining -= granted[s.frame];
         }
     }
-    const int32_t *avail_all = avail;
     avail = room_of.data();          // from here on a frame's capacity is what is left above its guarantee
 
     while (!live.empty() && remaining > 0) {
@@ -288,7 +287,6 @@ extern "C" pc_status pc_plan_budget(const pc_budget_params *p, int32_t n_frames,
         for (const Share &s : next) budget[s.frame] = 0;
         live.swap(next);
     }
-    (void)avail_all;
     for (int f = 0; f < W; ++f) budget[f] += granted[f];
     return PC_OK;
 }

@@ -361,28 +361,36 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         // ---------------------------------------------------------------- TMA producer
         reg_dealloc<72>();
         if (lane == 0) {
-            mbar_expect_tx(bar(BAR_Q), n_tiles_q * TILE_BYTES);
+            // The first K tile rides with the query tiles.  After that V(j) and K(j+1) always travel together: they are
+            // needed at the same point (top of step j) and their stages are released at the same point (end of step j),
+            // so one full / empty barrier pair serves both and the issuer has one wait and one commit less per step.
+            mbar_expect_tx(bar(BAR_Q), (n_tiles_q + (n_j > 0 ? 1 : 0)) * TILE_BYTES);
             for (int t = 0; t < n_tiles_q; ++t) {
                 const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
                 tma_load_2d(base + SM_Q + t * TILE_BYTES, &map_q, h * TILE, tb * TILE, bar(BAR_Q));
                 tma_load_2d(base + SM_Q + t * TILE_BYTES + HALF_BYTES, &map_q, h * TILE + 64, tb * TILE, bar(BAR_Q));
             }
+            if (n_j > 0) {
+                tma_load_2d(base + SM_K, &map_k, g * TILE, jt0 * TILE, bar(BAR_Q));
+                tma_load_2d(base + SM_K + HALF_BYTES, &map_k, g * TILE + 64, jt0 * TILE, bar(BAR_Q));
+            }
             bool alive = true;
             for (int j = 0; j < n_j && alive; ++j) {
-                const int st = j % KV_STAGES, use = j / KV_STAGES;
+                const int st = j % KV_STAGES, use = j / KV_STAGES, kst = (j + 1) % KV_STAGES;
                 int seg, local, n_valid;
                 kv_tile_info(P, jt0 + j, seg, local, n_valid);
                 const CUtensorMap *mv = seg == 0 ? &map_v0 : (seg == 1 ? &map_v1 : &map_v2);
-                if (use > 0) alive = mbar_wait(bar(BAR_KEMPTY + st), (use - 1) & 1, abort_flag, P.status);
-                if (!alive) break;
-                mbar_expect_tx(bar(BAR_KFULL + st), TILE_BYTES);
-                tma_load_2d(base + SM_K + st * TILE_BYTES, &map_k, g * TILE, (jt0 + j) * TILE, bar(BAR_KFULL + st));
-                tma_load_2d(base + SM_K + st * TILE_BYTES + HALF_BYTES, &map_k, g * TILE + 64, (jt0 + j) * TILE, bar(BAR_KFULL + st));
                 if (use > 0) alive = mbar_wait(bar(BAR_VEMPTY + st), (use - 1) & 1, abort_flag, P.status);
+                else if (j == 1) alive = mbar_wait(bar(BAR_KEMPTY + 0), 0, abort_flag, P.status);   // K(2) lands where K(0) was
                 if (!alive) break;
-                mbar_expect_tx(bar(BAR_VFULL + st), TILE_BYTES);
+                const bool more = j + 1 < n_j;
+                mbar_expect_tx(bar(BAR_VFULL + st), (more ? 2 : 1) * TILE_BYTES);
                 tma_load_2d(base + SM_V + st * TILE_BYTES, mv, g * TILE, local * TILE, bar(BAR_VFULL + st));
                 tma_load_2d(base + SM_V + st * TILE_BYTES + HALF_BYTES, mv, g * TILE + 64, local * TILE, bar(BAR_VFULL + st));
+                if (more) {
+                    tma_load_2d(base + SM_K + kst * TILE_BYTES, &map_k, g * TILE, (jt0 + j + 1) * TILE, bar(BAR_VFULL + st));
+                    tma_load_2d(base + SM_K + kst * TILE_BYTES + HALF_BYTES, &map_k, g * TILE + 64, (jt0 + j + 1) * TILE, bar(BAR_VFULL + st));
+                }
             }
             if (*abort_flag) {
                 // give the copies already issued a bounded chance to land before the CTA's shared memory goes away
@@ -406,7 +414,6 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 if (lead) mma_ss(tm + t * TILE, desc_kmajor(qa + off), desc_kmajor(ka + off), IDESC_QK, ks > 0);
             }
         };
-        if (alive && n_j > 0) alive = mbar_wait(bar(BAR_KFULL + 0), 0, abort_flag, P.status);
         if (alive && n_j > 0) {
             tc_fence_after();
             for (int t = 0; t < n_tiles_q; ++t) {
@@ -417,9 +424,8 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         }
         for (int j = 0; j < n_j && alive; ++j) {
             const int st = j % KV_STAGES, use = j / KV_STAGES;
-            const int nst = (j + 1) % KV_STAGES, nuse = (j + 1) / KV_STAGES;
-            alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status);
-            if (alive && j + 1 < n_j) alive = mbar_wait(bar(BAR_KFULL + nst), nuse & 1, abort_flag, P.status);
+            const int nst = (j + 1) % KV_STAGES;
+            alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status);      // V(j) and K(j+1)
             for (int t = 0; t < n_tiles_q && alive; ++t) {
                 const uint32_t va = base + SM_V + st * TILE_BYTES;
                 // P arrives in two halves of 64 keys: the first PV steps run while the rest is exponentiated
@@ -439,8 +445,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 if (lead) tc_commit(bar(BAR_SFULL + t));          // S_t(j+1) ready, or after the last tile: O_t final
             }
             if (alive && lead) {
-                tc_commit(bar(BAR_VEMPTY + st));
-                if (j + 1 < n_j) tc_commit(bar(BAR_KEMPTY + nst));
+                tc_commit(bar(BAR_VEMPTY + st));            // PV(j) and QK(j+1) are behind this: V stage st and K stage nst are free
             }
         }
         // make sure nothing of ours is still running on the tensor core before TMEM is freed
