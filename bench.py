@@ -34,7 +34,7 @@ N_LAYERS = 4          # rotated input sets; 4 x ~0.2 GB > L2 (--layers changes i
 KERNELS_PER_STEP = 8  # k_qpool, k_qpool_reduce, k_score, k_select, k_pack, k_rope_rows, k_attend_tc, k_combine
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_attend_tc launch at this workload, from the ncu capture
 # summarised in profiles/ncu_kernels_lumos47_small_case.md (same launch shape); None when the kernel has changed since
-ATTEND_DRAM_TRAFFIC = 43_983_616 + 3_283_968
+ATTEND_DRAM_TRAFFIC = 43_979_776 + 3_303_424
 
 
 def _peaks():
@@ -266,18 +266,20 @@ def run_cuda(args):
 
     # ---- one further attention pass over an unchanged cache (a frame is generated over several diffusion steps that all
     # attend to the same keys): keys rotated once by pc_attend_prepare, each pass rotates only its queries
-    pc.pc_attend_prepare(ctx, dsts[0], None, stream=stream)
-    for i in range(5):
-        pc.pc_attend_prepared(ctx, layers[i % N_LAYERS].q, layers[i % N_LAYERS].q_pos, out=out, stream=stream)
-    barrier()
-    n_pass = min(args.steps, 200)
-    e0.record(stream)
-    for i in range(n_pass):
-        pc.pc_attend_prepared(ctx, layers[i % N_LAYERS].q, layers[i % N_LAYERS].q_pos, out=out, stream=stream)
-    e1.record(stream)
-    barrier()
-    pass_ms = max_over_ranks(e0.elapsed_time(e1) / n_pass, dist, "cuda")
-    assert pc.pc_poll_status(ctx) == pc.PC_OK
+    pass_ms = None
+    if not args.no_extra_pass:
+        pc.pc_attend_prepare(ctx, dsts[0], None, stream=stream)
+        for i in range(5):
+            pc.pc_attend_prepared(ctx, layers[i % N_LAYERS].q, layers[i % N_LAYERS].q_pos, out=out, stream=stream)
+        barrier()
+        n_pass = min(args.steps, 200)
+        e0.record(stream)
+        for i in range(n_pass):
+            pc.pc_attend_prepared(ctx, layers[i % N_LAYERS].q, layers[i % N_LAYERS].q_pos, out=out, stream=stream)
+        e1.record(stream)
+        barrier()
+        pass_ms = max_over_ranks(e0.elapsed_time(e1) / n_pass, dist, "cuda")
+        assert pc.pc_poll_status(ctx) == pc.PC_OK
 
     # ---- the same frame step in the Slide regime of the cache window (incremental re-selection: the source of each pack is
     # what the last pack kept plus the newest frame, about 9 k tokens instead of the whole 47-frame history)
@@ -424,6 +426,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
     ap.add_argument("--no-incremental", action="store_true", help="skip the cache-window leg (profiler captures)")
+    ap.add_argument("--no-extra-pass", action="store_true", help="skip the prepared-attention leg (profiler captures)")
     ap.add_argument("--layers", type=int, default=N_LAYERS, help="rotated input sets (default 4, > L2)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
