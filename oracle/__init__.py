@@ -168,6 +168,22 @@ def attend(q, q_pos, segments, base=10000.0, rows=None, want_lse=False):
     return (out, lse) if want_lse else out
 
 
+def attend_mass(q, q_pos, segments, base=10000.0) -> np.ndarray:
+    """Mean attention probability every key receives (Sec. 3.4); segments: list of (k, pos) or (k, v, pos)."""
+    q, q_pos = _f32(q), _i32(q_pos)
+    n_q, hq, d = q.shape
+    segs = [(_f32(s[0]), _i32(s[-1])) for s in segments if len(s[0])]
+    hkv = segs[0][0].shape[1]
+    ns = len(segs)
+    ka = (C.POINTER(C.c_float) * ns)(*[_p(s[0], C.c_float) for s in segs])
+    pa = (C.POINTER(C.c_int32) * ns)(*[_p(s[1], C.c_int32) for s in segs])
+    na = (C.c_int64 * ns)(*[len(s[0]) for s in segs])
+    out = np.empty(sum(len(s[0]) for s in segs), dtype=np.float64)
+    _check(lib().po_attend_mass(_p(q, C.c_float), _p(q_pos, C.c_int32), C.c_int(n_q), C.c_int(hq), C.c_int(hkv),
+                                C.c_int(d), C.c_double(base), C.c_int(ns), ka, pa, na, _p(out, C.c_double)))
+    return out
+
+
 def full_block_causal_attention(q, k, v, pos, block, base=10000.0) -> np.ndarray:
     q, k, v, pos, block = _f32(q), _f32(k), _f32(v), _i32(pos), _i32(block)
     n, hq, d = q.shape

@@ -476,3 +476,73 @@ int po_full_block_causal_attention(const float *q, const float *k, const float *
     free(rk);
     return PO_OK;
 }
+
+/* ------------------------------------------------------------------------
+ * Attention mass of every key (Sec. 3.4: the mean attention score a cached
+ * token receives, the quantity "attention-guided" retention ranks by):
+ *   mass_j = 1/(n_q*Hq) * sum_i sum_h softmax_j( (R q_ih).(R k_j,g(h)) / sqrt(d) )
+ * over the same key set as po_attend (every key visible, Eq. 2).  The masses
+ * of all keys sum to one.  mass [n_k], keys in segment order.
+ * ------------------------------------------------------------------------ */
+int po_attend_mass(const float *q, const int32_t *q_pos, int n_q, int n_q_heads, int n_kv_heads, int d,
+                   double base, int n_seg, const float *const *seg_k, const int32_t *const *seg_pos,
+                   const int64_t *seg_n, double *mass) {
+    if (n_q_heads % n_kv_heads || n_q <= 0) return PO_ERR_ARG;
+    int G = n_q_heads / n_kv_heads;
+    int64_t n_k = 0;
+    for (int s = 0; s < n_seg; ++s) n_k += seg_n[s];
+    if (n_k <= 0) return PO_ERR_ARG;
+    double *rk = (double *)malloc(sizeof(double) * (size_t)n_k * n_kv_heads * d);
+    if (!rk) return PO_ERR_ARG;
+    int64_t off = 0;
+    for (int s = 0; s < n_seg; ++s) {
+        double *r = rope_all(seg_k[s], seg_pos[s], seg_n[s], n_kv_heads, d, base);
+        memcpy(rk + (size_t)off * n_kv_heads * d, r, sizeof(double) * (size_t)seg_n[s] * n_kv_heads * d);
+        free(r);
+        off += seg_n[s];
+    }
+    double *rq = rope_all(q, q_pos, n_q, n_q_heads, d, base);
+    int64_t total = (int64_t)n_q * n_q_heads;
+    double *lse = (double *)malloc(sizeof(double) * (size_t)total);
+    if (!rq || !lse) { free(rk); free(rq); free(lse); return PO_ERR_ARG; }
+    double inv_sqrt_d = 1.0 / sqrt((double)d);
+    /* first the normaliser of every query row: lse_e = log sum_j exp(logit_ej) */
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t e = 0; e < total; ++e) {
+        int g = (int)(e % n_q_heads) / G;
+        const double *qq = rq + (size_t)e * d;
+        double mx = -INFINITY;
+        for (int64_t j = 0; j < n_k; ++j) {
+            const double *kk = rk + ((size_t)j * n_kv_heads + g) * d;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += qq[c] * kk[c];
+            if (dot * inv_sqrt_d > mx) mx = dot * inv_sqrt_d;
+        }
+        double denom = 0.0;
+        for (int64_t j = 0; j < n_k; ++j) {
+            const double *kk = rk + ((size_t)j * n_kv_heads + g) * d;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += qq[c] * kk[c];
+            denom += exp(dot * inv_sqrt_d - mx);
+        }
+        lse[e] = mx + log(denom);
+    }
+    /* then every key's mean probability over the rows, rows in index order */
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t j = 0; j < n_k; ++j) {
+        double s = 0.0;
+        for (int64_t e = 0; e < total; ++e) {
+            int g = (int)(e % n_q_heads) / G;
+            const double *qq = rq + (size_t)e * d;
+            const double *kk = rk + ((size_t)j * n_kv_heads + g) * d;
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += qq[c] * kk[c];
+            s += exp(dot * inv_sqrt_d - lse[e]);
+        }
+        mass[j] = s / (double)total;
+    }
+    free(rq);
+    free(lse);
+    free(rk);
+    return PO_OK;
+}

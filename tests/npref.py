@@ -55,3 +55,8 @@ def attend_np(q, q_pos, k, v, k_pos, base=10000.0, mask=None):
 def score_np(k, k_pos, q, q_pos, base=10000.0):
     """Mean scaled logit of each key over all queries and query heads."""
     return logits_np(q, q_pos, k, k_pos, base).mean(axis=(0, 1))
+
+
+def attend_mass_np(q, q_pos, k, k_pos, base=10000.0):
+    """Mean softmax probability each key receives over all (query, head) rows."""
+    return softmax(logits_np(q, q_pos, k, k_pos, base), axis=-1).mean(axis=(0, 1))

@@ -430,3 +430,55 @@ def test_plan_minimum_quota_properties():
     assert u[0] == 2 and u[-1] == 64 and sum(u) == 100 and all(x >= 5 for x in u[1:-1])
     with pytest.raises(oracle.OracleError):
         oracle.plan_budget(oracle.LINEAR, 0.0, 10, 0, [5], min_quota=-1)
+
+
+# ---------------------------------------------------------------------------------------------- attention mass (Sec. 3.4)
+def test_attend_mass_matches_library_softmax():
+    L = _tiny_layer(seed=4)
+    k = np.concatenate([L.anchor_k, L.hist_k[:90]])
+    p = np.concatenate([L.anchor_pos, L.hist_pos[:90]])
+    got = oracle.attend_mass(L.q, L.q_pos, [(L.anchor_k, L.anchor_pos), (L.hist_k[:90], L.hist_pos[:90])])
+    np.testing.assert_allclose(got, npref.attend_mass_np(L.q, L.q_pos, k, p), rtol=0, atol=1e-14)
+    assert abs(got.sum() - 1.0) < 1e-12                          # every row's probabilities sum to one
+
+
+def test_attend_mass_is_the_mean_attention_row_read_through_one_hot_values():
+    # With v_j = e_j the attention output (pinned on its own above) is the probability row itself, so the mass is its
+    # mean over queries and heads: a wrong head-to-group map or normaliser in either function breaks the equality.
+    L = _tiny_layer(seed=5)
+    n, d = 40, L.q.shape[2]
+    k, p = L.hist_k[:n], L.hist_pos[:n]
+    v = np.zeros((n, k.shape[1], d), np.float32)
+    v[np.arange(n), :, np.arange(n)] = 1.0
+    rows = oracle.attend(L.q, L.q_pos, [(k, v, p)])               # [n_q][Hq][d]: entry j = P(row, key j)
+    np.testing.assert_allclose(oracle.attend_mass(L.q, L.q_pos, [(k, p)]), rows[:, :, :n].mean(axis=(0, 1)), rtol=0, atol=1e-14)
+
+
+def test_attend_mass_closed_forms():
+    L = _tiny_layer(seed=6)
+    hkv, d = L.hist_k.shape[1], L.hist_k.shape[2]
+    # identical keys at one position: every key gets 1/n
+    k = np.broadcast_to(L.hist_k[:1], (25, hkv, d)).copy()
+    p = np.broadcast_to(L.hist_pos[:1], (25, 4)).copy()
+    np.testing.assert_allclose(oracle.attend_mass(L.q, L.q_pos, [(k, p)]), 1.0 / 25, rtol=0, atol=1e-15)
+    # two keys, one query, one head, no rotation: the logistic function of the logit difference
+    rng = np.random.default_rng(3)
+    q1 = rng.standard_normal((1, 1, d)).astype(np.float32)
+    k2 = rng.standard_normal((2, 1, d)).astype(np.float32)
+    z = np.zeros((2, 4), np.int32)
+    diff = float((q1[0, 0].astype(np.float64) @ (k2[0, 0].astype(np.float64) - k2[1, 0].astype(np.float64))) / np.sqrt(d))
+    got = oracle.attend_mass(q1, z[:1], [(k2, z)])
+    np.testing.assert_allclose(got, [1 / (1 + np.exp(-diff)), 1 / (1 + np.exp(diff))], rtol=0, atol=1e-15)
+    # a key that every query matches far better than the rest takes nearly all of the mass
+    kk = (0.01 * rng.standard_normal((30, hkv, d))).astype(np.float32)
+    qq = np.ones_like(L.q)
+    kk[7] = 4.0
+    zp = np.zeros((30, 4), np.int32)
+    m = oracle.attend_mass(qq, np.zeros_like(L.q_pos), [(kk, zp)])
+    assert m.argmax() == 7 and m[7] > 0.999
+    # the split into segments and the key order do not matter
+    perm = rng.permutation(60)
+    a = oracle.attend_mass(L.q, L.q_pos, [(L.hist_k[:60], L.hist_pos[:60])])
+    b = oracle.attend_mass(L.q, L.q_pos, [(L.hist_k[:60][perm][:20], L.hist_pos[:60][perm][:20]),
+                                          (L.hist_k[:60][perm][20:], L.hist_pos[:60][perm][20:])])
+    np.testing.assert_allclose(a[perm], b, rtol=0, atol=1e-14)
