@@ -173,6 +173,22 @@ pc_status pc_attend_prepare(pc_ctx *ctx, const pc_cache *cache, const pc_segment
 pc_status pc_attend_prepared(pc_ctx *ctx, const void *q, const int32_t *q_pos, int32_t n_q, void *out, float *lse,
                              void *stream);
 
+/* Attention mass of every key (Sec. 3.4: retention is guided by the attention a cached token receives):
+ *   mass_j = 1/(n_q*Hq) * sum over the query rows (i, h) of softmax_j((R q_ih).(R k_j,g(h))/sqrt(d)),
+ * the mean, over the frame's queries and heads, of the probabilities of Eq. 2; the masses of all keys sum to one.
+ * It is computed for the key set and the queries of the most recent pc_attend_frame / pc_attend_prepared call on this
+ * context, whose rotated keys and queries are still in the context's scratch: call it after that call, ordered behind
+ * it on the GPU, with the lse that call wrote, and before any other attention call on the context.
+ *   lse device [n_q][Hq] fp32 (as written by the attention call); n_keys = all keys of that call;
+ *   mass device out [n_keys] fp32 in key order anchors ++ history ++ current.
+ * mass + (number of anchor tokens), i.e. the masses of history ++ current, can be passed as scores_override to
+ * pc_score or — once the current frame has been appended, and past the tokens of any frame the window is about to
+ * drop — to pc_window_update, which then ranks by attention mass instead of by the mean logit.
+ * bf16 tensor-core path only.  Errors: PC_ERR_UNSUPPORTED (fp32 context, head_dim != 128, CUDA-core kernel chosen),
+ * PC_ERR_INVALID_ARG (null or misaligned pointer, no such attention call precedes, n_keys differs from that call's),
+ * PC_ERR_CUDA. */
+pc_status pc_attend_mass(pc_ctx *ctx, const float *lse, float *mass, int32_t n_keys, void *stream);
+
 /* One frame step with inputs and output in HOST memory (pinned memory keeps the copies asynchronous): copies Q,
  * positions, anchors and the history frames into the caller's device workspace, plans the budget, scores, selects,
  * packs and attends (anchors ++ packed history), copies the output back and waits for the stream.  Everything the
@@ -310,7 +326,7 @@ pc_status pc_set_cluster_merge(pc_ctx *ctx, int32_t on);
  * writes the duration in milliseconds of each kernel of the most recent calls, -1 for a kernel that did not run.
  * ms is a host array [PC_N_STAGES]. */
 enum { PC_STAGE_QPOOL = 0, PC_STAGE_SCORE = 1, PC_STAGE_SELECT = 2, PC_STAGE_PACK = 3, PC_STAGE_ROPE = 4,
-       PC_STAGE_ATTEND = 5, PC_STAGE_COMBINE = 6, PC_N_STAGES = 7 };
+       PC_STAGE_ATTEND = 5, PC_STAGE_COMBINE = 6, PC_STAGE_MASS = 7, PC_N_STAGES = 8 };
 pc_status pc_set_timing(pc_ctx *ctx, int32_t on);
 pc_status pc_get_timing(pc_ctx *ctx, float *ms);
 

@@ -25,7 +25,7 @@ EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact"
            "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_set_timing", "pc_get_timing",
            "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge",
            "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_append_masked", "pc_window_update", "pc_window_cache",
-           "pc_window_state", "pc_attend_prepare", "pc_attend_prepared"]
+           "pc_window_state", "pc_attend_prepare", "pc_attend_prepared", "pc_attend_mass"]
 
 
 class pc_layer_desc(C.Structure):
@@ -64,7 +64,7 @@ class pc_device_workspace(C.Structure):
                 ("sel_idx", C.c_void_p), ("out", C.c_void_p)]
 
 
-STAGES = ["qpool", "score", "select", "pack", "rope", "attend", "combine"]
+STAGES = ["qpool", "score", "select", "pack", "rope", "attend", "combine", "mass"]
 
 
 class PackCacheError(RuntimeError):
@@ -109,6 +109,7 @@ def load() -> C.CDLL:
                                            C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.pc_attend_prepare.argtypes = [C.c_void_p, C.POINTER(pc_cache), C.POINTER(pc_segment), C.c_void_p]
     lib.pc_attend_prepared.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.pc_attend_mass.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
     lib.pc_window_create.argtypes = [C.c_void_p, C.POINTER(pc_window_params), C.POINTER(pc_segment), C.POINTER(pc_segment),
                                      C.POINTER(pc_segment), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p)]
     lib.pc_window_destroy.argtypes = [C.c_void_p]
@@ -270,6 +271,14 @@ def pc_attend_prepared(ctx: Context, q: torch.Tensor, q_pos: torch.Tensor, out: 
     _check(load().pc_attend_prepared(ctx.handle, _ptr(q), _ptr(q_pos), q.shape[0], _ptr(out), _ptr(lse), _stream(stream)),
            "pc_attend_prepared")
     return (out, lse) if want_lse else out
+
+
+def pc_attend_mass(ctx: Context, lse: torch.Tensor, n_keys: int, mass: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Attention mass of every key of the most recent attention call on ctx (lse = what that call wrote)."""
+    if mass is None:
+        mass = torch.empty(n_keys, dtype=torch.float32, device=lse.device)
+    _check(load().pc_attend_mass(ctx.handle, _ptr(lse), _ptr(mass), n_keys, _stream(stream)), "pc_attend_mass")
+    return mass
 
 
 def pc_poll_status(ctx: Context, stream=None) -> int:

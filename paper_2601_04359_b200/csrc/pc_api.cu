@@ -53,6 +53,7 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
     c->kv_splits = 0;
     c->cluster_merge = 0;
     c->prepared_n_seg = 0;
+    c->last_n_q = c->last_n_seg = 0;
     c->timing_on = 0;
     c->ev_mask = 0;
     for (int i = 0; i < PC_N_MARKS; ++i) c->ev[i] = nullptr;
@@ -96,6 +97,8 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
         PC_CUDA_TRY(cudaMalloc(&c->q_rot, (size_t)desc->max_q * desc->n_q_heads * desc->head_dim * sizeof(__nv_bfloat16)));
         PC_CUDA_TRY(cudaMalloc(&c->part_o, std::max<size_t>(c->part_o_floats, 1) * sizeof(float)));
         PC_CUDA_TRY(cudaMalloc(&c->part_ml, std::max<size_t>(c->part_ml_floats, 1) * sizeof(float)));
+        PC_CUDA_TRY(cudaMalloc(&c->mass_part, c->k_rot_rows * desc->n_kv_heads * 2 * sizeof(float)));
+        PC_CUDA_TRY(cudaMalloc(&c->mass_norm, (size_t)((desc->max_q + 127) / 128) * 128 * desc->n_q_heads * sizeof(float)));
     }
     *out = c;
     return PC_OK;
@@ -114,6 +117,8 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
     cudaFree(c->q_rot);
     cudaFree(c->part_o);
     cudaFree(c->part_ml);
+    cudaFree(c->mass_part);
+    cudaFree(c->mass_norm);
     delete c;
     return PC_OK;
 }
@@ -151,7 +156,7 @@ extern "C" pc_status pc_get_timing(pc_ctx *c, float *ms) {
     static const int span[PC_N_STAGES][2] = {{PC_MARK_SCORE0, PC_MARK_QPOOL}, {PC_MARK_QPOOL, PC_MARK_SCORE},
                                              {PC_MARK_SCORE, PC_MARK_SELECT}, {PC_MARK_PACK0, PC_MARK_PACK},
                                              {PC_MARK_ATT0, PC_MARK_ROPE},    {PC_MARK_ROPE, PC_MARK_ATTEND},
-                                             {PC_MARK_ATTEND, PC_MARK_COMBINE}};
+                                             {PC_MARK_ATTEND, PC_MARK_COMBINE}, {PC_MARK_MASS0, PC_MARK_MASS}};
     for (int s = 0; s < PC_N_STAGES; ++s) {
         ms[s] = -1.f;
         const int a = span[s][0], b = span[s][1];

@@ -44,6 +44,7 @@ extern "C" pc_status pc_attend_frame(pc_ctx *ctx, const pc_cache *cache, const p
     int n_seg = 0;
     st = gather_segments(ctx, cache, current, segs, &n_seg);
     if (st != PC_OK) return st;
+    ctx->last_n_q = 0;
     if (tensor_core_path(ctx)) {
         ctx->prepared_n_seg = 0;                       // the rotated-key scratch is about to be overwritten
         return pc_launch_attend_tc(ctx, n_seg, segs, q, q_pos, n_q, out, lse, stream, PC_TC_ALL);
@@ -59,6 +60,7 @@ extern "C" pc_status pc_attend_prepare(pc_ctx *ctx, const pc_cache *cache, const
     pc_status st = gather_segments(ctx, cache, current, segs, &n_seg);
     if (st != PC_OK) return st;
     ctx->prepared_n_seg = 0;
+    ctx->last_n_q = 0;
     if (tensor_core_path(ctx)) {
         st = pc_launch_attend_tc(ctx, n_seg, segs, nullptr, nullptr, 0, nullptr, nullptr, stream, PC_TC_ROPE_K);
         if (st != PC_OK) return st;
@@ -75,6 +77,7 @@ extern "C" pc_status pc_attend_prepared(pc_ctx *ctx, const void *q, const int32_
     pc_status st = check_queries(ctx, q, q_pos, n_q, out, lse);
     if (st != PC_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    ctx->last_n_q = 0;
     if (tensor_core_path(ctx))
         return pc_launch_attend_tc(ctx, ctx->prepared_n_seg, ctx->prepared_seg, q, q_pos, n_q, out, lse, stream,
                                    PC_TC_ROPE_Q | PC_TC_ATTEND);

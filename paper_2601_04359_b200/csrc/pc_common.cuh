@@ -28,11 +28,13 @@ enum {
     PC_WHERE_ROPE_POS = 7,
     PC_WHERE_SCORE_WAIT = 8,
     PC_WHERE_MASK_COUNT = 9,
+    PC_WHERE_MASS_WAIT = 10,
 };
 
-// event marks: score call 0-3, pack 4-5, attend 6-9
+// event marks: score call 0-3, pack 4-5, attend 6-9, attention mass 10-11
 enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT = 3, PC_MARK_PACK0 = 4, PC_MARK_PACK = 5,
-       PC_MARK_ATT0 = 6, PC_MARK_ROPE = 7, PC_MARK_ATTEND = 8, PC_MARK_COMBINE = 9, PC_N_MARKS = 10 };
+       PC_MARK_ATT0 = 6, PC_MARK_ROPE = 7, PC_MARK_ATTEND = 8, PC_MARK_COMBINE = 9, PC_MARK_MASS0 = 10, PC_MARK_MASS = 11,
+       PC_N_MARKS = 12 };
 
 constexpr int PC_QPOOL_BLOCKS = 128;
 constexpr int PC_MAX_SEGMENTS = 3;
@@ -69,6 +71,12 @@ struct pc_ctx {
     // key set fixed by pc_attend_prepare (its rotated keys sit in k_rot until the next prepare or pc_attend_frame)
     int prepared_n_seg;        // 0 = nothing prepared
     pc_segment prepared_seg[PC_MAX_SEGMENTS];
+    // shape of the most recent tensor-core attention call, whose rotated keys and queries are still in k_rot / q_rot
+    // (read by pc_attend_mass); last_n_q = 0 when there is none
+    int last_n_q, last_n_seg;
+    int last_seg_n[PC_MAX_SEGMENTS];
+    float *mass_part;          // attention mass: partial sums per KV head and column half, [Hkv][2][k_rot_rows]
+    float *mass_norm;          // attention mass: negated base-2 normalisers, [Hq][max_q rounded up to 128]
     // optional per-kernel timing (benchmarks): events at the boundaries of the kernels of each call
     int timing_on;
     unsigned ev_mask;

@@ -1,0 +1,179 @@
+"""Attention mass (Sec. 3.4: retention guided by the attention a cached token receives), GPU against the oracle.
+
+mass_j is the mean over the frame's query rows and heads of the softmax probability of key j.  The tensor-core path
+rounds the rotated queries and keys to bf16 before the product, so a logit moves by about 2^-9 relative per operand;
+the masses, averages over thousands of rows, were seen to move by 5e-4 relative at most.  The bound checked here is
+1e-2 relative plus 1e-3 of the uniform mass 1/n_keys; the masses of all keys must sum to one within 1e-4."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import window as ow
+from paper_2601_04359_b200 import binding as pc
+from paper_2601_04359_b200 import workload as wl
+from paper_2601_04359_b200.device import DeviceLayer, dev, host, idev, make_ctx, segment
+
+pytestmark = pytest.mark.gpu
+
+MASS_RTOL = 1e-2
+
+
+def _check_mass(got: np.ndarray, want: np.ndarray):
+    n = len(want)
+    assert got.shape == want.shape
+    assert abs(float(got.sum(dtype=np.float64)) - 1.0) <= 1e-4
+    assert (np.abs(got - want) <= MASS_RTOL * want + 1e-3 / n).all()
+
+
+def _segments(L, with_current):
+    segs = [(L.anchor_k, L.anchor_pos), (L.hist_k, L.hist_pos)]
+    if with_current:
+        segs.append((L.cur_k, L.q_pos))
+    return [s for s in segs if len(s[0])]
+
+
+@pytest.mark.parametrize("with_current", [False, True])
+@pytest.mark.parametrize("splits", [0, 1, 3])
+def test_mass_matches_oracle_on_ragged_segments(with_current, splits):
+    """Anchors, history and current frame of lengths that are no multiple of the 128-key tile, an odd number of key
+    tiles, a last query tile of 124 rows; the key ranges of the attention call split one, three or an automatic number
+    of ways (the mass only depends on the normalisers that call wrote)."""
+    cfg = wl.small_bf16(n_frames=4, grid=(12, 21), n_text=130, total=700, keep_full=1, seed=11)
+    L = wl.make_layer(cfg, with_current=True)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    pc.pc_set_kv_splits(ctx, splits)
+    _, lse = pc.pc_attend_frame(ctx, D.cache, D.current if with_current else None, D.q, D.q_pos, want_lse=True)
+    segs = _segments(L, with_current)
+    n_keys = sum(len(s[0]) for s in segs)
+    mass = pc.pc_attend_mass(ctx, lse, n_keys)
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+    _check_mass(host(mass).astype(np.float64), oracle.attend_mass(L.q, L.q_pos, segs, cfg.rope_base))
+    ctx.close()
+
+
+def test_mass_of_peaked_attention():
+    """Queries scaled up so that rows concentrate on few keys: the masses spread over most of a decade."""
+    cfg = wl.small_bf16(n_frames=3, grid=(11, 13), n_text=130, total=260, seed=5)
+    L = wl.make_layer(cfg, with_current=True)
+    L.q = wl.to_storage(4.0 * L.q, cfg.dtype)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    _, lse = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos, want_lse=True)
+    segs = _segments(L, True)
+    n_keys = sum(len(s[0]) for s in segs)
+    got = host(pc.pc_attend_mass(ctx, lse, n_keys)).astype(np.float64)
+    want = oracle.attend_mass(L.q, L.q_pos, segs, cfg.rope_base)
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+    assert want.max() / want.min() > 5
+    _check_mass(got, want)
+    ctx.close()
+
+
+def test_mass_after_prepared_attention_and_errors():
+    cfg = wl.small_bf16(n_frames=3, grid=(11, 13), n_text=130, total=260, seed=4)
+    L = wl.make_layer(cfg, with_current=True)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    segs = _segments(L, True)
+    n_keys = sum(len(s[0]) for s in segs)
+    lse = torch.zeros(cfg.n_q, cfg.n_q_heads, device="cuda")
+    with pytest.raises(pc.PackCacheError) as e:                    # no attention call precedes
+        pc.pc_attend_mass(ctx, lse, n_keys)
+    assert e.value.status == pc.PC_ERR_INVALID_ARG
+    _, lse = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos, want_lse=True)
+    with pytest.raises(pc.PackCacheError) as e:                    # key count of another call
+        pc.pc_attend_mass(ctx, lse, n_keys - 1)
+    assert e.value.status == pc.PC_ERR_INVALID_ARG
+    a = pc.pc_attend_mass(ctx, lse, n_keys).clone()
+    # the two-part form leaves the same rotated operands behind: the same bits come out
+    pc.pc_attend_prepare(ctx, D.cache, D.current)
+    with pytest.raises(pc.PackCacheError):                         # keys rotated, but no queries yet
+        pc.pc_attend_mass(ctx, lse, n_keys)
+    _, lse2 = pc.pc_attend_prepared(ctx, D.q, D.q_pos, want_lse=True)
+    b = pc.pc_attend_mass(ctx, lse2, n_keys)
+    assert torch.equal(lse, lse2) and torch.equal(a, b)
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+    _check_mass(host(a).astype(np.float64), oracle.attend_mass(L.q, L.q_pos, segs, cfg.rope_base))
+    # the CUDA-core kernel and fp32 contexts have no mass path
+    pc.pc_set_attend_impl(ctx, 1)
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_attend_mass(ctx, lse, n_keys)
+    assert e.value.status == pc.PC_ERR_UNSUPPORTED
+    ctx.close()
+    tiny = wl.CONFIGS["tiny"]
+    Lt = wl.make_layer(tiny)
+    Dt = DeviceLayer(Lt)
+    ctx = make_ctx(tiny)
+    _, lse = pc.pc_attend_frame(ctx, Dt.cache, None, Dt.q, Dt.q_pos, want_lse=True)
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_attend_mass(ctx, lse, tiny.n_anchor + tiny.n_src)
+    assert e.value.status == pc.PC_ERR_UNSUPPORTED
+    ctx.close()
+
+
+def test_mass_full_size():
+    """The 12-frame configuration at full size against the oracle, key by key."""
+    cfg = wl.CONFIGS["lumos12"]
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    _, lse = pc.pc_attend_frame(ctx, D.cache, None, D.q, D.q_pos, want_lse=True)
+    segs = _segments(L, False)
+    n_keys = sum(len(s[0]) for s in segs)
+    got = host(pc.pc_attend_mass(ctx, lse, n_keys)).astype(np.float64)
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+    _check_mass(got, oracle.attend_mass(L.q, L.q_pos, segs, cfg.rope_base))
+    ctx.close()
+
+
+def test_window_selection_guided_by_attention_mass():
+    """The cache window re-selected by attention mass instead of by the mean logit: every frame attends to
+    anchors ++ window ++ itself, the masses of that call (history ++ current part) rank the tokens once the frame has
+    been appended.  Masses are checked against the oracle's; selection, packed rows and positions must then match the
+    reference window bit for bit when it ranks on the same fp32 masses."""
+    cfg = wl.small_bf16(n_frames=7, grid=(12, 21), n_text=128, total=600, kind=wl.HALFLIFE, param=2.0, keep_full=1, seed=21)
+    n, W, total = cfg.frame_tokens, 3, 600
+    assert n % 4 == 0 and cfg.n_anchor % 4 == 0                     # score pointers handed to the window stay 16-byte aligned
+    L = wl.make_layer(cfg)
+    rng = np.random.Generator(np.random.Philox(key=[21, 5]))
+    st = lambda x: wl.to_storage(x.astype(np.float32), cfg.dtype)
+    ctx = make_ctx(cfg, max_keys=cfg.n_anchor + total + 3 * n)
+    cap = total + 2 * n
+    mk = lambda: pc.Segment(torch.zeros((cap, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((cap, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((cap, 4), dtype=torch.int32, device="cuda"), 0)
+    win = pc.Window(ctx, W, pc.PC_HALFLIFE, 2.0, total, 1, segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype), mk(), mk())
+    ref = ow.WindowRef(W, oracle.HALFLIFE, 2.0, total, 1)
+    regimes = []
+    for f in range(1, 7):
+        pos = wl.frame_positions(cfg, f, cfg.n_anchor + (f - 1) * n)
+        k, v = st(rng.standard_normal((n, cfg.n_kv_heads, cfg.head_dim))), st(rng.standard_normal((n, cfg.n_kv_heads, cfg.head_dim)))
+        q = st(2.0 * rng.standard_normal((n, cfg.n_q_heads, cfg.head_dim)))
+        cur = segment(k, v, pos, cfg.dtype)
+        _, lse = pc.pc_attend_frame(ctx, win.cache(), cur, dev(q, cfg.dtype), idev(pos), want_lse=True)
+        n_hist = 0 if ref.k is None else len(ref.k)
+        n_keys = cfg.n_anchor + n_hist + n
+        mass = pc.pc_attend_mass(ctx, lse, n_keys)
+        segs = [(L.anchor_k, L.anchor_pos)] + ([(ref.k, ref.pos)] if n_hist else []) + [(k, pos)]
+        _check_mass(host(mass).astype(np.float64), oracle.attend_mass(q, pos, segs, cfg.rope_base))
+        # the finished frame joins the history; the masses of history ++ frame rank what stays
+        ref.append(k, v, pos)
+        win.append(cur)
+        dropped = len(ref.k) - len(ref.source_after_drop()[0])
+        guide = mass[cfg.n_anchor + dropped:]
+        want = ref.update(None, None, scores32=host(guide))
+        got = win.update(None, None, scores_override=guide)
+        assert got == want and pc.pc_poll_status(ctx) == pc.PC_OK
+        regimes.append(got)
+        counts, _, _ = win.state()
+        assert counts.tolist() == ref.count
+        cache = win.cache()
+        m = int(counts.sum())
+        assert np.array_equal(host(cache.history.k)[:m], ref.k) and np.array_equal(host(cache.history.v)[:m], ref.v)
+        assert np.array_equal(cache.history.pos.cpu().numpy()[:m], ref.pos)
+    assert pc.PC_WINDOW_PACK in regimes and pc.PC_WINDOW_SLIDE in regimes
+    win.close(); ctx.close()
