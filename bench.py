@@ -281,6 +281,28 @@ def run_cuda(args):
         pass_ms = max_over_ranks(e0.elapsed_time(e1) / n_pass, dist, "cuda")
         assert pc.pc_poll_status(ctx) == pc.PC_OK
 
+    # ---- attention mass of every key of the packed cache (the score that attention-guided retention ranks by), computed
+    # once per frame after the frame's last attention pass, from the rotated operands and normalisers that pass left behind
+    mass_ms = None
+    if not args.no_extra_pass:
+        n_keys = cfg.n_anchor + n_sel
+        lse = torch.empty(cfg.n_q, cfg.n_q_heads, dtype=torch.float32, device="cuda")
+        mass = torch.empty(n_keys, dtype=torch.float32, device="cuda")
+        n_mass = min(args.steps, 100)
+        es = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_mass)]
+        for i in range(-3, n_mass):
+            pc.pc_attend_frame(ctx, dsts[i % N_LAYERS], None, layers[i % N_LAYERS].q, layers[i % N_LAYERS].q_pos, out=out, lse=lse,
+                               stream=stream)
+            if i >= 0:
+                es[i][0].record(stream)
+            pc.pc_attend_mass(ctx, lse, n_keys, mass=mass, stream=stream)
+            if i >= 0:
+                es[i][1].record(stream)
+        barrier()
+        mass_ms = max_over_ranks(float(np.mean([a.elapsed_time(b_) for a, b_ in es])), dist, "cuda")
+        assert pc.pc_poll_status(ctx) == pc.PC_OK
+        assert abs(float(mass.sum()) - 1.0) < 1e-3
+
     # ---- the same frame step in the Slide regime of the cache window (incremental re-selection: the source of each pack is
     # what the last pack kept plus the newest frame, about 9 k tokens instead of the whole 47-frame history)
     N = cfg.frame_tokens
@@ -396,6 +418,9 @@ def run_cuda(args):
         "kernels_ms": stages,
         "extra_pass": {"ms_per_pass": pass_ms, "what": "one more attention pass of the frame over the unchanged packed cache "
                        "(pc_attend_prepared: query rotation, attention, merge; keys were rotated once per frame)"},
+        "attention_mass": {"ms": mass_ms, "keys": cfg.n_anchor + n_sel,
+                           "what": "pc_attend_mass after an attention pass over the packed cache: K Q^T on tensor cores, "
+                                   "column sums of the normalised probabilities (three launches)"},
         "incremental": {"ms_per_frame": job_ms_per_frame(inc_ms, world) if inc_ms else None, "source_tokens": inc_src,
                         "mode": "cache window in the Slide regime: append the newest frame, drop the oldest, re-plan, "
                                 "score and re-select from packed + new, pack, attend (same keys attended)"},
