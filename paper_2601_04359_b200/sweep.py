@@ -100,17 +100,26 @@ def main():
         dsts = [x.empty_packed(2 * N + 6048) for x in stack]
         avail = np.full(cfg.n_frames, N, np.int32)
 
-        def frame():
+        def frame(st):
             for x, d in zip(stack, dsts):
                 budget = pc.pc_plan_budget(pc.PC_HALFLIFE, 4.0, 2 * N + 6048, 2, avail)
-                pc.pc_score(ctx, x.cache, x.q, x.q_pos, budget, scores=scores, sel_idx=sel, stream=stream)
-                pc.pc_compact(ctx, x.cache, sel, budget, 0, d, stream=stream)
-                pc.pc_attend_frame(ctx, d, None, x.q, x.q_pos, out=out, stream=stream)
+                pc.pc_score(ctx, x.cache, x.q, x.q_pos, budget, scores=scores, sel_idx=sel, stream=st)
+                pc.pc_compact(ctx, x.cache, sel, budget, 0, d, stream=st)
+                pc.pc_attend_frame(ctx, d, None, x.q, x.q_pos, out=out, stream=st)
 
-        t = _time(frame, max(3, args.reps // 4), stream)
+        reps = max(3, args.reps // 4)
+        t = _time(lambda: frame(stream), reps, stream)
+        assert pc.pc_poll_status(ctx) == pc.PC_OK
+        # the same frame captured once into a CUDA graph (8 kernels x layers, programmatic dependencies kept as graph
+        # edges) and replayed: the host's planning and launch work leaves the critical path
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            frame(torch.cuda.current_stream())
+        tg = _time(graph.replay, reps, torch.cuda.current_stream())
         assert pc.pc_poll_status(ctx) == pc.PC_OK
         print(json.dumps({"stack_layers": args.stack, "history_frames": cfg.n_frames, "ms_per_frame": round(t, 3),
-                          "ms_per_layer": round(t / args.stack, 4)}), flush=True)
+                          "ms_per_layer": round(t / args.stack, 4), "ms_per_frame_cuda_graph": round(tg, 3),
+                          "ms_per_layer_cuda_graph": round(tg / args.stack, 4)}), flush=True)
     late = [r for r in rows if r["history_frames"] >= 44]
     print(json.dumps({"summary": "last four frames (44-47 history frames), one layer",
                       "ms_full": round(sum(r["ms_full"] for r in late), 4), "ms_packcache": round(sum(r["ms_packcache"] for r in late), 4),

@@ -206,6 +206,67 @@ def test_prepared_attention_equals_attend_frame_over_several_passes(cfg_name):
     ctx.close()
 
 
+# ------------------------------------------------------------------------------------------- CUDA graph
+def test_frame_step_replays_from_a_cuda_graph():
+    """Three layers' frame steps (score, select, pack, attend: eight kernels each, launched with programmatic
+    dependencies) captured once into a CUDA graph.  A replay must give the bits of the eager calls, also after the
+    inputs were overwritten in place (a new frame's queries and history in the same buffers)."""
+    cfgs = [wl.small_bf16(n_frames=4, grid=(12, 21), n_text=130, total=500, keep_full=1, seed=30 + i) for i in range(3)]
+    Ls = [wl.make_layer(c) for c in cfgs]
+    Ds = [DeviceLayer(L) for L in Ls]
+    cfg = cfgs[0]
+    ctx = make_ctx(cfg)
+    budget = _plan(cfg)
+    n_sel = int(budget.sum())
+    scores = torch.empty(cfg.n_src, dtype=torch.float32, device="cuda")
+    sel = torch.empty(n_sel, dtype=torch.int32, device="cuda")
+    dsts = [D.empty_packed(n_sel) for D in Ds]
+    outs = [torch.empty_like(D.q) for D in Ds]
+
+    def frame(stream):
+        for D, dst, out in zip(Ds, dsts, outs):
+            pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget, scores=scores, sel_idx=sel, stream=stream)
+            pc.pc_compact(ctx, D.cache, sel, budget, 0, dst, stream=stream)
+            pc.pc_attend_frame(ctx, dst, None, D.q, D.q_pos, out=out, stream=stream)
+
+    frame(torch.cuda.current_stream())                              # warm-up: one-time attribute and occupancy queries
+    torch.cuda.synchronize()
+    eager = [o.clone() for o in outs]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        frame(torch.cuda.current_stream())
+    for o in outs:
+        o.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    _ok(ctx)
+    for o, e in zip(outs, eager):
+        assert torch.equal(o, e)
+    want = oracle.attend(Ls[1].q, Ls[1].q_pos, [(Ls[1].anchor_k, Ls[1].anchor_v, Ls[1].anchor_pos),
+                                                tuple(host(t) if t.dtype != torch.int32 else t.cpu().numpy()
+                                                      for t in (dsts[1].history.k[:n_sel], dsts[1].history.v[:n_sel], dsts[1].history.pos[:n_sel]))],
+                         cfg.rope_base)
+    assert np.abs(host(outs[1]).astype(np.float64) - want).max() <= BF16_ATOL
+    # new contents in the same buffers: layers swap their queries and history
+    for a, b in ((0, 1), (1, 2)):
+        for name in ("q",):
+            ta, tb = getattr(Ds[a], name), getattr(Ds[b], name)
+            tmp = ta.clone(); ta.copy_(tb); tb.copy_(tmp)
+        ha, hb = Ds[a].cache.history, Ds[b].cache.history
+        for ta, tb in ((ha.k, hb.k), (ha.v, hb.v)):
+            tmp = ta.clone(); ta.copy_(tb); tb.copy_(tmp)
+    graph.replay()
+    torch.cuda.synchronize()
+    replayed = [o.clone() for o in outs]
+    frame(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    _ok(ctx)
+    for o, e in zip(outs, replayed):
+        assert torch.equal(o, e)
+    assert not torch.equal(replayed[0], eager[0])
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------------- select
 def _select_case(frame_count, budget, scores, cfg=None):
     cfg = cfg or wl.CONFIGS["tiny"]
