@@ -156,8 +156,8 @@ pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, c
  * Rotary embedding is applied from the stored positions inside the call.
  *   current may be NULL; q device [n_q][Hq][d]; out device [n_q][Hq][d];
  *   lse device [n_q][Hq] fp32 natural-log sum of exponentials, or NULL.
- * bf16 runs on tcgen05 tensor cores (fp32 accumulate and softmax); fp32 runs on
- * CUDA cores.  Errors: PC_ERR_INVALID_ARG, PC_ERR_CAPACITY (keys > max_keys,
+ * bf16 with head_dim 128 runs on tcgen05 tensor cores (fp32 accumulate and softmax) when Hkv*d and Hq*d are
+ * multiples of 256; everything else runs on CUDA cores.  Errors: PC_ERR_INVALID_ARG, PC_ERR_CAPACITY (keys > max_keys,
  * n_q > max_q), PC_ERR_CUDA. */
 pc_status pc_attend_frame(pc_ctx *ctx, const pc_cache *cache, const pc_segment *current, const void *q,
                           const int32_t *q_pos, int32_t n_q, void *out, float *lse, void *stream);
@@ -184,7 +184,8 @@ pc_status pc_attend_prepared(pc_ctx *ctx, const void *q, const int32_t *q_pos, i
  * mass + (number of anchor tokens), i.e. the masses of history ++ current, can be passed as scores_override to
  * pc_score or — once the current frame has been appended, and past the tokens of any frame the window is about to
  * drop — to pc_window_update, which then ranks by attention mass instead of by the mean logit.
- * bf16 tensor-core path only.  Errors: PC_ERR_UNSUPPORTED (fp32 context, head_dim != 128, CUDA-core kernel chosen),
+ * bf16 tensor-core path only.  Errors: PC_ERR_UNSUPPORTED (fp32 context, head_dim != 128, Hkv*d or Hq*d not a
+ * multiple of 256, CUDA-core kernel chosen),
  * PC_ERR_INVALID_ARG (null or misaligned pointer, no such attention call precedes, n_keys differs from that call's),
  * PC_ERR_CUDA. */
 pc_status pc_attend_mass(pc_ctx *ctx, const float *lse, float *mass, int32_t n_keys, void *stream);

@@ -209,6 +209,13 @@ inline void pc_mark(pc_ctx *c, int idx, cudaStream_t s) {
     if (c->timing_on && c->ev[idx] && cudaEventRecord(c->ev[idx], s) == cudaSuccess) c->ev_mask |= 1u << idx;
 }
 
+// Shapes the tensor-core kernels take: bf16, head_dim 128, and K / Q rows that are whole 256-element granules of the
+// rotary pre-pass (a warp rotates 32 x 8 elements at a time).  Everything else runs on the CUDA-core kernel.
+inline bool pc_tensor_core_shape(const pc_ctx *ctx) {
+    const pc_layer_desc &d = ctx->desc;
+    return d.dtype == PC_BF16 && d.head_dim == 128 && (d.n_kv_heads * d.head_dim) % 256 == 0 && (d.n_q_heads * d.head_dim) % 256 == 0;
+}
+
 // host-side helpers implemented in pc_api.cu
 bool pc_aligned16(const void *p);
 pc_status pc_check_segment(const pc_segment *s, bool allow_empty);

@@ -177,3 +177,35 @@ def test_window_selection_guided_by_attention_mass():
         assert np.array_equal(cache.history.pos.cpu().numpy()[:m], ref.pos)
     assert pc.PC_WINDOW_PACK in regimes and pc.PC_WINDOW_SLIDE in regimes
     win.close(); ctx.close()
+
+
+@pytest.mark.parametrize("hq,hkv,grid,n_text", [(8, 8, (5, 9), 11),        # no grouping, fewer keys and queries than one tile
+                                                (16, 4, (10, 13), 40),     # four query heads per KV head, ragged everywhere
+                                                (2, 1, (16, 16), 0),       # one KV head, two whole query tiles, no text
+                                                (6, 2, (3, 43), 129)])     # 129 query rows: a second tile with one row
+def test_attention_and_mass_over_head_groupings_and_tile_edges(hq, hkv, grid, n_text):
+    """Tensor-core attention and attention mass on other head groupings and at the tile edges (one row past a tile, fewer
+    rows than a tile), each against the oracle; a single KV head is narrower than the tensor-core path takes and must
+    fall back to the CUDA-core kernel."""
+    from dataclasses import replace
+    cfg = replace(wl.small_bf16(n_frames=2, grid=grid, n_text=n_text, total=grid[0] * grid[1], keep_full=0, seed=40 + hq),
+                  n_q_heads=hq, n_kv_heads=hkv)
+    L = wl.make_layer(cfg, with_current=True)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    segs3 = [(L.anchor_k, L.anchor_v, L.anchor_pos), (L.hist_k, L.hist_v, L.hist_pos), (L.cur_k, L.cur_v, L.q_pos)]
+    out, lse = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos, want_lse=True)
+    n_keys = sum(len(s[0]) for s in segs3)
+    want, want_lse = oracle.attend(L.q, L.q_pos, segs3, cfg.rope_base, want_lse=True)
+    assert np.abs(host(out).astype(np.float64) - want).max() <= 2e-2
+    assert np.abs(host(lse) - want_lse).max() <= 2e-2
+    if hkv * cfg.head_dim % 256:                                   # narrower than the tensor-core path takes: CUDA cores, no mass
+        with pytest.raises(pc.PackCacheError) as e:
+            pc.pc_attend_mass(ctx, lse, n_keys)
+        assert e.value.status == pc.PC_ERR_UNSUPPORTED and pc.pc_poll_status(ctx) == pc.PC_OK
+        ctx.close()
+        return
+    mass = pc.pc_attend_mass(ctx, lse, n_keys)
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+    _check_mass(host(mass).astype(np.float64), oracle.attend_mass(L.q, L.q_pos, [(s[0], s[2]) for s in segs3], cfg.rope_base))
+    ctx.close()
