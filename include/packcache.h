@@ -307,8 +307,11 @@ pc_status pc_window_state(pc_window *w, int32_t *n_frames, int32_t *counts, int6
  * recorded since the last poll (PC_OK if none). */
 pc_status pc_poll_status(pc_ctx *ctx, void *stream);
 
-/* Choose the bf16 attention kernel: 0 = tcgen05 tensor-core kernel (default),
- * 1 = CUDA-core kernel (a slow second opinion).  Returns PC_ERR_INVALID_ARG otherwise. */
+/* Choose the bf16 attention kernel: 0 = tcgen05 tensor-core kernel (default), 1 = CUDA-core kernel (a slow second
+ * opinion), 2 = tcgen05 kernel that issues its multiply-adds for pairs of CTAs (cta_group::2: the two CTAs of a cluster
+ * share every key / value tile, each loading half of it; used when the query tiles per KV head divide by four, else as
+ * 0).  2 gives the bits of 0; on a B200 it is slower at the shapes measured (the pair's barrier traffic crosses SMs on
+ * every tile) and is kept for comparison.  Returns PC_ERR_INVALID_ARG otherwise. */
 pc_status pc_set_attend_impl(pc_ctx *ctx, int32_t impl);
 
 /* Fix the number of key ranges the tensor-core attention kernel splits the keys into (1..4); 0 lets each call

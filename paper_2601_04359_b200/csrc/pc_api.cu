@@ -124,7 +124,7 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
 }
 
 extern "C" pc_status pc_set_attend_impl(pc_ctx *c, int32_t impl) {
-    if (!c || impl < 0 || impl > 1) return PC_ERR_INVALID_ARG;
+    if (!c || impl < 0 || impl > 2) return PC_ERR_INVALID_ARG;
     c->attend_impl = impl;
     return PC_OK;
 }

@@ -29,7 +29,7 @@ pc_status check_queries(pc_ctx *ctx, const void *q, const int32_t *q_pos, int32_
 }
 
 bool tensor_core_path(const pc_ctx *ctx) {
-    return ctx->attend_impl == 0 && pc_tensor_core_shape(ctx);
+    return ctx->attend_impl != 1 && pc_tensor_core_shape(ctx);
 }
 
 }  // namespace

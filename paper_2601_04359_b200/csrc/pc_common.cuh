@@ -55,7 +55,7 @@ struct pc_ctx {
     int sm_count;
     int group;                 // Hq / Hkv
     int elem_size;             // bytes per element
-    int attend_impl;           // 0 tensor-core (bf16), 1 CUDA-core
+    int attend_impl;           // 0 tensor-core (bf16), 1 CUDA-core, 2 tensor-core with CTA-pair multiply-adds
     pc_rope_dev rope;
     float2 *rope_tab;          // owned
     int32_t *status;           // device [2]: code, where

@@ -231,7 +231,7 @@ extern "C" pc_status pc_attend_mass(pc_ctx *ctx, const float *lse, float *mass, 
     if (!ctx || !lse || !mass) return PC_ERR_INVALID_ARG;
     if (!pc_aligned16(lse) || !pc_aligned16(mass)) return PC_ERR_INVALID_ARG;
     const pc_layer_desc &D = ctx->desc;
-    if (!pc_tensor_core_shape(ctx) || ctx->attend_impl != 0) return PC_ERR_UNSUPPORTED;
+    if (!pc_tensor_core_shape(ctx) || ctx->attend_impl == 1) return PC_ERR_UNSUPPORTED;
     if (ctx->last_n_q <= 0 || ctx->last_n_seg <= 0) return PC_ERR_INVALID_ARG;   // no tensor-core attention call precedes
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
 

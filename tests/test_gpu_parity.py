@@ -174,6 +174,43 @@ def test_attention_key_ranges_merge_like_one_range(cluster):
     ctx.close()
 
 
+# ------------------------------------------------------------------------------------------- CTA-pair kernel
+@pytest.mark.parametrize("shape", ["group4", "four_row_tiles"])
+def test_cta_pair_attention_gives_the_bits_of_the_single_cta_kernel(shape):
+    """The kernel that issues its multiply-adds for pairs of CTAs (each CTA holds half of every key / value tile) against
+    the oracle and, bit for bit, against the default kernel, for one to four key ranges with ragged segments."""
+    if shape == "group4":        # four query heads per KV head, two row tiles: eight query tiles per KV head
+        cfg = replace(wl.small_bf16(n_frames=3, grid=(12, 21), n_text=130, total=500, keep_full=1, seed=50), n_q_heads=32, n_kv_heads=8)
+    else:                        # three query heads per KV head, four row tiles (the last one ragged)
+        cfg = wl.small_bf16(n_frames=2, grid=(16, 25), n_text=37, total=400, keep_full=1, seed=51)
+    L = wl.make_layer(cfg, with_current=True)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    segs = [(L.anchor_k, L.anchor_v, L.anchor_pos), (L.hist_k, L.hist_v, L.hist_pos), (L.cur_k, L.cur_v, L.q_pos)]
+    want, want_lse = oracle.attend(L.q, L.q_pos, segs, cfg.rope_base, want_lse=True)
+    for n in (1, 2, 3, 4):
+        pc.pc_set_kv_splits(ctx, n)
+        pc.pc_set_attend_impl(ctx, 0)
+        a, la = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos, want_lse=True)
+        a, la = a.clone(), la.clone()
+        pc.pc_set_attend_impl(ctx, 2)
+        b, lb = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos, want_lse=True)
+        _ok(ctx)
+        assert torch.equal(a, b) and torch.equal(la, lb)
+        assert np.abs(host(b).astype(np.float64) - want).max() <= BF16_ATOL
+        assert np.abs(host(lb) - want_lse).max() <= 2e-2
+    # a shape whose query tiles per KV head do not divide by four runs the default kernel under the same setting
+    cfg3 = wl.small_bf16(n_frames=2, grid=(8, 9), seed=52)
+    L3 = wl.make_layer(cfg3)
+    D3 = DeviceLayer(L3)
+    ctx3 = make_ctx(cfg3)
+    a = pc.pc_attend_frame(ctx3, D3.cache, None, D3.q, D3.q_pos).clone()
+    pc.pc_set_attend_impl(ctx3, 2)
+    assert torch.equal(a, pc.pc_attend_frame(ctx3, D3.cache, None, D3.q, D3.q_pos))
+    _ok(ctx3)
+    ctx.close(); ctx3.close()
+
+
 # ------------------------------------------------------------------------------------------- prepared key set
 @pytest.mark.parametrize("cfg_name", ["tiny", "small_bf16"])
 def test_prepared_attention_equals_attend_frame_over_several_passes(cfg_name):
