@@ -34,7 +34,7 @@ N_LAYERS = 4          # rotated input sets; 4 x ~0.2 GB > L2 (--layers changes i
 KERNELS_PER_STEP = 8  # k_qpool, k_qpool_reduce, k_score, k_select, k_pack, k_rope_rows, k_attend_tc, k_combine
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_attend_tc launch at this workload, from the ncu capture
 # summarised in profiles/ncu_kernels_lumos47_small_case.md (same launch shape); None when the kernel has changed since
-ATTEND_DRAM_TRAFFIC = 43_979_776 + 3_303_424
+ATTEND_DRAM_TRAFFIC = 43_979_008 + 3_339_520
 
 
 def _peaks():
