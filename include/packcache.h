@@ -130,7 +130,8 @@ pc_status pc_plan_budget(const pc_budget_params *params, int32_t n_frames, const
  *   q device [n_q][Hq][d]; q_pos device [n_q][4]; budget host [n_frames];
  *   valid device [n_src] bytes or NULL (0 = masked cache position, Eq. 1: never
  *   kept unless the budget exceeds the valid tokens);
- *   scores_override device [n_src] fp32 or NULL: skip scoring, select on these;
+ *   scores_override device [n_src] fp32 or NULL: skip scoring, select on these (4-byte alignment is enough here, so
+ *   an offset into a longer score array, such as the attention masses past the anchors, can be passed);
  *   scores device out [n_src] fp32 (may be NULL with an override);
  *   sel_idx device out [sum(budget)].
  * Errors: PC_ERR_INVALID_ARG, PC_ERR_BUDGET (budget[f] > frame_count[f]),

@@ -521,7 +521,7 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
             if (st != PC_OK) return st;
         }
         select_on = scores;
-    } else if (!pc_aligned16(scores_override)) {
+    } else if (reinterpret_cast<uintptr_t>(scores_override) & 3) {      // read element by element: any float address will do
         return PC_ERR_INVALID_ARG;
     }
     if (n_frames > 0 && out > 0) {

@@ -135,9 +135,9 @@ def test_window_selection_guided_by_attention_mass():
     anchors ++ window ++ itself, the masses of that call (history ++ current part) rank the tokens once the frame has
     been appended.  Masses are checked against the oracle's; selection, packed rows and positions must then match the
     reference window bit for bit when it ranks on the same fp32 masses."""
-    cfg = wl.small_bf16(n_frames=7, grid=(12, 21), n_text=128, total=600, kind=wl.HALFLIFE, param=2.0, keep_full=1, seed=21)
+    cfg = wl.small_bf16(n_frames=7, grid=(11, 23), n_text=129, total=600, kind=wl.HALFLIFE, param=2.0, keep_full=1, seed=21)
     n, W, total = cfg.frame_tokens, 3, 600
-    assert n % 4 == 0 and cfg.n_anchor % 4 == 0                     # score pointers handed to the window stay 16-byte aligned
+    assert n % 4 and cfg.n_anchor % 4                                # the score pointers handed to the window are only float-aligned
     L = wl.make_layer(cfg)
     rng = np.random.Generator(np.random.Philox(key=[21, 5]))
     st = lambda x: wl.to_storage(x.astype(np.float32), cfg.dtype)
