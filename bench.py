@@ -47,6 +47,16 @@ def _peaks():
 
 
 # --------------------------------------------------------------------------------------------- ranks
+def _cpu_model() -> str:
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.lower().startswith("model name"):
+                return ln.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def rank_layer_ids(rank: int, n_layers: int):
     """Layers a rank draws: disjoint seeded layers per rank (weak scaling by replication, nothing exchanged on the data
     path)."""
@@ -445,6 +455,13 @@ def run_cuda(args):
                                 n_rows=max(800, int(frac * cfg.n_q * cfg.n_q_heads)))
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
                                 "sample": what, "sample_seconds": round(time.perf_counter() - t0, 1)}
+        # the same oracle on one thread, from a small sample (a few seconds), and the host's CPU model
+        n_threads = oracle.max_threads()
+        oracle.set_threads(1)
+        v1, what1 = oracle_sample(cfg, host_layers[0], n_score=60, n_rows=120)
+        oracle.set_threads(n_threads)
+        line["cpu_baseline"]["single_thread"] = {"value": v1, "unit": UNIT, "sample": what1}
+        line["cpu_baseline"]["cpu_model"] = _cpu_model()
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

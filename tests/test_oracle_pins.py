@@ -91,6 +91,35 @@ def test_plan_equals_exact_rational_apportionment(W, B):
         assert got == _hamilton(wts, B, [N] * W), (kind, W, B)
 
 
+def _q32_halflife_weights(W, keep_full, half_life):
+    """floor(2^-((d - 1 - keep_full)/h) * 2^32 + 1/2) for d = keep_full + 1 .. W, in 60-digit decimal arithmetic."""
+    from decimal import ROUND_FLOOR, Decimal, getcontext
+    getcontext().prec = 60
+    out = []
+    for d in range(keep_full + 1, W + 1):
+        g = Decimal(2) ** (Decimal(-(d - 1 - keep_full)) / Decimal(half_life))
+        out.append(int((g * (1 << 32) + Decimal("0.5")).to_integral_value(rounding=ROUND_FLOOR)))
+    return out
+
+
+def test_plan_of_the_benchmark_configurations_by_exact_arithmetic():
+    """The budget vectors of the measured configurations (12 frames linear at 25 %; 24 frames at half-life 4; 47 frames
+    with the two newest whole and 6048 tokens at half-life 4; 47 frames at 10 % and half-life 2) against largest-remainder
+    apportionment in exact integers / rationals over weights quantised once to 2^-32."""
+    N = 1008
+    got = oracle.plan_budget(oracle.LINEAR, 0.0, (12 * N) // 4, 0, [N] * 12).tolist()[::-1]
+    assert got == _hamilton([Fraction(13 - d) for d in range(1, 13)], (12 * N) // 4, [N] * 12)
+    assert got[0] == 465 and got[-1] == 39                              # 3024 * 12/78 and 3024 * 1/78, rounded by remainder
+    got = oracle.plan_budget(oracle.HALFLIFE, 4.0, 6048, 0, [N] * 24).tolist()[::-1]
+    assert got == _hamilton([Fraction(w) for w in _q32_halflife_weights(24, 0, 4)], 6048, [N] * 24)
+    got = oracle.plan_budget(oracle.HALFLIFE, 4.0, 2 * N + 6048, 2, [N] * 47).tolist()[::-1]
+    tail = _hamilton([Fraction(w) for w in _q32_halflife_weights(47, 2, 4)], 6048, [N] * 45)
+    assert got == [N, N] + tail and sum(got) == 8064 and sum(1 for t in got if t) == 46
+    got = oracle.plan_budget(oracle.HALFLIFE, 2.0, (47 * N) // 10, 0, [N] * 47).tolist()[::-1]
+    assert got == _hamilton([Fraction(w) for w in _q32_halflife_weights(47, 0, 2)], (47 * N) // 10, [N] * 47)
+    assert got[:2] == [N, N] and sum(1 for t in got if t) == 24          # the two nearest frames are capped, the surplus re-shared
+
+
 def test_plan_identities():
     rng = np.random.default_rng(1)
     for kind, param in [(oracle.GEOMETRIC, 0.7), (oracle.GEOMETRIC, 0.5), (oracle.LINEAR, 0.0),
