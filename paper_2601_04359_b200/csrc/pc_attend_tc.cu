@@ -617,9 +617,9 @@ k_attend_tc_pair(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tc_fence_after();
                 for (int t = 0; t < 2; ++t) {
                     issue_qk(t, 0);
-                    if (lead) tc_commit_pair(bar(BAR_SFULL + t), 3);
+                    if (lead) tc_commit_pair(bar(BAR_SFULL + t));
                 }
-                if (lead) tc_commit_pair(bar(BAR_KEMPTY + 0), 3);
+                if (lead) tc_commit_pair(bar(BAR_KEMPTY + 0));
             }
             for (int j = 0; j < n_j && alive; ++j) {
                 const int st = j % KV_STAGES, use = j / KV_STAGES, nst = (j + 1) % KV_STAGES;
@@ -639,11 +639,11 @@ k_attend_tc_pair(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     }
                     if (!alive) break;
                     if (j + 1 < n_j) issue_qk(t, nst);
-                    if (lead) tc_commit_pair(bar(BAR_SFULL + t), 3);
+                    if (lead) tc_commit_pair(bar(BAR_SFULL + t));
                 }
-                if (alive && lead) tc_commit_pair(bar(BAR_VEMPTY + st), 3);
+                if (alive && lead) tc_commit_pair(bar(BAR_VEMPTY + st));
             }
-            if (lead) tc_commit_pair(bar(BAR_DONE), 3);
+            if (lead) tc_commit_pair(bar(BAR_DONE));
             __syncwarp();
         }
         // nothing of the pair may still be running on either tensor core when TMEM is freed
