@@ -62,6 +62,7 @@ struct RopeJob {
     const int32_t *pos;
     __nv_bfloat16 *dst;
     int n_rows, chunks_per_row /* 16-byte chunks, a multiple of 32 */, first_warp;
+    int rows_per_pos;      // consecutive rows that share one position record (a wide query row is cut into slices)
     float scale;
 };
 struct RopeJobs { RopeJob job[PC_MAX_SEGMENTS + 1]; int n_jobs, total_warps; };
@@ -100,7 +101,7 @@ __global__ void __launch_bounds__(256) k_rope_rows(const __grid_constant__ RopeJ
     while (ji + 1 < jobs.n_jobs && warp >= jobs.job[ji + 1].first_warp) ++ji;
     const RopeJob &J = jobs.job[ji];
     const int row = warp - J.first_warp;
-    const int4 pp = __ldg(reinterpret_cast<const int4 *>(J.pos) + row);
+    const int4 pp = __ldg(reinterpret_cast<const int4 *>(J.pos) + row / J.rows_per_pos);
     const int pair0 = ((lane * 8) % d) / 2;
     float2 cs[4];
 #pragma unroll
@@ -884,7 +885,7 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     for (int s = 0; s < n_seg; ++s) {
         if (what & PC_TC_ROPE_K) {
             jobs.job[n_jobs++] = RopeJob{static_cast<const __nv_bfloat16 *>(segs[s].k), segs[s].pos,
-                                         k_rot + (size_t)tiles * TILE * row_elems, segs[s].n_tokens, k_chunks, warps, 1.0f};
+                                         k_rot + (size_t)tiles * TILE * row_elems, segs[s].n_tokens, k_chunks, warps, 1, 1.0f};
             warps += segs[s].n_tokens;
         }
         tiles += div_up(segs[s].n_tokens, TILE);
@@ -894,9 +895,11 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     if ((size_t)tiles * TILE > ctx->k_rot_rows) return PC_ERR_CAPACITY;
     __nv_bfloat16 *q_rot = static_cast<__nv_bfloat16 *>(ctx->q_rot);
     if (what & PC_TC_ROPE_Q) {
-        jobs.job[n_jobs++] = RopeJob{static_cast<const __nv_bfloat16 *>(q), q_pos, q_rot, n_q, q_chunks, warps,
+        // a query row is as many slices as it holds key-row widths when that divides evenly: every warp then has the same job
+        const int slices = (q_chunks % k_chunks == 0) ? q_chunks / k_chunks : 1;
+        jobs.job[n_jobs++] = RopeJob{static_cast<const __nv_bfloat16 *>(q), q_pos, q_rot, n_q * slices, q_chunks / slices, warps, slices,
                                      (float)(1.4426950408889634 / std::sqrt((double)D.head_dim))};
-        warps += n_q;
+        warps += n_q * slices;
     }
     jobs.n_jobs = n_jobs;
     jobs.total_warps = warps;
