@@ -67,7 +67,8 @@ struct RopeJob {
 };
 struct RopeJobs { RopeJob job[PC_MAX_SEGMENTS + 1]; int n_jobs, total_warps; };
 
-// One warp per row.  32 lanes x 8 elements = 256 is a multiple of d, so all of a lane's chunks (lane, lane + 32, ...)
+// One warp per row (a query row wider than a key row is cut into key-row-wide slices, one warp each, so that all warps
+// carry the same load).  32 lanes x 8 elements = 256 is a multiple of d, so all of a lane's chunks (lane, lane + 32, ...)
 // hold the same four rotary pairs: four table entries per lane per row, with the output scale folded in, serve every
 // chunk.  All of a row's chunks are loaded before any is used.
 template <int CPL /* chunks per lane */>
