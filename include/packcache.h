@@ -258,6 +258,8 @@ pc_status pc_score_tokens_static(const pc_layer_desc *desc, const void *hist_k, 
  *          with `rebase` set the temporal coordinate of every retained history token drops by t_step per dropped frame
  *          (Eq. 9: only t moves; h, w and the tag are carried).  Anchors are never touched.  The caller builds the next
  *          frames' positions in the shifted frame of reference: pc_window_state reports the accumulated shift.
+ *          Frames that a plan leaves with nothing at the old end of the window (budget.min_quota starves the oldest frames first
+ *          when the budget cannot serve every frame) leave it in the same way and count in the rebase.
  * Re-selection is incremental: the source of a pack is what the last pack kept plus the frames appended since.
  * All device memory is the caller's: the two history buffers (each must hold budget.total tokens plus the frames
  * appended between two packs), a score buffer and an index buffer of the same token capacity. */
@@ -292,7 +294,8 @@ pc_status pc_window_append_masked(pc_window *w, const pc_segment *frame, const u
 
 /* Bring the cache back inside window and budget for the frame whose queries are q (see the regimes above); regime
  * (host out, may be NULL) receives PC_WINDOW_FILL / PACK / SLIDE.  scores_override: device fp32 scores of the source
- * tokens (after dropped frames) to select on instead of scoring, or NULL.  Errors as pc_score / pc_compact. */
+ * tokens (after the frames beyond the window; frames the plan then starves are skipped inside) to select on instead of
+ * scoring, or NULL.  Errors as pc_score / pc_compact. */
 pc_status pc_window_update(pc_window *w, const void *q, const int32_t *q_pos, int32_t n_q, const float *scores_override,
                            int32_t *regime, void *stream);
 

@@ -6,7 +6,9 @@ package.  Reading taken where the paper is silent: frames are appended whole whi
 token budget; otherwise frames beyond W leave first (first in, first out), the retained frames get quotas from the
 decay kernel over their *current* token counts, each keeps its best-scoring tokens (re-selection from what the last
 pack kept plus what was appended since), and with rebase the temporal coordinate of every retained token falls by
-t_step per dropped frame while (h, w, tag) stay as they are.
+t_step per dropped frame while (h, w, tag) stay as they are.  Frames that the plan leaves with nothing at the old end of
+the window (the minimum quota b_min starves the oldest frames first when the budget cannot serve every frame) leave the
+window like frames beyond W: first in, first out, counted in the rebase.
 """
 from __future__ import annotations
 
@@ -21,8 +23,9 @@ FILL, PACK, SLIDE = 0, 1, 2
 
 class WindowRef:
     def __init__(self, window: int, kind: int, param: float, total: int, keep_full: int, rebase: bool = False,
-                 t_step: int = 4, rope_base: float = 10000.0):
+                 t_step: int = 4, rope_base: float = 10000.0, min_quota: int = 0):
         self.window, self.kind, self.param, self.total, self.keep_full = window, kind, param, total, keep_full
+        self.min_quota = min_quota
         self.rebase, self.t_step, self.rope_base = rebase, t_step, rope_base
         self.k: Optional[np.ndarray] = None        # [tokens][Hkv][d], frames oldest -> newest
         self.v: Optional[np.ndarray] = None
@@ -48,9 +51,17 @@ class WindowRef:
         k, v, pos, counts, drop = self.source_after_drop()
         if drop == 0 and int(np.sum(counts)) <= self.total:
             return FILL
-        budget = oracle.plan_budget(self.kind, self.param, self.total, self.keep_full, counts)
+        budget = oracle.plan_budget(self.kind, self.param, self.total, self.keep_full, counts, self.min_quota)
+        lead = 0                                   # frames at the old end that the plan leaves with nothing: they leave too
+        while lead < len(budget) and budget[lead] == 0:
+            lead += 1
+        if lead:
+            first = int(np.sum(counts[:lead]))
+            k, v, pos, counts, budget, drop = k[first:], v[first:], pos[first:], counts[lead:], budget[lead:], drop + lead
+            if scores32 is not None:
+                scores32 = scores32[first:]
         if scores32 is None:
-            scores32 = oracle.score_pooled(k, pos, q, q_pos, self.rope_base).astype(np.float32)
+            scores32 = oracle.score_pooled(k, pos, q, q_pos, self.rope_base).astype(np.float32) if len(k) else np.zeros(0, np.float32)
         sel = oracle.select(scores32, counts, budget)
         delta = drop * self.t_step if self.rebase else 0
         self.k, self.v, self.pos = oracle.pack(k, v, pos, sel, delta)

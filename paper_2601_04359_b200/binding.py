@@ -343,14 +343,14 @@ class Window:
     is managed by the library).  Argument marshalling only: plan, score, select, pack run in the library."""
 
     def __init__(self, ctx: Context, window: int, kind: int, param: float, total: int, keep_full: int, anchors: Segment,
-                 hist_a: Segment, hist_b: Segment, rebase: bool = False, t_step: int = 4):
+                 hist_a: Segment, hist_b: Segment, rebase: bool = False, t_step: int = 4, min_quota: int = 0):
         self.ctx, self.anchors, self.bufs = ctx, anchors, (hist_a, hist_b)
         cap = min(hist_a.capacity, hist_b.capacity)
         dev = hist_a.k.device
         self.scores = torch.empty(cap, dtype=torch.float32, device=dev)
         self.sel_idx = torch.empty(cap, dtype=torch.int32, device=dev)
         self.window = window
-        p = pc_window_params(window, pc_budget_params(kind, param, total, keep_full, 0), 1 if rebase else 0, t_step)
+        p = pc_window_params(window, pc_budget_params(kind, param, total, keep_full, min_quota), 1 if rebase else 0, t_step)
         a, ha, hb = anchors.c(), hist_a.c(), hist_b.c()
         h = C.c_void_p()
         _check(load().pc_window_create(ctx.handle, C.byref(p), C.byref(a), C.byref(ha), C.byref(hb), _ptr(self.scores),

@@ -163,25 +163,42 @@ extern "C" pc_status pc_window_update(pc_window *w, const void *q, const int32_t
     w->budget.assign((size_t)std::max(kept, 1), 0);
     pc_status st = pc_plan_budget(&w->p.budget, kept, src.frame_count, w->budget.data());
     if (st != PC_OK) return st;
+    // Frames that the plan leaves with nothing at the old end (a minimum quota starves the oldest frames first) leave the
+    // window like frames beyond W: first in, first out, counted in the rebase.
+    int lead = 0;
+    int64_t lead_tokens = 0;
+    while (lead < kept && w->budget[lead] == 0) lead_tokens += src.frame_count[lead++];
+    const int32_t *budget = w->budget.data() + lead;
+    const int left = drop + lead, stay = kept - lead;
+    src.history.k = static_cast<char *>(src.history.k) + (size_t)lead_tokens * row;
+    src.history.v = static_cast<char *>(src.history.v) + (size_t)lead_tokens * row;
+    src.history.pos += 4 * (size_t)lead_tokens;
+    src.history.n_tokens -= (int32_t)lead_tokens;
+    src.history.capacity -= (int32_t)lead_tokens;
+    src.n_frames = stay;
+    src.frame_count += lead;
+    if (scores_override) scores_override += lead_tokens;
     int64_t n_sel = 0;
-    for (int f = 0; f < kept; ++f) n_sel += w->budget[f];
+    for (int f = 0; f < stay; ++f) n_sel += budget[f];
     if (n_sel > B.capacity) return PC_ERR_CAPACITY;
-    st = pc_score(w->ctx, &src, q, q_pos, n_q, w->budget.data(), nullptr, scores_override, w->scores, w->sel_idx, stream);
-    if (st != PC_OK) return st;
-    pc_cache dst;
-    dst.anchors = w->anchors;
-    dst.history = B;
-    dst.n_frames = kept;
-    dst.frame_count = w->budget.data();
-    const int32_t delta_t = w->p.rebase ? drop * w->p.t_step : 0;  // Eq. 9: t falls by the number of dropped frames
-    st = pc_compact(w->ctx, &src, w->sel_idx, w->budget.data(), delta_t, &dst, stream);
-    if (st != PC_OK) return st;
+    const int32_t delta_t = w->p.rebase ? left * w->p.t_step : 0;  // Eq. 9: t falls by the number of frames that left
+    if (stay > 0) {
+        st = pc_score(w->ctx, &src, q, q_pos, n_q, budget, nullptr, scores_override, w->scores, w->sel_idx, stream);
+        if (st != PC_OK) return st;
+        pc_cache dst;
+        dst.anchors = w->anchors;
+        dst.history = B;
+        dst.n_frames = stay;
+        dst.frame_count = budget;
+        st = pc_compact(w->ctx, &src, w->sel_idx, budget, delta_t, &dst, stream);
+        if (st != PC_OK) return st;
+    }
     B.n_tokens = (int32_t)n_sel;
     A.n_tokens = 0;
     w->active ^= 1;
-    w->count.assign(w->budget.begin(), w->budget.begin() + kept);
+    w->count.assign(budget, budget + stay);
     w->t_shift += delta_t;
-    if (regime) *regime = drop ? PC_WINDOW_SLIDE : PC_WINDOW_PACK;
+    if (regime) *regime = left ? PC_WINDOW_SLIDE : PC_WINDOW_PACK;
     return PC_OK;
 }
 

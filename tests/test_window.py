@@ -94,6 +94,39 @@ def test_window_rebase_moves_t_only_and_kept_sets_shrink():
         assert sum(plain.count) <= 96 and len(plain.count) <= 3
 
 
+def test_window_minimum_quota_lets_the_oldest_frames_leave():
+    """b_min of Sec. 3.4: every frame that stays keeps at least m tokens; when W * m exceeds the budget only floor(B / m)
+    frames can be served and the oldest leave first (first in, first out) — as whole frames, counted in the rebase."""
+    cfg = wl.CONFIGS["tiny"]
+    n = cfg.frame_tokens                                                      # 64 tokens per frame
+    fr = _frames(cfg, 8, seed=5)
+    W, B, m = 6, 128, 48                                                      # floor(128 / 48) = 2 frames can be served
+    ref = ow.WindowRef(W, oracle.CLOSED_HALF, 0.5, B, 0, rebase=True, t_step=4, min_quota=m)
+    left_total = 0
+    for f in range(8):
+        pos = fr[f]["pos"].copy(); pos[:, 0] -= ref.t_shift
+        qpos = fr[f + 1]["pos"].copy(); qpos[:, 0] -= ref.t_shift
+        before = len(ref.count) + 1
+        ref.append(fr[f]["k"], fr[f]["v"], pos)
+        regime = ref.update(fr[f + 1]["q"], qpos)
+        left_total += before - len(ref.count)
+        assert ref.t_shift == 4 * left_total                                  # every frame that left moved t by one step
+        if f == 0:
+            assert regime == ow.FILL and ref.count == [n]
+            continue
+        assert len(ref.count) == 2 and sum(ref.count) == B and min(ref.count) >= m
+        frames_of = (ref.pos[:, 3] - cfg.n_anchor) // n
+        assert sorted(set(frames_of.tolist())) == [f - 1, f]                  # the two newest frames, nothing older
+        assert regime == (ow.FILL if f == 1 else ow.SLIDE)                    # two whole frames are exactly the budget
+    # a quota that every frame of the window can have changes nothing about who stays
+    easy = ow.WindowRef(W, oracle.CLOSED_HALF, 0.5, B, 0, min_quota=8)        # 6 * 8 <= 128
+    for f in range(8):
+        easy.append(fr[f]["k"], fr[f]["v"], fr[f]["pos"])
+        easy.update(fr[f + 1]["q"], fr[f + 1]["pos"])
+        assert len(easy.count) == min(f + 1, W) and (f == 0 or min(easy.count) >= 8)
+        assert sum(easy.count) == min(B, (f + 1) * n)
+
+
 # ------------------------------------------------------------------------------------------------ GPU
 @pytest.mark.gpu
 @pytest.mark.parametrize("rebase", [False, True])
@@ -243,4 +276,42 @@ def test_window_masked_append_matches_reference():
     valid = np.ones(n, np.uint8)
     win.append_masked(segment(fr[0]["k"], fr[0]["v"], fr[0]["pos"], cfg.dtype), torch.from_numpy(valid).cuda(), n - 5)
     assert pc.pc_poll_status(ctx) == pc.PC_ERR_INVALID_ARG
+    win.close(); ctx.close()
+
+
+@pytest.mark.gpu
+def test_window_minimum_quota_matches_reference():
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200.device import dev, host, idev, make_ctx, segment
+
+    cfg = wl.small_bf16(n_frames=8, grid=(9, 15), n_text=37, total=300, kind=wl.HALFLIFE, param=2.0, keep_full=0, seed=31)
+    n, W, total, m = cfg.frame_tokens, 5, 300, 90                             # floor(300 / 90) = 3 of the 5 frames can be served
+    L = wl.make_layer(cfg)
+    fr = _frames(cfg, 7, seed=32)
+    ctx = make_ctx(cfg, max_keys=cfg.n_anchor + total + 3 * n)
+    cap = total + 2 * n
+    mk = lambda: pc.Segment(torch.zeros((cap, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((cap, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((cap, 4), dtype=torch.int32, device="cuda"), 0)
+    win = pc.Window(ctx, W, pc.PC_HALFLIFE, 2.0, total, 0, segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype), mk(), mk(),
+                    rebase=True, t_step=4, min_quota=m)
+    ref = ow.WindowRef(W, oracle.HALFLIFE, 2.0, total, 0, rebase=True, t_step=4, min_quota=m)
+    for f in range(7):
+        pos = fr[f]["pos"].copy(); pos[:, 0] -= ref.t_shift
+        qpos = fr[f + 1]["pos"].copy(); qpos[:, 0] -= ref.t_shift
+        ref.append(fr[f]["k"], fr[f]["v"], pos)
+        win.append(segment(fr[f]["k"], fr[f]["v"], pos, cfg.dtype))
+        sk, _, spos, _, _ = ref.source_after_drop()
+        s32 = oracle.score_pooled(sk, spos, fr[f + 1]["q"], qpos, cfg.rope_base).astype(np.float32)
+        want = ref.update(fr[f + 1]["q"], qpos, scores32=s32)
+        got = win.update(dev(fr[f + 1]["q"], cfg.dtype), idev(qpos), scores_override=torch.from_numpy(s32).cuda())
+        assert got == want and pc.pc_poll_status(ctx) == pc.PC_OK
+        counts, shift, _ = win.state()
+        assert counts.tolist() == ref.count and shift == ref.t_shift
+        assert len(ref.count) <= 3 and (f == 0 or min(ref.count) >= m)
+        cache = win.cache()
+        k = int(counts.sum())
+        assert np.array_equal(host(cache.history.k)[:k], ref.k) and np.array_equal(cache.history.pos.cpu().numpy()[:k], ref.pos)
+    assert ref.t_shift > 0
     win.close(); ctx.close()
