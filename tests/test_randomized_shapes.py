@@ -74,3 +74,72 @@ def test_random_shapes_against_the_oracle(seed):
             assert pc.pc_poll_status(ctx) == pc.PC_OK, what
             assert (np.abs(got - want_mass) <= 1e-2 * want_mass + 1e-3 / n_keys).all(), what
         ctx.close()
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_random_cache_windows_against_the_reference(seed):
+    """Seeded random cache-window runs (window length 1-6, all decay kernels, budgets from a few tokens to several frames,
+    kept-whole frames, minimum quotas, cache masks at append time, rebase on and off): the library's window against the
+    reference state machine after every frame — regime, token counts, accumulated shift, packed K / V / positions bit for
+    bit — both deciding on the same fp32 scores."""
+    from oracle import window as ow
+    from paper_2601_04359_b200.device import dev, idev, segment
+
+    rng = np.random.default_rng(100 + seed)
+    for case in range(8):
+        grid = (int(rng.integers(2, 14)), int(rng.integers(2, 20)))
+        n = grid[0] * grid[1]
+        n_text, n_steps, W = int(rng.integers(0, 100)), int(rng.integers(3, 9)), int(rng.integers(1, 7))
+        kind = list(DECAY)[rng.integers(4)]
+        total = int(rng.integers(1, 4 * n))
+        keep_full = int(rng.integers(0, 2)) if total >= n else 0
+        m = int(rng.integers(0, max(1, n // 2))) if rng.integers(2) else 0
+        rebase, masked = bool(rng.integers(2)), bool(rng.integers(2))
+        hq, hkv = [(24, 8), (8, 8), (4, 2), (6, 2)][rng.integers(4)]
+        cfg = replace(wl.small_bf16(n_frames=n_steps + 1, grid=grid, n_text=n_text, total=total, kind=kind, param=DECAY[kind],
+                                    keep_full=keep_full, seed=6000 + 10 * seed + case), n_q_heads=hq, n_kv_heads=hkv)
+        what = f"grid {grid} W {W} decay {kind} budget {total}/{keep_full}/{m} rebase {rebase} masked {masked} heads {hq}/{hkv}"
+        L = wl.make_layer(cfg)
+        g = np.random.Generator(np.random.Philox(key=[seed, case]))
+        st = lambda x: wl.to_storage(x.astype(np.float32), cfg.dtype)
+        cap = total + 2 * n + 8
+        ctx = make_ctx(cfg, max_keys=cfg.n_anchor + cap + n)
+        mk = lambda: pc.Segment(torch.zeros((cap, hkv, 128), dtype=torch.bfloat16, device="cuda"),
+                                torch.zeros((cap, hkv, 128), dtype=torch.bfloat16, device="cuda"),
+                                torch.zeros((cap, 4), dtype=torch.int32, device="cuda"), 0)
+        win = pc.Window(ctx, W, kind, DECAY[kind], total, keep_full, segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype),
+                        mk(), mk(), rebase=rebase, t_step=4, min_quota=m)
+        ref = ow.WindowRef(W, kind, DECAY[kind], total, keep_full, rebase=rebase, t_step=4, min_quota=m)
+        for f in range(1, n_steps + 1):
+            pos = wl.frame_positions(cfg, f, cfg.n_anchor + (f - 1) * n)
+            qpos = wl.frame_positions(cfg, f + 1, cfg.n_anchor + f * n)
+            pos[:, 0] -= ref.t_shift
+            qpos[:, 0] -= ref.t_shift
+            k, v = st(g.standard_normal((n, hkv, 128))), st(g.standard_normal((n, hkv, 128)))
+            q = st(g.standard_normal((n, hq, 128)))
+            if masked and rng.integers(2):
+                valid = (rng.random(n) < rng.random()).astype(np.uint8)
+                ref.append(k, v, pos, valid=valid)
+                win.append_masked(segment(k, v, pos, cfg.dtype), torch.from_numpy(valid).cuda(), int(valid.sum()))
+            else:
+                ref.append(k, v, pos)
+                win.append(segment(k, v, pos, cfg.dtype))
+            sk, _, spos, _, _ = ref.source_after_drop()
+            s32 = oracle.score_pooled(sk, spos, q, qpos, cfg.rope_base).astype(np.float32) if len(sk) else np.zeros(1, np.float32)
+            try:
+                want = ref.update(q, qpos, scores32=s32 if len(sk) else None)
+            except oracle.OracleError:                              # kept-whole frames exceed the budget: both must refuse
+                with pytest.raises(pc.PackCacheError):
+                    win.update(dev(q, cfg.dtype), idev(qpos), scores_override=torch.from_numpy(s32).cuda())
+                break
+            got = win.update(dev(q, cfg.dtype), idev(qpos), scores_override=torch.from_numpy(s32).cuda())
+            assert got == want and pc.pc_poll_status(ctx) == pc.PC_OK, what
+            counts, shift, _ = win.state()
+            assert counts.tolist() == ref.count and shift == ref.t_shift, what
+            kk = int(counts.sum())
+            if kk:
+                cache = win.cache()
+                assert np.array_equal(host(cache.history.k)[:kk], ref.k) and np.array_equal(host(cache.history.v)[:kk], ref.v), what
+                assert np.array_equal(cache.history.pos.cpu().numpy()[:kk], ref.pos), what
+        win.close()
+        ctx.close()
