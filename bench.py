@@ -31,10 +31,8 @@ METRIC = "late_frame_attn_plus_compaction_latency"
 UNIT = "ms/frame"
 WORKLOAD = "lumos47"
 N_LAYERS = 4          # rotated input sets; 4 x ~0.2 GB > L2 (--layers changes it for small profiler captures)
-KERNELS_PER_STEP = 8  # k_qpool, k_qpool_reduce, k_score, k_select, k_pack, k_rope_rows, k_attend_tc, k_combine
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_attend_tc launch at this workload, from the ncu capture
-# summarised in profiles/ncu_kernels_lumos47_small_case.md (same launch shape); None when the kernel has changed since
-ATTEND_DRAM_TRAFFIC = 43_979_008 + 3_339_520
+KERNELS_PER_STEP = 6  # k_qprep, k_score, k_select, k_pack, k_attend_tc, k_combine (anchors' rotated keys are kept per layer)
+ATTEND_DRAM_TRAFFIC = None
 
 
 def _peaks():
@@ -225,7 +223,9 @@ def run_cuda(args):
     # every rank draws its own layers (weak scaling: independent layers, no exchange on the data path)
     host_layers = [wl.make_layer(cfg, layer=i) for i in rank_layer_ids(rank, N_LAYERS)]
     layers = [DeviceLayer(L) for L in host_layers]
-    ctx = make_ctx(cfg)
+    # one context per layer, as a model would hold them: each keeps its layer's rotated anchor keys between frames
+    ctxs = [make_ctx(cfg) for _ in layers]
+    ctx = ctxs[0]
     n_sel = b.total
     dsts = [D.empty_packed(n_sel) for D in layers]
     scores = torch.empty(cfg.n_src, dtype=torch.float32, device="cuda")
@@ -235,6 +235,12 @@ def run_cuda(args):
     stream = torch.cuda.current_stream()
 
     def step(i):
+        D, dst = layers[i % N_LAYERS], dsts[i % N_LAYERS]
+        budget = pc.pc_plan_budget(b.kind, b.param, b.total, b.keep_full, avail)
+        pc.pc_frame_step(ctxs[i % N_LAYERS], D.cache, budget, 0, dst, D.q, D.q_pos, scores=scores, sel_idx=sel, out=out,
+                         stream=stream)
+
+    def step_separate(i):
         D, dst = layers[i % N_LAYERS], dsts[i % N_LAYERS]
         budget = pc.pc_plan_budget(b.kind, b.param, b.total, b.keep_full, avail)
         pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget, scores=scores, sel_idx=sel, stream=stream)
@@ -250,7 +256,7 @@ def run_cuda(args):
     for i in range(max(args.warmup, 3)):
         step(i)
     barrier()
-    assert pc.pc_poll_status(ctx) == pc.PC_OK, "device-side error during warm-up"
+    assert all(pc.pc_poll_status(c) == pc.PC_OK for c in ctxs), "device-side error during warm-up"
     sampler.start()
 
     # ---- timed region: K steps, device time between two events on the launching stream
@@ -264,18 +270,32 @@ def run_cuda(args):
     ms_total = e0.elapsed_time(e1)
     ms_total = max_over_ranks(ms_total, dist, "cuda")
     ms_step = ms_total / args.steps
-    assert pc.pc_poll_status(ctx) == pc.PC_OK, "device-side error in the timed region"
+    assert all(pc.pc_poll_status(c) == pc.PC_OK for c in ctxs), "device-side error in the timed region"
 
     # ---- per-kernel durations (CUDA events recorded by the library at kernel boundaries, same steps again)
-    pc.pc_set_timing(ctx, True)
+    for c in ctxs:
+        pc.pc_set_timing(c, True)
     acc = {k: [] for k in pc.STAGES}
     for i in range(min(args.steps, 200)):
         step(i)
-        for k, v in pc.pc_get_timing(ctx).items():
+        for k, v in pc.pc_get_timing(ctxs[i % N_LAYERS]).items():
             if v >= 0:
                 acc[k].append(v)
-    pc.pc_set_timing(ctx, False)
+    for c in ctxs:
+        pc.pc_set_timing(c, False)
     kern_ms = {k: (float(np.mean(v)) if v else None) for k, v in acc.items()}
+
+    # ---- the same frame through the three separate calls (pc_score, pc_compact, pc_attend_frame: eight launches)
+    for i in range(3):
+        step_separate(i)
+    barrier()
+    n_sep = min(args.steps, 200)
+    e0.record(stream)
+    for i in range(n_sep):
+        step_separate(i)
+    e1.record(stream)
+    barrier()
+    sep_ms = max_over_ranks(e0.elapsed_time(e1) / n_sep, dist, "cuda")
 
     # ---- one further attention pass over an unchanged cache (a frame is generated over several diffusion steps that all
     # attend to the same keys): keys rotated once by pc_attend_prepare, each pass rotates only its queries
@@ -429,6 +449,8 @@ def run_cuda(args):
                      "peak_source": f"{peaks['source']} (burst; sustained {peaks['bf16_tflops_sustained']})",
                      "flops_per_launch": flops, "ms_per_launch": att_ms},
         "kernels_ms": stages,
+        "separate_calls": {"ms_per_frame": sep_ms, "what": "the same frame through pc_score, pc_compact and pc_attend_frame "
+                           "(eight launches: Q read twice, rotary pre-pass over anchors and packed history)"},
         "extra_pass": {"ms_per_pass": pass_ms, "what": "one more attention pass of the frame over the unchanged packed cache "
                        "(pc_attend_prepared: query rotation, attention, merge; keys were rotated once per frame)"},
         "attention_mass": {"ms": mass_ms, "keys": cfg.n_anchor + n_sel,

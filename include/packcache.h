@@ -174,6 +174,25 @@ pc_status pc_attend_prepare(pc_ctx *ctx, const pc_cache *cache, const pc_segment
 pc_status pc_attend_prepared(pc_ctx *ctx, const void *q, const int32_t *q_pos, int32_t n_q, void *out, float *lse,
                              void *stream);
 
+/* One frame of the steady state in one call (Fig. 6b-c: score, keep each frame's quota, pack, then attend with Eq. 2):
+ * the same results as pc_score (no mask, no override) -> pc_compact -> pc_attend_frame over src's anchors ++ the packed
+ * history, with q serving both the scores and the attention.  What the one call saves on the bf16 tensor-core path: Q is
+ * read and rotated once (the pass that pools it for the scores also leaves the rotated queries of Eq. 2), the pack
+ * kernel also leaves the rotated keys of the rows it packs (at their rebased positions, Eq. 9), and the anchors'
+ * rotated keys are kept in the context from the first step that sees an anchor segment (same k / pos pointers and
+ * token count) — anchors never move (Sec. 3.4, condition anchoring) — so attention starts without a rotary pre-pass.
+ * Outputs are bit-identical to the three separate calls.
+ *   budget host [src.n_frames] (from pc_plan_budget); dst: its history buffers receive the packed rows, its
+ *   history.n_tokens and n_frames are set to sum(budget) and src.n_frames (frame_count is left to the caller), its
+ *   anchors field is ignored; scores device out [n_src]; sel_idx device out [sum(budget)]; out, lse as pc_attend_frame.
+ * Call pc_forget_anchors after changing the anchors' K or positions in place; pc_attend_frame / pc_attend_prepare on
+ * the same context drop the kept anchor keys as well (they are rebuilt by the next step).
+ * Errors: as the three calls. */
+pc_status pc_frame_step(pc_ctx *ctx, const pc_cache *src, const int32_t *budget, int32_t delta_t, pc_cache *dst,
+                        const void *q, const int32_t *q_pos, int32_t n_q, float *scores, int32_t *sel_idx, void *out,
+                        float *lse, void *stream);
+pc_status pc_forget_anchors(pc_ctx *ctx);
+
 /* Attention mass of every key (Sec. 3.4: retention is guided by the attention a cached token receives):
  *   mass_j = 1/(n_q*Hq) * sum over the query rows (i, h) of softmax_j((R q_ih).(R k_j,g(h))/sqrt(d)),
  * the mean, over the frame's queries and heads, of the probabilities of Eq. 2; the masses of all keys sum to one.
@@ -227,8 +246,8 @@ pc_status pc_frame_step_host(pc_ctx *ctx, const pc_host_frame *in, pc_device_wor
  * was given to an arena of their own at start-up and driver allocations are forbidden afterwards, or they sit on a
  * latency-critical thread that cannot take the device-wide synchronisation an allocation or a free implies — and so
  * cannot create a pc_ctx either.  This call needs no context and calls neither cudaMalloc nor cudaFree nor any
- * allocating routine: the rotary table, the pooled query and its reduction scratch live in one fixed device array
- * of 790,784 bytes that is part of the library image (every GPU that loads the library holds it until exit).
+ * allocating routine: the rotary table and the accumulator of the pooled query live in one fixed device array
+ * of 270,592 bytes that is part of the library image (every GPU that loads the library holds it until exit).
  *
  * Computes the same scores as pc_score (mean scaled rotary logit of every history token over the n_q queries and
  * all query heads, fp32); selection is not included.  desc->max_q / max_keys are ignored.
@@ -240,7 +259,7 @@ pc_status pc_frame_step_host(pc_ctx *ctx, const pc_host_frame *in, pc_device_wor
  * sum over the three axes of max_pos[a] * (rotary pairs on axis a) <= 32768; n_q_heads*head_dim <= 12288.
  * The first call on each device looks up the array's device address (that device must be current); make that
  * first call outside any stream capture.  All calls share the one array, which keeps the previous call's
- * contents (the call rewrites or clears what it relies on): two calls that may overlap on the GPU — different
+ * contents (the call rewrites the table and clears the accumulator before it uses them): two calls that may overlap on the GPU — different
  * streams without an ordering between them — race; order them.  Work is asynchronous on the given stream.
  * Other errors: PC_ERR_INVALID_ARG (null or misaligned pointer, n_src or n_q <= 0), PC_ERR_UNSUPPORTED, PC_ERR_CUDA. */
 pc_status pc_score_tokens_static(const pc_layer_desc *desc, const void *hist_k, const int32_t *hist_pos,
@@ -312,10 +331,7 @@ pc_status pc_window_state(pc_window *w, int32_t *n_frames, int32_t *counts, int6
 pc_status pc_poll_status(pc_ctx *ctx, void *stream);
 
 /* Choose the bf16 attention kernel: 0 = tcgen05 tensor-core kernel (default), 1 = CUDA-core kernel (a slow second
- * opinion), 2 = tcgen05 kernel that issues its multiply-adds for pairs of CTAs (cta_group::2: the two CTAs of a cluster
- * share every key / value tile, each loading half of it; used when the query tiles per KV head divide by four, else as
- * 0).  2 gives the bits of 0; on a B200 it is slower at the shapes measured (the pair's barrier traffic crosses SMs on
- * every tile) and is kept for comparison.  Returns PC_ERR_INVALID_ARG otherwise. */
+ * opinion).  Returns PC_ERR_INVALID_ARG otherwise. */
 pc_status pc_set_attend_impl(pc_ctx *ctx, int32_t impl);
 
 /* Fix the number of key ranges the tensor-core attention kernel splits the keys into (1..4); 0 lets each call
@@ -329,11 +345,20 @@ pc_status pc_set_kv_splits(pc_ctx *ctx, int32_t n);
  * number of work items fits that; results agree up to fp32 rounding order. */
 pc_status pc_set_cluster_merge(pc_ctx *ctx, int32_t on);
 
+/* Limit of every bounded device-side wait of the context's tensor-core attention kernel, in microseconds (0 = the
+ * default of about one second).  A wait that runs out records PC_ERR_TIMEOUT in the status word, the CTA gives up its
+ * remaining work, lets its copies land, frees its tensor memory and exits; the context stays usable. */
+pc_status pc_set_wait_limit_us(pc_ctx *ctx, uint32_t limit_us);
+/* Test hook for that path: the attention kernel's first barrier of every CTA is told to expect n_bytes more than are
+ * ever sent, so its wait runs out after the limit above and pc_poll_status returns PC_ERR_TIMEOUT; the call's output
+ * is then undefined.  0 switches the hook off.  Nothing traps and nothing waits without a limit. */
+pc_status pc_test_expect_extra_bytes(pc_ctx *ctx, uint32_t n_bytes);
+
 /* Per-kernel timing for benchmarks.  With timing on, each call records CUDA events on its stream at the boundaries
  * of its kernels (a few microseconds of overhead per call); pc_get_timing waits for the last recorded events and
  * writes the duration in milliseconds of each kernel of the most recent calls, -1 for a kernel that did not run.
  * ms is a host array [PC_N_STAGES]. */
-enum { PC_STAGE_QPOOL = 0, PC_STAGE_SCORE = 1, PC_STAGE_SELECT = 2, PC_STAGE_PACK = 3, PC_STAGE_ROPE = 4,
+enum { PC_STAGE_QPOOL = 0 /* the query pass */, PC_STAGE_SCORE = 1, PC_STAGE_SELECT = 2, PC_STAGE_PACK = 3, PC_STAGE_ROPE = 4,
        PC_STAGE_ATTEND = 5, PC_STAGE_COMBINE = 6, PC_STAGE_MASS = 7, PC_N_STAGES = 8 };
 pc_status pc_set_timing(pc_ctx *ctx, int32_t on);
 pc_status pc_get_timing(pc_ctx *ctx, float *ms);

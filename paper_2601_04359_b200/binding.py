@@ -25,7 +25,8 @@ EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact"
            "pc_poll_status", "pc_set_attend_impl", "pc_set_kv_splits", "pc_set_timing", "pc_get_timing",
            "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge",
            "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_append_masked", "pc_window_update", "pc_window_cache",
-           "pc_window_state", "pc_attend_prepare", "pc_attend_prepared", "pc_attend_mass"]
+           "pc_window_state", "pc_attend_prepare", "pc_attend_prepared", "pc_attend_mass", "pc_frame_step",
+           "pc_forget_anchors", "pc_set_wait_limit_us", "pc_test_expect_extra_bytes"]
 
 
 class pc_layer_desc(C.Structure):
@@ -110,6 +111,11 @@ def load() -> C.CDLL:
     lib.pc_attend_prepare.argtypes = [C.c_void_p, C.POINTER(pc_cache), C.POINTER(pc_segment), C.c_void_p]
     lib.pc_attend_prepared.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.pc_attend_mass.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+    lib.pc_frame_step.argtypes = [C.c_void_p, C.POINTER(pc_cache), C.POINTER(C.c_int32), C.c_int32, C.POINTER(pc_cache),
+                                  C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.pc_forget_anchors.argtypes = [C.c_void_p]
+    lib.pc_set_wait_limit_us.argtypes = [C.c_void_p, C.c_uint32]
+    lib.pc_test_expect_extra_bytes.argtypes = [C.c_void_p, C.c_uint32]
     lib.pc_window_create.argtypes = [C.c_void_p, C.POINTER(pc_window_params), C.POINTER(pc_segment), C.POINTER(pc_segment),
                                      C.POINTER(pc_segment), C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p)]
     lib.pc_window_destroy.argtypes = [C.c_void_p]
@@ -253,6 +259,39 @@ def pc_attend_frame(ctx: Context, cache: Cache, current: Optional[Segment], q: t
     _check(load().pc_attend_frame(ctx.handle, C.byref(c), C.byref(cur) if cur is not None else None, _ptr(q),
                                   _ptr(q_pos), q.shape[0], _ptr(out), _ptr(lse), _stream(stream)), "pc_attend_frame")
     return (out, lse) if want_lse else out
+
+
+def pc_frame_step(ctx: Context, src: Cache, budget, delta_t: int, dst: Cache, q: torch.Tensor, q_pos: torch.Tensor,
+                  scores: Optional[torch.Tensor] = None, sel_idx: Optional[torch.Tensor] = None,
+                  out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None, want_lse: bool = False, stream=None):
+    """score -> select -> pack -> attend in one call; returns (out, scores, sel_idx[, lse]); dst receives the packed rows."""
+    budget = _i32(budget)
+    if scores is None:
+        scores = torch.empty(max(src.history.n_tokens, 1), dtype=torch.float32, device=q.device)
+    if sel_idx is None:
+        sel_idx = torch.empty(max(int(budget.sum()), 1), dtype=torch.int32, device=q.device)
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None and want_lse:
+        lse = torch.empty(q.shape[0], q.shape[1], dtype=torch.float32, device=q.device)
+    cs, cd = src.c(), dst.c()
+    _check(load().pc_frame_step(ctx.handle, C.byref(cs), _i32p(budget), delta_t, C.byref(cd), _ptr(q), _ptr(q_pos), q.shape[0],
+                                _ptr(scores), _ptr(sel_idx), _ptr(out), _ptr(lse), _stream(stream)), "pc_frame_step")
+    dst.history.n_tokens = int(budget.sum())
+    dst.frame_count = budget.copy()
+    return (out, scores, sel_idx, lse) if want_lse else (out, scores, sel_idx)
+
+
+def pc_forget_anchors(ctx: Context) -> None:
+    _check(load().pc_forget_anchors(ctx.handle), "pc_forget_anchors")
+
+
+def pc_set_wait_limit_us(ctx: Context, limit_us: int) -> None:
+    _check(load().pc_set_wait_limit_us(ctx.handle, limit_us), "pc_set_wait_limit_us")
+
+
+def pc_test_expect_extra_bytes(ctx: Context, n_bytes: int) -> None:
+    _check(load().pc_test_expect_extra_bytes(ctx.handle, n_bytes), "pc_test_expect_extra_bytes")
 
 
 def pc_attend_prepare(ctx: Context, cache: Cache, current: Optional[Segment] = None, stream=None) -> None:

@@ -32,31 +32,8 @@ extern "C" const char *pc_status_string(pc_status s) {
 
 static int pairs_of_axis(int n_pairs, int axis) { return (n_pairs - axis + 2) / 3; }
 
-extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
-    if (!desc || !out) return PC_ERR_INVALID_ARG;
-    *out = nullptr;
-    if (desc->head_dim != 64 && desc->head_dim != 128) return PC_ERR_UNSUPPORTED;
-    if (desc->dtype != PC_F32 && desc->dtype != PC_BF16) return PC_ERR_UNSUPPORTED;
-    if (desc->n_q_heads <= 0 || desc->n_kv_heads <= 0 || desc->n_q_heads % desc->n_kv_heads) return PC_ERR_UNSUPPORTED;
-    if (desc->n_kv_heads * desc->head_dim > 4096) return PC_ERR_UNSUPPORTED;
-    if (!(desc->rope_base > 1.0)) return PC_ERR_INVALID_ARG;
-    if (desc->max_q <= 0 || desc->max_keys <= 0) return PC_ERR_INVALID_ARG;
-    for (int a = 0; a < 3; ++a)
-        if (desc->max_pos[a] <= 0 || desc->max_pos[a] > (1 << 20)) return PC_ERR_INVALID_ARG;
-
-    pc_ctx *c = new (std::nothrow) pc_ctx();
-    if (!c) return PC_ERR_CUDA;
-    c->desc = *desc;
-    c->group = desc->n_q_heads / desc->n_kv_heads;
-    c->elem_size = desc->dtype == PC_BF16 ? 2 : 4;
-    c->attend_impl = 0;
-    c->kv_splits = 0;
-    c->cluster_merge = 0;
-    c->prepared_n_seg = 0;
-    c->last_n_q = c->last_n_seg = 0;
-    c->timing_on = 0;
-    c->ev_mask = 0;
-    for (int i = 0; i < PC_N_MARKS; ++i) c->ev[i] = nullptr;
+static pc_status create_on_device(pc_ctx *c) {
+    const pc_layer_desc *desc = &c->desc;
     PC_CUDA_TRY(cudaGetDevice(&c->device));
     PC_CUDA_TRY(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
 
@@ -87,8 +64,8 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
     PC_CUDA_TRY(cudaMalloc(&c->status, 2 * sizeof(int32_t)));
     PC_CUDA_TRY(cudaMemset(c->status, 0, 2 * sizeof(int32_t)));
     PC_CUDA_TRY(cudaMallocHost(&c->host_status, 2 * sizeof(int32_t)));
-    PC_CUDA_TRY(cudaMalloc(&c->qpool_partial, (size_t)PC_QPOOL_BLOCKS * row * sizeof(float)));
-    PC_CUDA_TRY(cudaMalloc(&c->qpool, (size_t)row * sizeof(float)));
+    PC_CUDA_TRY(cudaMalloc(&c->qpool_fx, 2 * (size_t)row * sizeof(long long)));
+    PC_CUDA_TRY(cudaMemset(c->qpool_fx, 0, 2 * (size_t)row * sizeof(long long)));
     if (desc->dtype == PC_BF16) {
         pc_status st = pc_attend_tc_scratch(desc, c->sm_count, &c->k_rot_rows, &c->part_o_floats, &c->part_ml_floats);
         if (st != PC_OK) return st;
@@ -100,6 +77,31 @@ extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
         PC_CUDA_TRY(cudaMalloc(&c->mass_part, c->k_rot_rows * desc->n_kv_heads * 2 * sizeof(float)));
         PC_CUDA_TRY(cudaMalloc(&c->mass_norm, (size_t)((desc->max_q + 127) / 128) * 128 * desc->n_q_heads * sizeof(float)));
     }
+    return PC_OK;
+}
+
+extern "C" pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out) {
+    if (!desc || !out) return PC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (desc->head_dim != 64 && desc->head_dim != 128) return PC_ERR_UNSUPPORTED;
+    if (desc->dtype != PC_F32 && desc->dtype != PC_BF16) return PC_ERR_UNSUPPORTED;
+    if (desc->n_q_heads <= 0 || desc->n_kv_heads <= 0 || desc->n_q_heads % desc->n_kv_heads) return PC_ERR_UNSUPPORTED;
+    if (desc->n_kv_heads * desc->head_dim > 4096) return PC_ERR_UNSUPPORTED;
+    if (!(desc->rope_base > 1.0)) return PC_ERR_INVALID_ARG;
+    if (desc->max_q <= 0 || desc->max_keys <= 0) return PC_ERR_INVALID_ARG;
+    for (int a = 0; a < 3; ++a)
+        if (desc->max_pos[a] <= 0 || desc->max_pos[a] > (1 << 20)) return PC_ERR_INVALID_ARG;
+
+    pc_ctx *c = new (std::nothrow) pc_ctx();       // value-initialised: every pointer starts out null
+    if (!c) return PC_ERR_CUDA;
+    c->desc = *desc;
+    c->group = desc->n_q_heads / desc->n_kv_heads;
+    c->elem_size = desc->dtype == PC_BF16 ? 2 : 4;
+    const pc_status st = create_on_device(c);
+    if (st != PC_OK) {                             // one way out on failure: whatever was allocated so far is released
+        pc_destroy(c);
+        return st;
+    }
     *out = c;
     return PC_OK;
 }
@@ -108,9 +110,8 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
     if (!c) return PC_ERR_INVALID_ARG;
     cudaFree(c->rope_tab);
     cudaFree(c->status);
-    cudaFreeHost(c->host_status);
-    cudaFree(c->qpool_partial);
-    cudaFree(c->qpool);
+    if (c->host_status) cudaFreeHost(c->host_status);
+    cudaFree(c->qpool_fx);
     for (int i = 0; i < PC_N_MARKS; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     cudaFree(c->k_rot);
@@ -124,8 +125,26 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
 }
 
 extern "C" pc_status pc_set_attend_impl(pc_ctx *c, int32_t impl) {
-    if (!c || impl < 0 || impl > 2) return PC_ERR_INVALID_ARG;
+    if (!c || impl < 0 || impl > 1) return PC_ERR_INVALID_ARG;
     c->attend_impl = impl;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_set_wait_limit_us(pc_ctx *c, uint32_t limit_us) {
+    if (!c) return PC_ERR_INVALID_ARG;
+    c->wait_limit_us = limit_us;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_test_expect_extra_bytes(pc_ctx *c, uint32_t n_bytes) {
+    if (!c) return PC_ERR_INVALID_ARG;
+    c->test_extra_tx = n_bytes;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_forget_anchors(pc_ctx *c) {
+    if (!c) return PC_ERR_INVALID_ARG;
+    c->anchor_rot_n = 0;
     return PC_OK;
 }
 
@@ -153,13 +172,17 @@ extern "C" pc_status pc_set_timing(pc_ctx *c, int32_t on) {
 
 extern "C" pc_status pc_get_timing(pc_ctx *c, float *ms) {
     if (!c || !ms) return PC_ERR_INVALID_ARG;
+    // (first mark, last mark) of each stage; the attention kernel starts at the rotary pre-pass's end mark when that
+    // pre-pass ran in the call, else at the call's first mark
     static const int span[PC_N_STAGES][2] = {{PC_MARK_SCORE0, PC_MARK_QPOOL}, {PC_MARK_QPOOL, PC_MARK_SCORE},
                                              {PC_MARK_SCORE, PC_MARK_SELECT}, {PC_MARK_PACK0, PC_MARK_PACK},
                                              {PC_MARK_ATT0, PC_MARK_ROPE},    {PC_MARK_ROPE, PC_MARK_ATTEND},
                                              {PC_MARK_ATTEND, PC_MARK_COMBINE}, {PC_MARK_MASS0, PC_MARK_MASS}};
     for (int s = 0; s < PC_N_STAGES; ++s) {
         ms[s] = -1.f;
-        const int a = span[s][0], b = span[s][1];
+        int a = span[s][0];
+        const int b = span[s][1];
+        if (s == PC_STAGE_ATTEND && !((c->ev_mask >> a) & 1u)) a = PC_MARK_ATT0;
         if (!((c->ev_mask >> a) & 1u) || !((c->ev_mask >> b) & 1u)) continue;
         PC_CUDA_TRY(cudaEventSynchronize(c->ev[b]));
         PC_CUDA_TRY(cudaEventElapsedTime(&ms[s], c->ev[a], c->ev[b]));

@@ -47,6 +47,8 @@ struct TcParams {
     int n_q, n_q_heads, group, n_tb, tiles_per_g, pairs_per_g, n_splits, n_kv_tiles;
     int n_seg;
     int cluster;      // 1: the KV ranges of one item form a thread-block cluster and merge through shared memory
+    uint32_t wait_us; // limit of every bounded wait in microseconds (0 = about one second)
+    uint32_t extra_tx; // test hook: bytes the first barrier expects beyond what is sent, so that its wait runs out (0 = off)
     int seg_tile_end[PC_MAX_SEGMENTS];
     int seg_n[PC_MAX_SEGMENTS];
     __nv_bfloat16 *out;
@@ -84,8 +86,8 @@ __device__ __forceinline__ void rope_row(const RopeJob &J, int row, int lane, co
         uint32_t o[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const float x0 = pc_bf16_lo(w[u]), x1 = pc_bf16_hi(w[u]);
-            o[u] = pc_pack_bf16(x0 * cs[u].x - x1 * cs[u].y, x0 * cs[u].y + x1 * cs[u].x);
+            const float2 y = pc_rotate(pc_bf16_lo(w[u]), pc_bf16_hi(w[u]), cs[u]);
+            o[u] = pc_pack_bf16(y.x, y.y);
         }
         dst[c * 32] = make_uint4(o[0], o[1], o[2], o[3]);
     }
@@ -127,8 +129,8 @@ __global__ void __launch_bounds__(256) k_rope_rows(const __grid_constant__ RopeJ
             uint32_t o[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const float x0 = pc_bf16_lo(w[u]), x1 = pc_bf16_hi(w[u]);
-                o[u] = pc_pack_bf16(x0 * cs[u].x - x1 * cs[u].y, x0 * cs[u].y + x1 * cs[u].x);
+                const float2 y = pc_rotate(pc_bf16_lo(w[u]), pc_bf16_hi(w[u]), cs[u]);
+                o[u] = pc_pack_bf16(y.x, y.y);
             }
             *dst = make_uint4(o[0], o[1], o[2], o[3]);
         }
@@ -202,7 +204,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             // The first K tile rides with the query tiles.  After that V(j) and K(j+1) always travel together: they are
             // needed at the same point (top of step j) and their stages are released at the same point (end of step j),
             // so one full / empty barrier pair serves both and the issuer has one wait and one commit less per step.
-            mbar_expect_tx(bar(BAR_Q), (n_tiles_q + (n_j > 0 ? 1 : 0)) * TILE_BYTES);
+            mbar_expect_tx(bar(BAR_Q), (n_tiles_q + (n_j > 0 ? 1 : 0)) * TILE_BYTES + P.extra_tx);
             for (int t = 0; t < n_tiles_q; ++t) {
                 const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
                 tma_load_2d(base + SM_Q + t * TILE_BYTES, &map_q, h * TILE, tb * TILE, bar(BAR_Q));
@@ -218,8 +220,8 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 int seg, local, n_valid;
                 kv_tile_info(P, jt0 + j, seg, local, n_valid);
                 const CUtensorMap *mv = seg == 0 ? &map_v0 : (seg == 1 ? &map_v1 : &map_v2);
-                if (use > 0) alive = mbar_wait(bar(BAR_VEMPTY + st), (use - 1) & 1, abort_flag, P.status);
-                else if (j == 1) alive = mbar_wait(bar(BAR_KEMPTY + 0), 0, abort_flag, P.status);   // K(2) lands where K(0) was
+                if (use > 0) alive = mbar_wait(bar(BAR_VEMPTY + st), (use - 1) & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
+                else if (j == 1) alive = mbar_wait(bar(BAR_KEMPTY + 0), 0, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);   // K(2) lands where K(0) was
                 if (!alive) break;
                 const bool more = j + 1 < n_j;
                 mbar_expect_tx(bar(BAR_VFULL + st), (more ? 2 : 1) * TILE_BYTES);
@@ -243,7 +245,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         reg_dealloc<72>();
         const bool lead = elect_one();
         const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-        bool alive = mbar_wait(bar(BAR_Q), 0, abort_flag, P.status);
+        bool alive = mbar_wait(bar(BAR_Q), 0, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
         auto issue_qk = [&](int t, int st) {
             const uint32_t qa = base + SM_Q + t * TILE_BYTES, ka = base + SM_K + st * TILE_BYTES;
 #pragma unroll
@@ -263,12 +265,12 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         for (int j = 0; j < n_j && alive; ++j) {
             const int st = j % KV_STAGES, use = j / KV_STAGES;
             const int nst = (j + 1) % KV_STAGES;
-            alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status);      // V(j) and K(j+1)
+            alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);      // V(j) and K(j+1)
             for (int t = 0; t < n_tiles_q && alive; ++t) {
                 const uint32_t va = base + SM_V + st * TILE_BYTES;
                 // P arrives in two halves of 64 keys: the first PV steps run while the rest is exponentiated
                 for (int hf = 0; hf < 2 && alive; ++hf) {
-                    alive = mbar_wait(bar(BAR_PHALF + 2 * t + hf), j & 1, abort_flag, P.status);
+                    alive = mbar_wait(bar(BAR_PHALF + 2 * t + hf), j & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
                     if (!alive) break;
                     tc_fence_after();
 #pragma unroll
@@ -289,7 +291,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         // make sure nothing of ours is still running on the tensor core before TMEM is freed
         if (lead) tc_commit(bar(BAR_DONE));
         __syncwarp();
-        mbar_wait(bar(BAR_DONE), 0, abort_flag, P.status);
+        mbar_wait(bar(BAR_DONE), 0, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
     } else if (warp < 4) {
         reg_dealloc<72>();
     } else {
@@ -306,7 +308,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         for (int j = 0; j < n_j && alive; ++j) {
             int seg, local, n_valid;
             kv_tile_info(P, jt0 + j, seg, local, n_valid);
-            alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), j & 1, abort_flag, P.status));
+            alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), j & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us));
             if (!alive) break;
             tc_fence_after();
             // the whole score row of this thread: one TMEM pass
@@ -376,7 +378,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             l += (la.x + la.y) + (lb.x + lb.y);
         }
         // epilogue: O_t is final once the last PV has committed
-        if (alive && n_j > 0) alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), n_j & 1, abort_flag, P.status));
+        if (alive && n_j > 0) alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), n_j & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us));
         if (alive && n_j > 0) {
             tc_fence_after();
             const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
@@ -487,302 +489,6 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     }
 }
 
-// ------------------------------------------------------------------------------------------------ CTA-pair kernel
-// The same attention with the multiply-adds issued for a pair of CTAs at once (`cta_group::2`, M = 256): the two CTAs
-// of a cluster hold two query tiles each, all four of one KV head, and share every key / value tile: each CTA loads
-// only its half of the B operands — 64 of the 128 keys of a K tile (N of S = Q K^T), 64 of the 128 head-dim columns of
-// a V tile (N of O += P V) — and the tensor cores of both read both halves.  Per key tile a CTA then moves 160 KB
-// through its shared memory instead of 256 KB; in k_attend_tc that traffic alone takes as long as the multiply-adds.
-// The even CTA issues every multiply-add and owns the "full" barriers (both CTAs' TMA loads count their bytes there,
-// both CTAs' softmax warps arrive there); completion is committed to the barriers of both CTAs at once.
-// Used when every CTA has two whole query tiles (tiles per head group divisible by four).  Results are bit-identical to
-// k_attend_tc.  Measured on a B200 it is slower (139 us against 100 us at 9,200 keys): the S-ready commit to the peer and
-// the peer's P-ready arrivals cross SMs on every tile and lengthen the chain the loop is bound by (about 5,000 cycles
-// per key tile against 3,300), and only about 72 clusters of two are resident.  Opt-in through pc_set_attend_impl.
-constexpr int K_HALF_BYTES = 64 * 64 * 2;                 // [64 keys][64 head-dim elements] box: 8 KB
-constexpr int K_SHARE_BYTES = 2 * K_HALF_BYTES;           // this CTA's 64 keys of a key tile
-constexpr int V_SHARE_BYTES = HALF_BYTES;                 // this CTA's 64 head-dim columns of a value tile: [128 keys][64]
-constexpr int SP_Q = 0;                                   // 2 query tiles
-constexpr int SP_K = SP_Q + 2 * TILE_BYTES;
-constexpr int SP_V = SP_K + KV_STAGES * K_SHARE_BYTES;
-constexpr int SP_BAR = SP_V + KV_STAGES * V_SHARE_BYTES;
-constexpr int SP_TOTAL = SP_BAR + 256;
-constexpr int SP_ALLOC = SP_TOTAL + 1024;
-
-__global__ void __launch_bounds__(TC_THREADS, 1)
-k_attend_tc_pair(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k64,
-                 const __grid_constant__ CUtensorMap map_v0, const __grid_constant__ CUtensorMap map_v1,
-                 const __grid_constant__ CUtensorMap map_v2, const __grid_constant__ TcParams P) {
-    pc_grid_dep_launch();
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(gen + SP_BAR + N_BARS * 8);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(gen + SP_BAR + N_BARS * 8 + 8);
-    const uint32_t bar0 = base + SP_BAR;
-    auto bar = [&](int i) { return bar0 + 8u * i; };
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_rank();                       // 0: the CTA that issues the pair's multiply-adds
-    const int cl = blockIdx.x >> 1;                             // cluster = (group of four query tiles, key range)
-    const int pitem = cl / P.n_splits, split = cl % P.n_splits;
-    const int item = 2 * pitem + (int)rank;                     // this CTA's two query tiles, numbered as in k_attend_tc
-    const int g = item / P.pairs_per_g, pair = item % P.pairs_per_g;
-    const int jt0 = (int)(((long long)P.n_kv_tiles * split) / P.n_splits);
-    const int jt1 = (int)(((long long)P.n_kv_tiles * (split + 1)) / P.n_splits);
-    const int n_j = jt1 - jt0;
-
-    if (threadIdx.x == 0) {
-        mbar_init(bar(BAR_Q), 1);
-        for (int s = 0; s < KV_STAGES; ++s) {
-            mbar_init(bar(BAR_KFULL + s), 1);
-            mbar_init(bar(BAR_KEMPTY + s), 1);
-            mbar_init(bar(BAR_VFULL + s), 1);
-            mbar_init(bar(BAR_VEMPTY + s), 1);
-        }
-        for (int t = 0; t < 2; ++t) {
-            mbar_init(bar(BAR_SFULL + t), 1);
-            mbar_init(bar(BAR_PHALF + 2 * t), 256);             // the softmax warps of both CTAs
-            mbar_init(bar(BAR_PHALF + 2 * t + 1), 256);
-        }
-        mbar_init(bar(BAR_DONE), 1);
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 2) {   // TMEM: all 512 columns, in both CTAs of the pair at once
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();        // the peer's barriers exist before anything of ours can reach them
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    pc_grid_dep_wait();
-
-    if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer (both CTAs: own tiles, own halves)
-        reg_dealloc<72>();
-        if (lane == 0) {
-            const uint32_t lead_q = peer_addr(bar(BAR_Q), 0);
-            if (rank == 0) mbar_expect_tx(bar(BAR_Q), 4 * TILE_BYTES + (n_j > 0 ? TILE_BYTES : 0));   // four query tiles, one key tile
-            for (int t = 0; t < 2; ++t) {
-                const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
-                tma_load_2d_pair(base + SP_Q + t * TILE_BYTES, &map_q, h * TILE, tb * TILE, lead_q);
-                tma_load_2d_pair(base + SP_Q + t * TILE_BYTES + HALF_BYTES, &map_q, h * TILE + 64, tb * TILE, lead_q);
-            }
-            if (n_j > 0) {
-                tma_load_2d_pair(base + SP_K, &map_k64, g * TILE, jt0 * TILE + (int)rank * 64, lead_q);
-                tma_load_2d_pair(base + SP_K + K_HALF_BYTES, &map_k64, g * TILE + 64, jt0 * TILE + (int)rank * 64, lead_q);
-            }
-            bool alive = true;
-            for (int j = 0; j < n_j && alive; ++j) {
-                const int st = j % KV_STAGES, use = j / KV_STAGES, kst = (j + 1) % KV_STAGES;
-                int seg, local, n_valid;
-                kv_tile_info(P, jt0 + j, seg, local, n_valid);
-                const CUtensorMap *mv = seg == 0 ? &map_v0 : (seg == 1 ? &map_v1 : &map_v2);
-                if (use > 0) alive = mbar_wait(bar(BAR_VEMPTY + st), (use - 1) & 1, abort_flag, P.status);
-                else if (j == 1) alive = mbar_wait(bar(BAR_KEMPTY + 0), 0, abort_flag, P.status);   // K(2) lands where K(0) was
-                if (!alive) break;
-                const bool more = j + 1 < n_j;
-                const uint32_t lead_v = peer_addr(bar(BAR_VFULL + st), 0);
-                if (rank == 0) mbar_expect_tx(bar(BAR_VFULL + st), (more ? 2 : 1) * TILE_BYTES);      // both CTAs' shares
-                tma_load_2d_pair(base + SP_V + st * V_SHARE_BYTES, mv, g * TILE + (int)rank * 64, local * TILE, lead_v);
-                if (more) {
-                    const int row = (jt0 + j + 1) * TILE + (int)rank * 64;
-                    tma_load_2d_pair(base + SP_K + kst * K_SHARE_BYTES, &map_k64, g * TILE, row, lead_v);
-                    tma_load_2d_pair(base + SP_K + kst * K_SHARE_BYTES + K_HALF_BYTES, &map_k64, g * TILE + 64, row, lead_v);
-                }
-            }
-            if (*abort_flag) {
-                const uint64_t t0 = global_ns();
-                while (global_ns() - t0 < 2000000ull) {}
-            }
-        }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer: the even CTA, for both
-        reg_dealloc<72>();
-        if (rank == 0) {
-            const bool lead = elect_one();
-            const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-            bool alive = mbar_wait_cluster(bar(BAR_Q), 0, abort_flag, P.status);
-            auto issue_qk = [&](int t, int st) {
-                const uint32_t qa = base + SP_Q + t * TILE_BYTES, ka = base + SP_K + st * K_SHARE_BYTES;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t qoff = (ks >> 2) * HALF_BYTES + (ks & 3) * 32, koff = (ks >> 2) * K_HALF_BYTES + (ks & 3) * 32;
-                    if (lead) mma_ss_pair(tm + t * TILE, desc_kmajor(qa + qoff), desc_kmajor(ka + koff), IDESC_PAIR_QK, ks > 0);
-                }
-            };
-            if (alive && n_j > 0) {
-                tc_fence_after();
-                for (int t = 0; t < 2; ++t) {
-                    issue_qk(t, 0);
-                    if (lead) tc_commit_pair(bar(BAR_SFULL + t));
-                }
-                if (lead) tc_commit_pair(bar(BAR_KEMPTY + 0));
-            }
-            for (int j = 0; j < n_j && alive; ++j) {
-                const int st = j % KV_STAGES, use = j / KV_STAGES, nst = (j + 1) % KV_STAGES;
-                alive = mbar_wait_cluster(bar(BAR_VFULL + st), use & 1, abort_flag, P.status);      // V(j) and K(j+1), both shares
-                for (int t = 0; t < 2 && alive; ++t) {
-                    const uint32_t va = base + SP_V + st * V_SHARE_BYTES;
-                    for (int hf = 0; hf < 2 && alive; ++hf) {
-                        alive = mbar_wait_cluster(bar(BAR_PHALF + 2 * t + hf), j & 1, abort_flag, P.status);
-                        if (!alive) break;
-                        tc_fence_after();
-#pragma unroll
-                        for (int k4 = 0; k4 < 4; ++k4) {
-                            const int ks = hf * 4 + k4;
-                            if (lead)
-                                mma_ts_pair(tm + 256 + t * TILE, tm + t * TILE + ks * 8, desc_mnmajor64(va + ks * 2048), IDESC_PAIR_PV, (j > 0 || ks > 0));
-                        }
-                    }
-                    if (!alive) break;
-                    if (j + 1 < n_j) issue_qk(t, nst);
-                    if (lead) tc_commit_pair(bar(BAR_SFULL + t));
-                }
-                if (alive && lead) tc_commit_pair(bar(BAR_VEMPTY + st));
-            }
-            if (lead) tc_commit_pair(bar(BAR_DONE));
-            __syncwarp();
-        }
-        // nothing of the pair may still be running on either tensor core when TMEM is freed
-        mbar_wait(bar(BAR_DONE), 0, abort_flag, P.status);
-    } else if (warp < 4) {
-        reg_dealloc<72>();
-    } else {
-        // ---------------------------------------------------------------- softmax + correction + epilogue (as in k_attend_tc)
-        reg_alloc<208>();
-        const int t = (warp - 4) >> 2;
-        const int quad = warp & 3;
-        const int r = quad * 32 + lane;
-        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        const uint32_t s_addr = tmem + lane_addr + t * TILE;
-        const uint32_t o_addr = tmem + lane_addr + 256 + t * TILE;
-        const uint32_t lead_p = peer_addr(bar(BAR_PHALF + 2 * t), 0);          // the issuing CTA's barriers for this tile's P halves
-        float m_used = -INFINITY, l = 0.f;
-        bool alive = true;
-        for (int j = 0; j < n_j && alive; ++j) {
-            int seg, local, n_valid;
-            kv_tile_info(P, jt0 + j, seg, local, n_valid);
-            alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), j & 1, abort_flag, P.status));
-            if (!alive) break;
-            tc_fence_after();
-            uint32_t sv[128];
-            tmem_ld32(s_addr, sv);
-            tmem_ld32(s_addr + 32, sv + 32);
-            tmem_ld32(s_addr + 64, sv + 64);
-            tmem_ld32(s_addr + 96, sv + 96);
-            tmem_wait_ld();
-            if (n_valid < TILE) {
-#pragma unroll
-                for (int i = 0; i < TILE; ++i)
-                    if (i >= n_valid) sv[i] = 0xFF800000u;
-            }
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < TILE; i += 4) {
-                mx0 = fmaxf(mx0, __uint_as_float(sv[i]));
-                mx1 = fmaxf(mx1, __uint_as_float(sv[i + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(sv[i + 2]));
-                mx3 = fmaxf(mx3, __uint_as_float(sv[i + 3]));
-            }
-            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            const bool grow = mx > m_used + RESCALE_THRESHOLD;
-            if (__any_sync(0xffffffffu, grow)) {
-                const float m_new = fmaxf(m_used, mx);
-                const float corr = fast_exp2(m_used - m_new);
-                l *= corr;
-                if (j > 0) {
-                    uint32_t v[32];
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        tmem_ld32(o_addr + c * 32, v);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
-                        tmem_st32(o_addr + c * 32, v);
-                    }
-                }
-                m_used = m_new;
-            }
-            const float2 neg_m = make_float2(-m_used, -m_used);
-            float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    float2 x = add2(make_float2(__uint_as_float(sv[c * 32 + 2 * i]), __uint_as_float(sv[c * 32 + 2 * i + 1])), neg_m);
-                    float2 y = add2(make_float2(__uint_as_float(sv[c * 32 + 2 * i + 2]), __uint_as_float(sv[c * 32 + 2 * i + 3])), neg_m);
-                    x.x = fast_exp2(x.x); x.y = fast_exp2(x.y);
-                    y.x = fast_exp2(y.x); y.y = fast_exp2(y.y);
-                    la = add2(la, x);
-                    lb = add2(lb, y);
-                    pk[i] = pc_pack_bf16(x.x, x.y);
-                    pk[i + 1] = pc_pack_bf16(y.x, y.y);
-                }
-                tmem_st16(s_addr + c * 16, pk);
-                if (c & 1) {                               // keys 0-63, then 64-127, handed to the issuing CTA
-                    tmem_wait_st();
-                    tc_fence_before();
-                    mbar_arrive_cluster(lead_p + 8u * (c >> 1));
-                }
-            }
-            l += (la.x + la.y) + (lb.x + lb.y);
-        }
-        if (alive && n_j > 0) alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), n_j & 1, abort_flag, P.status));
-        if (alive && n_j > 0) {
-            tc_fence_after();
-            const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
-            const int row = tb * TILE + r;
-            uint32_t v[32];
-            if (P.n_splits == 1) {
-                const float inv = 1.f / l;
-                __nv_bfloat16 *orow = P.out + ((size_t)row * P.n_q_heads + h) * TILE;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    tmem_ld32(o_addr + c * 32, v);
-                    tmem_wait_ld();
-                    if (row < P.n_q) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            uint4 w;
-                            w.x = pc_pack_bf16(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
-                            w.y = pc_pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
-                            w.z = pc_pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
-                            w.w = pc_pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
-                            *reinterpret_cast<uint4 *>(orow + c * 32 + i * 8) = w;
-                        }
-                    }
-                }
-                if (P.lse && row < P.n_q) P.lse[(size_t)row * P.n_q_heads + h] = (m_used + log2f(l)) * 0.6931471805599453f;
-            } else {
-                const size_t tile_slot = ((size_t)item * P.n_splits + split) * 2 + t;      // where k_combine looks for it
-                uint4 *ptile = reinterpret_cast<uint4 *>(P.part_o) + tile_slot * (TILE * TILE / 4) + r;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    tmem_ld32(o_addr + c * 32, v);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        ptile[(c * 8 + i) * TILE] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                }
-                *reinterpret_cast<float2 *>(P.part_ml + (tile_slot * TILE + r) * 2) = make_float2(m_used, l);
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();        // neither CTA frees TMEM or leaves while the pair's multiply-adds or barrier traffic may still touch it
-    if (warp == 2) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
-    }
-}
-
 // ------------------------------------------------------------------------------------------------ combine
 // Merge of the KV ranges' partials.  One block per (query tile of one head, 32-row quadrant); its eight warps take four
 // 16-byte column units each, lanes are consecutive rows, so every load of the partial tiles is a 512-byte run.  Every
@@ -884,7 +590,7 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     if (k_chunks % 32 || q_chunks % 32) return PC_ERR_UNSUPPORTED;
     int tiles = 0, warps = 0, n_jobs = 0;
     for (int s = 0; s < n_seg; ++s) {
-        if (what & PC_TC_ROPE_K) {
+        if ((what & PC_TC_ROPE_K) || (s == 0 && (what & PC_TC_ROPE_K0))) {
             jobs.job[n_jobs++] = RopeJob{static_cast<const __nv_bfloat16 *>(segs[s].k), segs[s].pos,
                                          k_rot + (size_t)tiles * TILE * row_elems, segs[s].n_tokens, k_chunks, warps, 1, 1.0f};
             warps += segs[s].n_tokens;
@@ -899,17 +605,18 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
         // a query row is as many slices as it holds key-row widths when that divides evenly: every warp then has the same job
         const int slices = (q_chunks % k_chunks == 0) ? q_chunks / k_chunks : 1;
         jobs.job[n_jobs++] = RopeJob{static_cast<const __nv_bfloat16 *>(q), q_pos, q_rot, n_q * slices, q_chunks / slices, warps, slices,
-                                     (float)(1.4426950408889634 / std::sqrt((double)D.head_dim))};
+                                     pc_q_rot_scale(D.head_dim)};
         warps += n_q * slices;
     }
     jobs.n_jobs = n_jobs;
     jobs.total_warps = warps;
+    ctx->ev_mask &= ~((1u << PC_MARK_ATT0) | (1u << PC_MARK_ROPE) | (1u << PC_MARK_ATTEND) | (1u << PC_MARK_COMBINE));
     pc_mark(ctx, PC_MARK_ATT0, stream);
     if (n_jobs > 0) {
         PC_LAUNCH(k_rope_rows, dim3(div_up(warps, 8)), dim3(256), 0, stream, jobs, ctx->rope, D.head_dim, ctx->status);
         PC_CUDA_TRY(cudaGetLastError());
+        pc_mark(ctx, PC_MARK_ROPE, stream);          // no pre-pass (a fused frame step with cached anchors): no mark
     }
-    pc_mark(ctx, PC_MARK_ROPE, stream);
     if (!(what & PC_TC_ATTEND)) return PC_OK;
 
     P.n_q = n_q;
@@ -927,6 +634,8 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     P.part_o = ctx->part_o;
     P.part_ml = ctx->part_ml;
     P.status = ctx->status;
+    P.wait_us = ctx->wait_limit_us;
+    P.extra_tx = ctx->test_extra_tx;
     if (P.n_splits > 1 && !ctx->cluster_merge && (size_t)n_items * P.n_splits * 2 * TILE * TILE > ctx->part_o_floats) return PC_ERR_CAPACITY;
 
     CUtensorMap mq, mk, mv[PC_MAX_SEGMENTS];
@@ -946,36 +655,8 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
         PC_CUDA_TRY(cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
         attr_set[ctx->device] = true;
     }
-    const bool pair_kernel = ctx->attend_impl == 2 && P.tiles_per_g % 4 == 0;
-    P.cluster = (P.n_splits > 1 && ctx->cluster_merge && !pair_kernel) ? 1 : 0;
-    if (pair_kernel) {
-        // two CTAs per cluster share every key / value tile (see k_attend_tc_pair)
-        CUtensorMap mk64;
-        if (!make_map(&mk64, k_rot, (uint64_t)tiles * TILE, (uint64_t)row_elems, 64)) {
-            fprintf(stderr, "packcache: cuTensorMapEncodeTiled failed\n");
-            return PC_ERR_CUDA;
-        }
-        static bool pair_attr_set[PC_MAX_DEVICES] = {};
-        if (!pair_attr_set[ctx->device]) {
-            PC_CUDA_TRY(cudaFuncSetAttribute(k_attend_tc_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, SP_ALLOC));
-            pair_attr_set[ctx->device] = true;
-        }
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(n_items * P.n_splits);
-        cfg.blockDim = dim3(TC_THREADS);
-        cfg.dynamicSmemBytes = SP_ALLOC;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 2;
-        PC_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_attend_tc_pair, mq, mk64, mv[0], mv[1], mv[2], P));
-    } else if (P.cluster) {
+    P.cluster = (P.n_splits > 1 && ctx->cluster_merge) ? 1 : 0;
+    if (P.cluster) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(n_items * P.n_splits);
         cfg.blockDim = dim3(TC_THREADS);

@@ -5,6 +5,8 @@
 #include <stdint.h>
 #include <stdio.h>
 
+#include <cmath>
+
 #include "packcache.h"
 
 #define PC_CUDA_TRY(expr)                                                                     \
@@ -36,7 +38,6 @@ enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT 
        PC_MARK_ATT0 = 6, PC_MARK_ROPE = 7, PC_MARK_ATTEND = 8, PC_MARK_COMBINE = 9, PC_MARK_MASS0 = 10, PC_MARK_MASS = 11,
        PC_N_MARKS = 12 };
 
-constexpr int PC_QPOOL_BLOCKS = 128;
 constexpr int PC_MAX_SEGMENTS = 3;
 constexpr int PC_MAX_DEVICES = 64;            // per-device launch state is kept in arrays of this size
 
@@ -55,19 +56,30 @@ struct pc_ctx {
     int sm_count;
     int group;                 // Hq / Hkv
     int elem_size;             // bytes per element
-    int attend_impl;           // 0 tensor-core (bf16), 1 CUDA-core, 2 tensor-core with CTA-pair multiply-adds
+    int attend_impl;           // 0 tensor-core (bf16), 1 CUDA-core
     pc_rope_dev rope;
     float2 *rope_tab;          // owned
     int32_t *status;           // device [2]: code, where
     int32_t *host_status;      // pinned [2]
-    float *qpool_partial;      // device [PC_QPOOL_BLOCKS][Hkv*d]
-    float *qpool;              // device [Hkv*d]
+    // Pooled query of the scoring pass as fixed-point sums (units of 2^-32), two buffers of Hkv*d 64-bit integers used
+    // in turn: the query pass of call n adds into buffer n & 1 (integer addition: the result does not depend on the
+    // order of the blocks), the scoring kernel of call n reads it and clears the other one for call n + 1.
+    long long *qpool_fx;       // device [2][Hkv*d], zero between uses
+    int qpool_turn;            // buffer the next query pass adds into
+    int qpool_dirty;           // 1: a call failed between the two kernels, both buffers are cleared before the next use
     // attention scratch (tensor-core path)
     void *k_rot;               // rotated keys, bf16 [rows][Hkv][d]
     size_t k_rot_rows;
     void *q_rot;               // rotated, pre-scaled queries, bf16 [max_q][Hq][d]
     int kv_splits;             // 0 = chosen per call
     int cluster_merge;         // 1 = KV ranges merge inside the kernel through cluster shared memory (default 0)
+    uint32_t wait_limit_us;    // limit of every bounded device-side wait in microseconds; 0 = about one second
+    uint32_t test_extra_tx;    // test hook: bytes the attention kernel's first barrier expects beyond what is sent (0 = off)
+    // rotated anchor keys kept in k_rot across fused frame steps (anchors never move): the segment they were made from
+    const void *anchor_rot_k;
+    const int32_t *anchor_rot_pos;
+    int anchor_rot_n;          // 0 = none cached
+    int q_rot_n;               // rows of q_rot written by the query pass of the running fused step (0 = none)
     // key set fixed by pc_attend_prepare (its rotated keys sit in k_rot until the next prepare or pc_attend_frame)
     int prepared_n_seg;        // 0 = nothing prepared
     pc_segment prepared_seg[PC_MAX_SEGMENTS];
@@ -100,6 +112,12 @@ __device__ __forceinline__ float2 pc_rope_cs(const pc_rope_dev &r, int pair, int
         pa = pa < 0 ? 0 : r.max_pos[a] - 1;
     }
     return __ldg(r.tab + r.off[a] + (size_t)pa * r.n_axis[a] + m);
+}
+
+// One rotary pair turned by (cos, sin), with the roundings spelt out: every kernel that rotates (query pass, key
+// pre-pass, pack with rotation) produces the same bits for the same inputs.
+__device__ __forceinline__ float2 pc_rotate(float x0, float x1, float2 cs) {
+    return make_float2(__fmaf_rn(x0, cs.x, -__fmul_rn(x1, cs.y)), __fmaf_rn(x0, cs.y, __fmul_rn(x1, cs.x)));
 }
 
 __device__ __forceinline__ float pc_bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -146,16 +164,20 @@ __device__ __forceinline__ uint64_t pc_global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait on an mbarrier phase: gives up after about one second, or at once when another thread of the CTA
-// already gave up (abort_flag), records PC_ERR_TIMEOUT with `where`, and returns false.
-static __device__ __noinline__ bool pc_mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status, int where) {
+// Bounded wait on an mbarrier phase, the one wait routine of every kernel of the library: gives up after limit_us
+// microseconds (0 = the default of about one second), or at once when another thread of the CTA already gave up
+// (abort_flag), records PC_ERR_TIMEOUT with `where` in the status word, and returns false.  The caller then skips the
+// work that depended on the wait, drains what it has in flight and leaves: no trap, no unbounded spin.
+__device__ __forceinline__ bool pc_mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status, int where,
+                                             uint32_t limit_us = 0) {
     for (int i = 0; i < 2048; ++i)
         if (pc_mbar_try(bar, parity)) return true;
     const uint64_t t0 = pc_global_ns();
+    const uint64_t limit_ns = limit_us ? (uint64_t)limit_us * 1000ull : 1000000000ull;
     for (;;) {
         if (pc_mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (pc_global_ns() - t0 > 1000000000ull) {
+        if (pc_global_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             pc_flag(status, PC_ERR_TIMEOUT, where);
             return false;
@@ -221,11 +243,23 @@ bool pc_aligned16(const void *p);
 pc_status pc_check_segment(const pc_segment *s, bool allow_empty);
 
 // stage launchers (each validates nothing: the pc_* entry points did)
+// k_rot_dst: where the rotated copy of each packed K row goes as well (bf16 tensor-core shapes), or NULL
 pc_status pc_launch_pack(pc_ctx *ctx, const void *src_k, const void *src_v, const int32_t *src_pos, const int32_t *sel_idx,
-                         int n_sel, int n_src, int delta_t, void *dst_k, void *dst_v, int32_t *dst_pos, cudaStream_t stream);
+                         int n_sel, int n_src, int delta_t, void *dst_k, void *dst_v, int32_t *dst_pos, void *k_rot_dst,
+                         cudaStream_t stream);
+// pc_score / pc_compact with the extras of the fused frame step: q_rot_out (NULL or the context's rotated-query scratch,
+// filled by the query pass that also pools), k_rot_dst (as pc_launch_pack)
+pc_status pc_score_impl(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q, const int32_t *budget,
+                        const uint8_t *valid, const float *scores_override, float *scores, int32_t *sel_idx, void *q_rot_out,
+                        cudaStream_t stream);
+pc_status pc_compact_impl(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget, int32_t delta_t,
+                          pc_cache *dst, void *k_rot_dst, cudaStream_t stream);
+// log2(e) / sqrt(d): folded into the rotated queries of the tensor-core attention kernel (its softmax runs in base 2)
+inline float pc_q_rot_scale(int head_dim) { return (float)(1.4426950408889634 / std::sqrt((double)head_dim)); }
 pc_status pc_launch_attend_simt(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
                                 int32_t n_q, void *out, float *lse, cudaStream_t stream);
-enum { PC_TC_ROPE_K = 1, PC_TC_ROPE_Q = 2, PC_TC_ATTEND = 4, PC_TC_ALL = 7 };
+// PC_TC_ROPE_K0: rotate the keys of the first segment only (the anchors of a fused frame step)
+enum { PC_TC_ROPE_K = 1, PC_TC_ROPE_Q = 2, PC_TC_ATTEND = 4, PC_TC_ALL = 7, PC_TC_ROPE_K0 = 8 };
 pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, const void *q, const int32_t *q_pos,
                               int32_t n_q, void *out, float *lse, cudaStream_t stream, int what);
 pc_status pc_attend_tc_scratch(const pc_layer_desc *d, int sm_count, size_t *k_rot_rows, size_t *part_o_floats,

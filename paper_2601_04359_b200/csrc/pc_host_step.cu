@@ -19,6 +19,14 @@ extern "C" pc_status pc_frame_step_host(pc_ctx *ctx, const pc_host_frame *in, pc
     }
     if (n_src > ws->src.history.capacity || in->n_anchor > ws->src.anchors.capacity) return PC_ERR_CAPACITY;
     if (!ws->q || !ws->q_pos || !ws->out || (n_src > 0 && (!ws->scores || !ws->sel_idx))) return PC_ERR_INVALID_ARG;
+    // every argument is checked before the first copy is enqueued
+    if (in->n_anchor > 0 && (!in->anchor_k || !in->anchor_v || !in->anchor_pos || !ws->src.anchors.k || !ws->src.anchors.v ||
+                             !ws->src.anchors.pos))
+        return PC_ERR_INVALID_ARG;
+    if (n_src > 0 && (!in->hist_k || !in->hist_v || !in->hist_pos || !ws->src.history.k || !ws->src.history.v ||
+                      !ws->src.history.pos || !ws->dst.history.k || !ws->dst.history.v || !ws->dst.history.pos))
+        return PC_ERR_INVALID_ARG;
+    if (in->n_q > ctx->desc.max_q) return PC_ERR_CAPACITY;
 
     std::vector<int32_t> budget((size_t)std::max(in->n_frames, 1));
     pc_status st = pc_plan_budget(params, in->n_frames, in->frame_count, budget.data());
@@ -31,13 +39,11 @@ extern "C" pc_status pc_frame_step_host(pc_ctx *ctx, const pc_host_frame *in, pc
     PC_CUDA_TRY(cudaMemcpyAsync(ws->q, in->q, (size_t)in->n_q * qrow, cudaMemcpyHostToDevice, stream));
     PC_CUDA_TRY(cudaMemcpyAsync(ws->q_pos, in->q_pos, (size_t)in->n_q * 16, cudaMemcpyHostToDevice, stream));
     if (in->n_anchor > 0) {
-        if (!in->anchor_k || !in->anchor_v || !in->anchor_pos) return PC_ERR_INVALID_ARG;
         PC_CUDA_TRY(cudaMemcpyAsync(ws->src.anchors.k, in->anchor_k, in->n_anchor * row, cudaMemcpyHostToDevice, stream));
         PC_CUDA_TRY(cudaMemcpyAsync(ws->src.anchors.v, in->anchor_v, in->n_anchor * row, cudaMemcpyHostToDevice, stream));
         PC_CUDA_TRY(cudaMemcpyAsync(ws->src.anchors.pos, in->anchor_pos, (size_t)in->n_anchor * 16, cudaMemcpyHostToDevice, stream));
     }
     if (n_src > 0) {
-        if (!in->hist_k || !in->hist_v || !in->hist_pos) return PC_ERR_INVALID_ARG;
         PC_CUDA_TRY(cudaMemcpyAsync(ws->src.history.k, in->hist_k, n_src * row, cudaMemcpyHostToDevice, stream));
         PC_CUDA_TRY(cudaMemcpyAsync(ws->src.history.v, in->hist_v, n_src * row, cudaMemcpyHostToDevice, stream));
         PC_CUDA_TRY(cudaMemcpyAsync(ws->src.history.pos, in->hist_pos, (size_t)n_src * 16, cudaMemcpyHostToDevice, stream));

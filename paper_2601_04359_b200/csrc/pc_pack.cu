@@ -3,19 +3,22 @@
 // One warp moves one retained token: its K row and V row over all KV heads (16-byte vector loads and stores,
 // consecutive lanes on consecutive 16-byte chunks, so every request is a full 512-byte line run) and its position
 // record with t shifted by delta_t.  Rows are streamed (no L1 allocation): nothing here is read twice.
+// For the fused frame step the same warp also writes the row's rotated keys (3D rotary embedding at the rebased
+// position, bf16) into the attention kernel's key scratch: the row is in registers anyway, and the kernel is bound by
+// memory, not by issue, so the attention call that follows needs no rotary pre-pass over the packed history.
 #include "pc_common.cuh"
 
 namespace {
 
 constexpr int PACK_THREADS = 256;
 
-template <int CPL /* 16-byte chunks per lane per row; 0 = generic loop */>
+template <int CPL /* 16-byte chunks per lane per row; 0 = generic loop */, bool ROT /* also write rotated bf16 keys */>
 __global__ void __launch_bounds__(PACK_THREADS) k_pack(const char *__restrict__ src_k, const char *__restrict__ src_v,
                                                        const int32_t *__restrict__ src_pos,
                                                        const int32_t *__restrict__ sel_idx, int n_sel, int n_src,
                                                        int row_bytes, int delta_t, char *__restrict__ dst_k,
                                                        char *__restrict__ dst_v, int32_t *__restrict__ dst_pos,
-                                                       int32_t *status) {
+                                                       char *__restrict__ rot_k, pc_rope_dev rope, int d, int32_t *status) {
     pc_grid_dep_launch();
     pc_grid_dep_wait();
     const int lane = threadIdx.x & 31;
@@ -28,6 +31,8 @@ __global__ void __launch_bounds__(PACK_THREADS) k_pack(const char *__restrict__ 
     }
     const char *sk = src_k + (size_t)s * row_bytes, *sv = src_v + (size_t)s * row_bytes;
     char *dk = dst_k + (size_t)r * row_bytes, *dv = dst_v + (size_t)r * row_bytes;
+    int4 p = __ldg(reinterpret_cast<const int4 *>(src_pos) + s);
+    p.x -= delta_t;                                  // only t moves; h, w and the tag are carried as they are
     if constexpr (CPL > 0) {
         uint4 a[CPL], b[CPL];
 #pragma unroll
@@ -38,6 +43,25 @@ __global__ void __launch_bounds__(PACK_THREADS) k_pack(const char *__restrict__ 
         for (int c = 0; c < CPL; ++c) pc_stg_stream(dk + (size_t)(c * 32 + lane) * 16, a[c]);
 #pragma unroll
         for (int c = 0; c < CPL; ++c) pc_stg_stream(dv + (size_t)(c * 32 + lane) * 16, b[c]);
+        if constexpr (ROT) {
+            // 32 lanes x 8 elements span a multiple of d: all of this lane's chunks hold the same four rotary pairs
+            const int pair0 = ((lane * 8) % d) / 2;
+            float2 cs[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) cs[u] = pc_rope_cs(rope, pair0 + u, p.x, p.y, p.z, status, PC_WHERE_ROPE_POS);
+            char *rk = rot_k + (size_t)r * row_bytes;
+#pragma unroll
+            for (int c = 0; c < CPL; ++c) {
+                const uint32_t w[4] = {a[c].x, a[c].y, a[c].z, a[c].w};
+                uint32_t o[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float2 y = pc_rotate(pc_bf16_lo(w[u]), pc_bf16_hi(w[u]), cs[u]);
+                    o[u] = pc_pack_bf16(y.x, y.y);
+                }
+                *reinterpret_cast<uint4 *>(rk + (size_t)(c * 32 + lane) * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
     } else {
         for (int off = lane * 16; off < row_bytes; off += 32 * 16) {
             const uint4 a = pc_ldg_stream(sk + off), b = pc_ldg_stream(sv + off);
@@ -45,11 +69,7 @@ __global__ void __launch_bounds__(PACK_THREADS) k_pack(const char *__restrict__ 
             pc_stg_stream(dv + off, b);
         }
     }
-    if (lane == 0) {
-        int4 p = __ldg(reinterpret_cast<const int4 *>(src_pos) + s);
-        p.x -= delta_t;                              // only t moves; h, w and the tag are carried as they are
-        reinterpret_cast<int4 *>(dst_pos)[r] = p;
-    }
+    if (lane == 0) reinterpret_cast<int4 *>(dst_pos)[r] = p;
 }
 
 bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
@@ -59,10 +79,9 @@ bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
 
 }  // namespace
 
-extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget,
-                                int32_t delta_t, pc_cache *dst, void *stream_) {
+pc_status pc_compact_impl(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget, int32_t delta_t,
+                          pc_cache *dst, void *k_rot_dst, cudaStream_t stream) {
     if (!ctx || !src || !dst || !budget) return PC_ERR_INVALID_ARG;
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (src->n_frames < 0 || (src->n_frames > 0 && !src->frame_count)) return PC_ERR_INVALID_ARG;
     pc_status st = pc_check_segment(&src->history, true);
     if (st != PC_OK) return st;
@@ -88,25 +107,44 @@ extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t 
         return PC_ERR_INVALID_ARG;
     pc_mark(ctx, PC_MARK_PACK0, stream);
     st = pc_launch_pack(ctx, src->history.k, src->history.v, src->history.pos, sel_idx, (int)n_sel, (int)n_src, delta_t, D.k, D.v,
-                        D.pos, stream);
+                        D.pos, k_rot_dst, stream);
     if (st != PC_OK) return st;
     pc_mark(ctx, PC_MARK_PACK, stream);
     return PC_OK;
 }
 
+extern "C" pc_status pc_compact(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget,
+                                int32_t delta_t, pc_cache *dst, void *stream_) {
+    return pc_compact_impl(ctx, src, sel_idx, budget, delta_t, dst, nullptr, static_cast<cudaStream_t>(stream_));
+}
+
 // Gather n_sel rows (K, V, position records) of a source of n_src rows into a destination; arguments already checked.
 pc_status pc_launch_pack(pc_ctx *ctx, const void *src_k, const void *src_v, const int32_t *src_pos, const int32_t *sel_idx,
-                         int n_sel, int n_src, int delta_t, void *dst_k, void *dst_v, int32_t *dst_pos, cudaStream_t stream) {
+                         int n_sel, int n_src, int delta_t, void *dst_k, void *dst_v, int32_t *dst_pos, void *k_rot_dst,
+                         cudaStream_t stream) {
     const int row_bytes = ctx->desc.n_kv_heads * ctx->desc.head_dim * ctx->elem_size;
     const int blocks = (int)(((int64_t)n_sel * 32 + PACK_THREADS - 1) / PACK_THREADS);
     const char *sk = static_cast<const char *>(src_k), *sv = static_cast<const char *>(src_v);
-    char *dk = static_cast<char *>(dst_k), *dv = static_cast<char *>(dst_v);
-#define PC_PACK_ARGS sk, sv, src_pos, sel_idx, n_sel, n_src, row_bytes, delta_t, dk, dv, dst_pos, ctx->status
-    switch (row_bytes) {
-    case 512: PC_LAUNCH((k_pack<1>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
-    case 1024: PC_LAUNCH((k_pack<2>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
-    case 2048: PC_LAUNCH((k_pack<4>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
-    default: PC_LAUNCH((k_pack<0>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+    char *dk = static_cast<char *>(dst_k), *dv = static_cast<char *>(dst_v), *rk = static_cast<char *>(k_rot_dst);
+    const int d = ctx->desc.head_dim;
+#define PC_PACK_ARGS sk, sv, src_pos, sel_idx, n_sel, n_src, row_bytes, delta_t, dk, dv, dst_pos, rk, ctx->rope, d, ctx->status
+    if (rk) {
+        // rotated keys are written for bf16 rows whose 32 x 16-byte chunk rows span whole heads (the tensor-core shapes)
+        if (ctx->desc.dtype != PC_BF16 || 256 % d) return PC_ERR_UNSUPPORTED;
+        switch (row_bytes) {
+        case 512: PC_LAUNCH((k_pack<1, true>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+        case 1024: PC_LAUNCH((k_pack<2, true>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+        case 2048: PC_LAUNCH((k_pack<4, true>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+        case 4096: PC_LAUNCH((k_pack<8, true>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+        default: return PC_ERR_UNSUPPORTED;
+        }
+    } else {
+        switch (row_bytes) {
+        case 512: PC_LAUNCH((k_pack<1, false>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+        case 1024: PC_LAUNCH((k_pack<2, false>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+        case 2048: PC_LAUNCH((k_pack<4, false>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+        default: PC_LAUNCH((k_pack<0, false>), dim3(blocks), dim3(PACK_THREADS), 0, stream, PC_PACK_ARGS); break;
+        }
     }
 #undef PC_PACK_ARGS
     PC_CUDA_TRY(cudaGetLastError());

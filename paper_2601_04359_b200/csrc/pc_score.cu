@@ -1,6 +1,7 @@
 // Token scoring and per-frame top-k selection (the "attention-relevant" retention of Sec. 3.4).
 //
-//   k_qpool  : pooled query  q~[g][c] = sum_{h in group g} (1/n_q) sum_i (R(p_i) q_ih)[c]        (fp32, deterministic)
+//   k_qprep  : one pass over Q: pooled query  q~[g][c] = sum_{h in group g} (1/n_q) sum_i (R(p_i) q_ih)[c]  (fixed-point
+//              sums, deterministic) and, on request, the rotated bf16 queries the attention kernel reads
 //   k_score  : s_j = 1/(Hq sqrt(d)) * sum_g q~_g . R(p_j) k_jg   — one pass over the history keys, HBM-bound
 //   k_select : per frame the budget[f] best scores (ties to the lower index), ascending indices out
 //
@@ -9,6 +10,8 @@
 //   q_a (k_a cos - k_b sin) + q_b (k_a sin + k_b cos) = cos (q_a k_a + q_b k_b) + sin (q_b k_a - q_a k_b),
 // and the angle is the same for every KV head, so the two brackets are summed over heads first and each pair costs
 // one table look-up per token.
+#include <algorithm>
+
 #include "pc_common.cuh"
 
 namespace {
@@ -29,192 +32,155 @@ template <> struct Elem<__nv_bfloat16> {
 };
 
 // ---------------------------------------------------------------------------------------------------------
-// Pooled query.  The rotation is the same for every head at a given token and rotary pair, so the heads of a group
-// are added first and the sum is rotated once:  q~[g] = (1/n_q) sum_i R(p_i) (sum_{h in g} q_ih).
-// A block owns a contiguous run of query tokens.  Its 512 threads form `slices` token slices x n_cols pair-columns
-// of the [Hkv][d/2] pooled grid (a warp reads 128 contiguous bytes of each head); a thread walks its slice's tokens
-// eight at a time with all loads of a batch issued before any is used.  Slices are added in slice order through
-// shared memory; a second small kernel adds the per-block partials in a fixed order, so the result does not depend
-// on scheduling.
+// Query pass.  One read of Q serves both consumers of the rotated queries: the pooled query of the scoring pass
+//   q~[g] = (1/n_q) sum_i sum_{h in g} R(p_i) q_ih
+// and, for the tensor-core attention kernel, the rotated bf16 queries with log2(e)/sqrt(d) folded in (q_rot).
+// One warp takes one query token: lane l reads the 16-byte chunks l, l + 32, ... of the row (all in flight at once);
+// 32 chunks span a multiple of d, so all of a lane's chunks hold the same rotary pairs and the lane needs PER/2 table
+// entries per token.  The rotated row also goes to a per-warp slab in shared memory; after a block barrier the threads
+// add, in a fixed order, the slabs' entries of each pooled element (heads of the group, then warps), turn the sum
+// into a 64-bit fixed-point number (units of 2^-32) and add it to the global accumulator with an integer atomic:
+// integer addition is associative, so the pooled query does not depend on the order in which blocks arrive.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int QPOOL_THREADS = 512;
-constexpr int QPOOL_BATCH = 8;
+constexpr int QPREP_MAX_WARPS = 8;
+constexpr float FX_ONE = 4294967296.0f;             // 2^32
 
-template <typename T, int GROUP /* query heads per KV head; 0 = any */>
-__global__ void __launch_bounds__(QPOOL_THREADS) k_qpool(const T *__restrict__ q, const int32_t *__restrict__ q_pos, int n_q,
-                                                         int n_q_heads, int group_rt, int d, pc_rope_dev rope,
-                                                         float *__restrict__ partial, int32_t *status) {
-    pc_grid_dep_launch();
-    pc_grid_dep_wait();
-    __shared__ float2 slice_sum[QPOOL_THREADS];
-    const int group = GROUP > 0 ? GROUP : group_rt;
-    const int half = d / 2, n_kv = n_q_heads / group, n_cols = n_kv * half, row_len = n_kv * d;
-    const size_t q_row = (size_t)n_q_heads * d;
-    const int per_block = (n_q + gridDim.x - 1) / gridDim.x;
-    const int first = blockIdx.x * per_block, end = min(n_q, first + per_block);
-    const int slices = max(1, QPOOL_THREADS / n_cols);
-    const int sl = threadIdx.x / n_cols;
-    for (int col0 = 0; col0 < n_cols; col0 += QPOOL_THREADS) {        // one pass unless n_cols > 1024
-        const int col = col0 + (n_cols >= QPOOL_THREADS ? threadIdx.x : threadIdx.x % n_cols);
-        const bool active = sl < slices && col < n_cols;
-        float acc0 = 0.f, acc1 = 0.f;
-        if (active) {
-            const int g = col / half, pair = col % half;
-            const T *base = q + (size_t)g * group * d + 2 * pair;
-            const int axis = pair % 3, amax = rope.max_pos[axis], astride = rope.n_axis[axis];
-            const float2 *tab = rope.tab + rope.off[axis] + pair / 3;
-            for (int i0 = first + sl; i0 < end; i0 += slices * QPOOL_BATCH) {
-                int pa[QPOOL_BATCH];                                   // this pair's own coordinate of each token
-                float x0[QPOOL_BATCH], x1[QPOOL_BATCH];
-#pragma unroll
-                for (int t = 0; t < QPOOL_BATCH; ++t) {
-                    const int i = min(i0 + t * slices, end - 1);       // out-of-range slots re-read the last token, unused
-                    pa[t] = __ldg(q_pos + 4 * (size_t)i + axis);
-                    const T *row = base + (size_t)i * q_row;
-                    x0[t] = 0.f; x1[t] = 0.f;
-#pragma unroll
-                    for (int u = 0; u < (GROUP > 0 ? GROUP : 1); ++u) {
-                        for (int uu = u; uu < group; uu += (GROUP > 0 ? group : 1)) {
-                            if constexpr (sizeof(T) == 2) {
-                                const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(row + (size_t)uu * d));
-                                x0[t] += pc_bf16_lo(w); x1[t] += pc_bf16_hi(w);
-                            } else {
-                                const float2 w = __ldg(reinterpret_cast<const float2 *>(row + (size_t)uu * d));
-                                x0[t] += w.x; x1[t] += w.y;
-                            }
-                        }
-                    }
-                }
-                float2 cs[QPOOL_BATCH];
-#pragma unroll
-                for (int t = 0; t < QPOOL_BATCH; ++t) {
-                    int p = pa[t];
-                    if ((unsigned)p >= (unsigned)amax) {               // outside the table: record, clamp
-                        pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_QPOOL_POS);
-                        p = p < 0 ? 0 : amax - 1;
-                    }
-                    cs[t] = __ldg(tab + (size_t)p * astride);
-                }
-#pragma unroll
-                for (int t = 0; t < QPOOL_BATCH; ++t)
-                    if (i0 + t * slices < end) {
-                        acc0 += x0[t] * cs[t].x - x1[t] * cs[t].y;
-                        acc1 += x0[t] * cs[t].y + x1[t] * cs[t].x;
-                    }
-            }
-        }
-        slice_sum[threadIdx.x] = make_float2(acc0, acc1);
-        __syncthreads();
-        if (active && sl == 0) {
-            float2 tot = make_float2(0.f, 0.f);
-            const int stride = n_cols >= QPOOL_THREADS ? QPOOL_THREADS : n_cols;
-            for (int k = 0; k < slices; ++k) { const float2 v = slice_sum[k * stride + threadIdx.x]; tot.x += v.x; tot.y += v.y; }
-            *reinterpret_cast<float2 *>(partial + (size_t)blockIdx.x * row_len + 2 * col) = tot;
-        }
-        __syncthreads();
-    }
+template <typename T> __device__ __forceinline__ uint4 pack_row(const float *f);
+template <> __device__ __forceinline__ uint4 pack_row<float>(const float *f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+}
+template <> __device__ __forceinline__ uint4 pack_row<__nv_bfloat16>(const float *f) {
+    return make_uint4(pc_pack_bf16(f[0], f[1]), pc_pack_bf16(f[2], f[3]), pc_pack_bf16(f[4], f[5]), pc_pack_bf16(f[6], f[7]));
 }
 
-// pooled[e] = (1/n_q) * sum over blocks of partial[b][e].  32 columns per block; 32 threads per column each add every
-// 32nd partial (in block order, at most four loads, all in flight together), and the 32 sums are added in slice order.
-__global__ void __launch_bounds__(1024) k_qpool_reduce(const float *__restrict__ partial, int n_partials, int row_len, float inv_n,
-                                                       float *__restrict__ pooled) {
+template <typename T, int QCPL /* chunks per lane of a query row; 0 = any count, looped */>
+__global__ void __launch_bounds__(QPREP_MAX_WARPS * 32) k_qprep(const T *__restrict__ q, const int32_t *__restrict__ q_pos, int n_q,
+                                                                 int n_q_heads, int group, int d, int cpl_rt, pc_rope_dev rope,
+                                                                 float out_scale, T *__restrict__ q_rot,
+                                                                 unsigned long long *__restrict__ fx, int32_t *status) {
     pc_grid_dep_launch();
     pc_grid_dep_wait();
-    __shared__ float part[32][33];
-    const int c = threadIdx.x & 31, sl = threadIdx.x >> 5, e = blockIdx.x * 32 + c;
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
-    if (e < row_len) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int b = sl + 32 * i;
-            if (b < n_partials) v[i] = __ldcg(partial + (size_t)b * row_len + e);
-        }
-    }
-    part[sl][c] = (v[0] + v[1]) + (v[2] + v[3]);
-    __syncthreads();
-    if (sl == 0 && e < row_len) {
-        float tot = 0.f;
-#pragma unroll
-        for (int k = 0; k < 32; ++k) tot += part[k][c];
-        pooled[e] = tot * inv_n;
-    }
-}
-
-// ---------------------------------------------------------------------------------------------------------
-// Score.  History keys are contiguous, so a tile of 8 tokens is one run of 8 rows (16 KB at 8 KV heads x 128 bf16)
-// plus 128 bytes of positions.  A producer warp streams tiles into a four-stage shared-memory ring with bulk
-// asynchronous copies tracked by mbarriers; eight consumer warps take one token each.  A token's row over all KV
-// heads is CPL x 32 sixteen-byte chunks; lane l reads chunks l, l+32, ...  Because 32 chunks span a multiple of d,
-// all of a lane's chunks cover the same PER16/2 rotary pairs (of different heads), so the lane sums the two brackets
-// over its chunks and needs PER16/2 table look-ups per token.  Chunks are processed two at a time so that every
-// multiply-add is a two-lane fp32 instruction.  Blocks are persistent and take tiles round-robin.
-// ---------------------------------------------------------------------------------------------------------
-constexpr int SCORE_TOK = 8;                       // tokens per tile = consumer warps
-constexpr int SCORE_STAGES = 4;
-constexpr int SCORE_THREADS = (SCORE_TOK + 1) * 32;
-
-template <typename T, int CPL /* chunks per lane */>
-__global__ void __launch_bounds__(SCORE_THREADS) k_score(const T *__restrict__ k, const int32_t *__restrict__ k_pos,
-                                                         const uint8_t *__restrict__ valid, int n_src, int d, float scale,
-                                                         pc_rope_dev rope, const float *__restrict__ pooled,
-                                                         float *__restrict__ scores, int32_t *status) {
-    pc_grid_dep_launch();
     constexpr int PER = Elem<T>::PER16, NP = PER / 2;
-    constexpr uint32_t ROW_BYTES = CPL * 32 * 16;
-    constexpr uint32_t STAGE_BYTES = SCORE_TOK * ROW_BYTES + SCORE_TOK * 16;
-    extern __shared__ __align__(128) uint8_t ring[];
-    __shared__ __align__(8) uint64_t bars[2 * SCORE_STAGES];
-    __shared__ int abort_word;
-    volatile int *abort_flag = &abort_word;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t ring0 = pc_smem_u32(ring), bar0 = pc_smem_u32(bars);
-    auto full = [&](int s) { return bar0 + 8u * s; };
-    auto empty = [&](int s) { return bar0 + 8u * (SCORE_STAGES + s); };
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < SCORE_STAGES; ++s) { pc_mbar_init(full(s), 1); pc_mbar_init(empty(s), SCORE_TOK); }
-        abort_word = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-    pc_grid_dep_wait();   // the pooled query comes from the kernel before
-    const int n_tiles = (n_src + SCORE_TOK - 1) / SCORE_TOK;
-
-    if (warp == SCORE_TOK) {
-        // ------------------------------------------------------------ producer
-        if (lane == 0) {
-            int it = 0;
-            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-                const int s = it % SCORE_STAGES, use = it / SCORE_STAGES;
-                if (use > 0 && !pc_mbar_wait(empty(s), (use - 1) & 1, abort_flag, status, PC_WHERE_SCORE_WAIT)) break;
-                const int tok0 = tile * SCORE_TOK, n_tok = min(SCORE_TOK, n_src - tok0);
-                const uint32_t dst = ring0 + s * STAGE_BYTES;
-                pc_mbar_expect_tx(full(s), n_tok * (ROW_BYTES + 16));
-                pc_bulk_g2s(dst, reinterpret_cast<const char *>(k) + (size_t)tok0 * ROW_BYTES, n_tok * ROW_BYTES, full(s));
-                pc_bulk_g2s(dst + SCORE_TOK * ROW_BYTES, k_pos + 4 * (size_t)tok0, n_tok * 16, full(s));
-            }
-            if (*abort_flag) {   // let copies already issued land before the block's shared memory goes away
-                const uint64_t t0 = pc_global_ns();
-                while (pc_global_ns() - t0 < 2000000ull) {}
-            }
-        }
-        return;
-    }
-
-    // ---------------------------------------------------------------- consumers
-    // this lane's slice of the pooled query stays in registers, chunks paired for the two-lane multiply-adds
-    constexpr int CP = CPL / 2;                                     // chunk pairs; an odd CPL leaves one single chunk
-    float2 qa[CP > 0 ? CP : 1][NP], qb[CP > 0 ? CP : 1][NP];
-    float qa1[NP], qb1[NP];
+    extern __shared__ __align__(16) float slab[];                     // [warps][Hq*d]
+    const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row_len = n_q_heads * d;
+    const int cpl = QCPL > 0 ? QCPL : cpl_rt;
+    const int i = blockIdx.x * warps + warp;
+    if (i < n_q) {
+        const int4 pp = __ldg(reinterpret_cast<const int4 *>(q_pos) + i);
+        const uint4 *src = reinterpret_cast<const uint4 *>(q + (size_t)i * row_len) + lane;
+        uint4 raw[QCPL > 0 ? QCPL : 1];
+        if constexpr (QCPL > 0) {
 #pragma unroll
-    for (int c = 0; c < CPL; ++c)
+            for (int c = 0; c < QCPL; ++c) raw[c] = pc_ldg_stream(src + c * 32);
+        }
+        const int pair0 = ((lane * PER) % d) / 2;
+        float2 cs[NP];
 #pragma unroll
         for (int u = 0; u < NP; ++u) {
-            const float a = pooled[(size_t)(c * 32 + lane) * PER + 2 * u], b = pooled[(size_t)(c * 32 + lane) * PER + 2 * u + 1];
-            if (c < 2 * CP) {
-                if (c & 1) { qa[c / 2][u].y = a; qb[c / 2][u].y = b; } else { qa[c / 2][u].x = a; qb[c / 2][u].x = b; }
-            } else { qa1[u] = a; qb1[u] = b; }
+            cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_QPOOL_POS);
+            cs[u].x *= out_scale;
+            cs[u].y *= out_scale;
         }
+        float *mine = slab + (size_t)warp * row_len + lane * PER;
+        uint4 *dst = q_rot ? reinterpret_cast<uint4 *>(q_rot + (size_t)i * row_len) + lane : nullptr;
+        auto one_chunk = [&](const uint4 &v, int c) {
+            float x[PER], r[PER];
+            Elem<T>::unpack(v, x);
+#pragma unroll
+            for (int u = 0; u < NP; ++u) {
+                const float2 y = pc_rotate(x[2 * u], x[2 * u + 1], cs[u]);
+                r[2 * u] = y.x;
+                r[2 * u + 1] = y.y;
+            }
+            float4 *s4 = reinterpret_cast<float4 *>(mine + (size_t)c * 32 * PER);
+#pragma unroll
+            for (int k = 0; k < PER / 4; ++k) s4[k] = make_float4(r[4 * k], r[4 * k + 1], r[4 * k + 2], r[4 * k + 3]);
+            if (dst) dst[c * 32] = pack_row<T>(r);
+        };
+        if constexpr (QCPL > 0) {
+#pragma unroll
+            for (int c = 0; c < QCPL; ++c) one_chunk(raw[c], c);
+        } else {
+            for (int c = 0; c < cpl; ++c) one_chunk(pc_ldg_stream(src + c * 32), c);
+        }
+    }
+    __syncthreads();
+    const int n_warps_used = min(warps, n_q - blockIdx.x * warps);
+    const int n_out = (n_q_heads / group) * d;
+    for (int e = threadIdx.x; e < n_out; e += blockDim.x) {
+        const int g = e / d, x = e - g * d;
+        float sum = 0.f;
+        for (int w = 0; w < n_warps_used; ++w) {
+            const float *s = slab + (size_t)w * row_len + (size_t)g * group * d + x;
+            for (int h = 0; h < group; ++h) sum += s[h * d];
+        }
+        const long long v = __float2ll_rn(sum * FX_ONE);
+        atomicAdd(fx + e, (unsigned long long)v);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Score.  One warp takes two history tokens at a time: lane l loads the 16-byte chunks l, l + 32, ... of both rows
+// (streaming loads, all in flight before the first is used: 2 x CPL x 512 bytes per warp) and both position records.
+// 32 chunks span a multiple of d, so all of a lane's chunks cover the same PER/2 rotary pairs (of different heads): the
+// lane sums the two brackets over its chunks and needs PER/2 table look-ups per token.  The pooled query sits in shared
+// memory, converted once per block from the fixed-point accumulator and laid out so that one 16-byte read gives a
+// lane its (q_a, q_b) of two chunks at once: chunks are processed two at a time and every multiply-add is a two-lane
+// fp32 instruction.  Blocks are persistent; warps take token pairs round-robin, so the tokens in flight at any time
+// form one contiguous window of the history.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int SCORE_WARPS = 8;
+constexpr int SCORE_THREADS = SCORE_WARPS * 32;
+
+template <typename T, int CPL /* chunks per lane */>
+__global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict__ k, const int32_t *__restrict__ k_pos,
+                                                            const uint8_t *__restrict__ valid, int n_src, int d, float scale,
+                                                            pc_rope_dev rope, const long long *__restrict__ fx, double fx_scale,
+                                                            long long *__restrict__ fx_clear, float *__restrict__ scores,
+                                                            int32_t *status) {
+    pc_grid_dep_launch();
+    constexpr int PER = Elem<T>::PER16, NP = PER / 2, CP = (CPL + 1) / 2;
+    __shared__ float4 qs[CP * NP * 32];                               // (q_a chunk 2cp, q_a chunk 2cp+1, q_b ..., q_b ...)
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gw = blockIdx.x * SCORE_WARPS + warp, n_warps = gridDim.x * SCORE_WARPS;
+    const int n_pairs = (n_src + 1) >> 1;
+    const uint4 *krow = reinterpret_cast<const uint4 *>(k) + lane;
+    pc_grid_dep_wait();   // the pooled query comes from the kernel before
+
+    // this warp's first two rows are requested before the pooled query is staged: both latencies overlap
+    int tp = gw;
+    uint4 raw0[CPL], raw1[CPL];
+    int4 p0 = make_int4(0, 0, 0, 0), p1 = p0;
+    auto request = [&](int pair_idx) {
+        const int j0 = 2 * pair_idx, j1 = min(j0 + 1, n_src - 1);
+        p0 = __ldg(reinterpret_cast<const int4 *>(k_pos) + j0);
+        p1 = __ldg(reinterpret_cast<const int4 *>(k_pos) + j1);
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) raw0[c] = pc_ldg_stream(krow + (size_t)j0 * (CPL * 32) + c * 32);
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) raw1[c] = pc_ldg_stream(krow + (size_t)j1 * (CPL * 32) + c * 32);
+    };
+    if (tp < n_pairs) request(tp);
+
+    for (int idx = threadIdx.x; idx < CP * NP * 32; idx += SCORE_THREADS) {
+        const int l = idx & 31, u = (idx >> 5) % NP, cp = idx / (32 * NP);
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int c = 2 * cp + half;
+            if (c < CPL) {
+                const longlong2 w = __ldcg(reinterpret_cast<const longlong2 *>(fx + (size_t)(c * 32 + l) * PER + 2 * u));
+                v[half] = (float)((double)w.x * fx_scale);
+                v[2 + half] = (float)((double)w.y * fx_scale);
+            }
+        }
+        qs[idx] = make_float4(v[0], v[1], v[2], v[3]);
+    }
+    if (fx_clear && blockIdx.x == 0)                                  // the other accumulator, for the next call's query pass
+        for (int e = threadIdx.x; e < CPL * 32 * PER; e += SCORE_THREADS) fx_clear[e] = 0;
+    __syncthreads();
+
     // table slots of this lane's pairs: entry = tbase + coordinate(axis) * stride
     const int pair0 = ((lane * PER) % d) / 2;
     int tbase[NP], tstride[NP], taxis[NP];
@@ -226,74 +192,78 @@ __global__ void __launch_bounds__(SCORE_THREADS) k_score(const T *__restrict__ k
         tstride[u] = rope.n_axis[a];
     }
     const unsigned mt = rope.max_pos[0], mh = rope.max_pos[1], mw = rope.max_pos[2];
+    const float4 *ql = qs + lane;
 
-    int it = 0;
-    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-        const int s = it % SCORE_STAGES, use = it / SCORE_STAGES;
-        if (!__all_sync(0xffffffffu, pc_mbar_wait(full(s), use & 1, abort_flag, status, PC_WHERE_SCORE_WAIT))) return;
-        const int j = tile * SCORE_TOK + warp;
-        if (j < n_src) {
-            const uint32_t row = ring0 + s * STAGE_BYTES + warp * ROW_BYTES + lane * 16;
-            uint4 raw[CPL];
+    auto table = [&](int4 p, float2 (&cs)[NP]) {
+        int pt = p.x, ph = p.y, pw = p.z;
+        if (!((unsigned)pt < mt && (unsigned)ph < mh && (unsigned)pw < mw)) {   // outside the tables: record, clamp
+            pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_SCORE_POS);
+            pt = min(max(pt, 0), (int)mt - 1); ph = min(max(ph, 0), (int)mh - 1); pw = min(max(pw, 0), (int)mw - 1);
+        }
 #pragma unroll
-            for (int c = 0; c < CPL; ++c) raw[c] = pc_lds128(row + c * 512);
-            const uint4 pw4 = pc_lds128(ring0 + s * STAGE_BYTES + SCORE_TOK * ROW_BYTES + warp * 16);
-            int pt = (int)pw4.x, ph = (int)pw4.y, pw = (int)pw4.z;
-            if (!((unsigned)pt < mt && (unsigned)ph < mh && (unsigned)pw < mw)) {   // outside the tables: record, clamp
-                pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_SCORE_POS);
-                pt = min(max(pt, 0), (int)mt - 1); ph = min(max(ph, 0), (int)mh - 1); pw = min(max(pw, 0), (int)mw - 1);
+        for (int u = 0; u < NP; ++u) {
+            const int pa = taxis[u] == 0 ? pt : (taxis[u] == 1 ? ph : pw);
+            cs[u] = __ldg(rope.tab + tbase[u] + pa * tstride[u]);
+        }
+    };
+    // brackets per pair:  A = sum q_a k_a + q_b k_b,  B = sum q_b k_a - q_a k_b  (B kept as two sums)
+    auto row_score = [&](const uint4 (&raw)[CPL], const float2 (&cs)[NP]) {
+        float2 A2[NP], B2[NP], C2[NP];
+#pragma unroll
+        for (int u = 0; u < NP; ++u) A2[u] = B2[u] = C2[u] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int cp = 0; cp < CP; ++cp) {
+            float k0[PER], k1[PER];
+            Elem<T>::unpack(raw[2 * cp], k0);
+            if (2 * cp + 1 < CPL) {
+                Elem<T>::unpack(raw[2 * cp + 1 < CPL ? 2 * cp + 1 : 0], k1);
+            } else {
+#pragma unroll
+                for (int e = 0; e < PER; ++e) k1[e] = 0.f;
             }
-            float2 cs[NP];
 #pragma unroll
             for (int u = 0; u < NP; ++u) {
-                const int pa = taxis[u] == 0 ? pt : (taxis[u] == 1 ? ph : pw);
-                cs[u] = __ldg(rope.tab + tbase[u] + pa * tstride[u]);
+                const float4 qq = ql[(cp * NP + u) * 32];
+                const float2 qa = make_float2(qq.x, qq.y), qb = make_float2(qq.z, qq.w);
+                const float2 ka = make_float2(k0[2 * u], k1[2 * u]), kb = make_float2(k0[2 * u + 1], k1[2 * u + 1]);
+                pc_fma2(A2[u], qa, ka);
+                pc_fma2(A2[u], qb, kb);
+                pc_fma2(B2[u], qb, ka);
+                pc_fma2(C2[u], qa, kb);
             }
-            // brackets per pair:  A = sum qa ka + qb kb,  B = sum qb ka - qa kb  (B kept as two sums)
-            float2 A2[NP], B2[NP], C2[NP];
-            float A1[NP], B1[NP];
+        }
+        float sum = 0.f;
 #pragma unroll
-            for (int u = 0; u < NP; ++u) { A2[u] = B2[u] = C2[u] = make_float2(0.f, 0.f); A1[u] = B1[u] = 0.f; }
+        for (int u = 0; u < NP; ++u) {
+            const float A = A2[u].x + A2[u].y;
+            const float B = (B2[u].x + B2[u].y) - (C2[u].x + C2[u].y);
+            sum = fmaf(cs[u].x, A, fmaf(cs[u].y, B, sum));
+        }
+        return sum;
+    };
+
+    for (; tp < n_pairs; tp += n_warps) {
+        float2 cs0[NP], cs1[NP];
+        table(p0, cs0);
+        table(p1, cs1);
+        float s0 = row_score(raw0, cs0);
+        float s1 = row_score(raw1, cs1);
+        const int j0 = 2 * tp;
+        if (tp + n_warps < n_pairs) request(tp + n_warps);           // the next two rows travel while these are reduced
+        // both sums with six shuffles: after the first exchange the lower half-warp carries token 0, the upper token 1
+        s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+        s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+        float s = lane < 16 ? s0 : s1;
 #pragma unroll
-            for (int c = 0; c < CP; ++c) {
-                float k0[PER], k1[PER];
-                Elem<T>::unpack(raw[2 * c], k0);
-                Elem<T>::unpack(raw[2 * c + 1], k1);
-#pragma unroll
-                for (int u = 0; u < NP; ++u) {
-                    const float2 ka = make_float2(k0[2 * u], k1[2 * u]), kb = make_float2(k0[2 * u + 1], k1[2 * u + 1]);
-                    pc_fma2(A2[u], qa[c][u], ka);
-                    pc_fma2(A2[u], qb[c][u], kb);
-                    pc_fma2(B2[u], qb[c][u], ka);
-                    pc_fma2(C2[u], qa[c][u], kb);
-                }
-            }
-            if constexpr (CPL & 1) {
-                float k0[PER];
-                Elem<T>::unpack(raw[CPL - 1], k0);
-#pragma unroll
-                for (int u = 0; u < NP; ++u) {
-                    A1[u] = fmaf(qa1[u], k0[2 * u], fmaf(qb1[u], k0[2 * u + 1], A1[u]));
-                    B1[u] = fmaf(qb1[u], k0[2 * u], fmaf(-qa1[u], k0[2 * u + 1], B1[u]));
-                }
-            }
-            float sum = 0.f;
-#pragma unroll
-            for (int u = 0; u < NP; ++u) {
-                const float A = (A2[u].x + A2[u].y) + A1[u];
-                const float B = ((B2[u].x + B2[u].y) - (C2[u].x + C2[u].y)) + B1[u];
-                sum = fmaf(cs[u].x, A, fmaf(cs[u].y, B, sum));
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) {
-                float r = sum * scale;
+        for (int o = 8; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if ((lane & 15) == 0) {
+            const int j = j0 + (lane >> 4);
+            if (j < n_src) {
+                float r = s * scale;
                 if (valid && !valid[j]) r = -INFINITY;
                 scores[j] = r;
             }
         }
-        __syncwarp();
-        if (lane == 0) pc_mbar_arrive(empty(s));
     }
 }
 
@@ -419,51 +389,63 @@ __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict_
     }
 }
 
-// Enqueue pooling and scoring on caller-given scratch (a context's, or the library's fixed array).
+// Enqueue the query pass and the scoring kernel on caller-given scratch (a context's, or the library's fixed array).
+// fx: the fixed-point accumulator of this call, all zero on entry; fx_clear: the accumulator the scoring kernel clears
+// for the next call, or NULL; q_rot / q_scale: where the rotated queries go as well and the factor folded into them.
 template <typename T>
-pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev &rope, float *partial, float *pooled,
-                        int32_t *status, const void *hist_k, const int32_t *hist_pos, int n_src,
-                        const void *q, const int32_t *q_pos, int32_t n_q, const uint8_t *valid, float *scores,
+pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev &rope, long long *fx, long long *fx_clear,
+                        int32_t *status, const void *hist_k, const int32_t *hist_pos, int n_src, const void *q,
+                        const int32_t *q_pos, int32_t n_q, const uint8_t *valid, float *scores, void *q_rot, float q_scale,
                         cudaStream_t stream, pc_ctx *marks) {
+    constexpr int PER = Elem<T>::PER16;
     const int row = D.n_kv_heads * D.head_dim;
     const int group = D.n_q_heads / D.n_kv_heads;
-    const int pool_blocks = std::min<int>(PC_QPOOL_BLOCKS, (n_q + QPOOL_BATCH - 1) / QPOOL_BATCH);
+    const int q_row = D.n_q_heads * D.head_dim;
+    const int q_chunks = q_row / PER, chunks = row / PER;            // 16-byte chunks per query row / key row
+    if (chunks % 32 || q_chunks % 32 || (32 * PER) % D.head_dim) return PC_ERR_UNSUPPORTED;
+    const int warps = std::max(1, std::min<int>(QPREP_MAX_WARPS, (int)((200u * 1024u) / ((size_t)q_row * sizeof(float)))));
+    const int q_smem = warps * q_row * (int)sizeof(float);
+    const int q_blocks = (n_q + warps - 1) / warps;
+    int dev_id = 0;
+    PC_CUDA_TRY(cudaGetDevice(&dev_id));
+    if (dev_id < 0 || dev_id >= PC_MAX_DEVICES) return PC_ERR_UNSUPPORTED;
     if (marks) pc_mark(marks, PC_MARK_SCORE0, stream);
-#define PC_QPOOL_ARGS static_cast<const T *>(q), q_pos, n_q, D.n_q_heads, group, D.head_dim, rope, partial, status
-    switch (group) {
-    case 1: PC_LAUNCH((k_qpool<T, 1>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
-    case 2: PC_LAUNCH((k_qpool<T, 2>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
-    case 3: PC_LAUNCH((k_qpool<T, 3>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
-    case 4: PC_LAUNCH((k_qpool<T, 4>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
-    default: PC_LAUNCH((k_qpool<T, 0>), dim3(pool_blocks), dim3(QPOOL_THREADS), 0, stream, PC_QPOOL_ARGS); break;
+#define PC_QPREP_CASE(QCPL)                                                                                          \
+    {                                                                                                               \
+        static int smem_of[PC_MAX_DEVICES] = {};                      /* largest dynamic size allowed so far */      \
+        if (q_smem > 48 * 1024 && smem_of[dev_id] < q_smem) {                                                       \
+            PC_CUDA_TRY(cudaFuncSetAttribute(k_qprep<T, QCPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, q_smem)); \
+            smem_of[dev_id] = q_smem;                                                                               \
+        }                                                                                                           \
+        PC_LAUNCH((k_qprep<T, QCPL>), dim3(q_blocks), dim3(warps * 32), q_smem, stream, static_cast<const T *>(q), q_pos, n_q, \
+                  D.n_q_heads, group, D.head_dim, q_chunks / 32, rope, q_rot ? q_scale : 1.0f, static_cast<T *>(q_rot),        \
+                  reinterpret_cast<unsigned long long *>(fx), status);                                              \
     }
-#undef PC_QPOOL_ARGS
-    PC_CUDA_TRY(cudaGetLastError());
-    PC_LAUNCH(k_qpool_reduce, dim3((row + 31) / 32), dim3(1024), 0, stream, partial, pool_blocks, row, 1.f / (float)n_q, pooled);
+    switch (q_chunks / 32) {
+    case 12: PC_QPREP_CASE(12) break;      // 24 query heads x 128 bf16
+    case 4: PC_QPREP_CASE(4) break;
+    case 2: PC_QPREP_CASE(2) break;
+    default: PC_QPREP_CASE(0) break;
+    }
+#undef PC_QPREP_CASE
     PC_CUDA_TRY(cudaGetLastError());
     if (marks) pc_mark(marks, PC_MARK_QPOOL, stream);
     const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
-    const int chunks = row / Elem<T>::PER16;          // 16-byte chunks per token row
-    if (chunks % 32) return PC_ERR_UNSUPPORTED;
-    const int n_tiles = (n_src + SCORE_TOK - 1) / SCORE_TOK;
+    const double fx_scale = 1.0 / (4294967296.0 * (double)n_q * (double)(q_rot ? q_scale : 1.0f));
+    const int n_pairs = (n_src + 1) / 2;
     const T *k = static_cast<const T *>(hist_k);
 #define PC_SCORE_CASE(CPL)                                                                                          \
     case CPL: {                                                                                                     \
-        const int smem = SCORE_STAGES * (SCORE_TOK * CPL * 512 + SCORE_TOK * 16);                                   \
         /* resident blocks per SM of this instance (the grid is persistent), looked up once per device */          \
         static int per_sm_of[PC_MAX_DEVICES] = {};                                                                  \
-        int dev_id = 0;                                                                                             \
-        PC_CUDA_TRY(cudaGetDevice(&dev_id));                                                                        \
-        if (dev_id < 0 || dev_id >= PC_MAX_DEVICES) return PC_ERR_UNSUPPORTED;                                      \
         if (per_sm_of[dev_id] == 0) {                                                                               \
-            PC_CUDA_TRY(cudaFuncSetAttribute(k_score<T, CPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));  \
             int occ = 0;                                                                                            \
-            PC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_score<T, CPL>, SCORE_THREADS, smem)); \
+            PC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_score<T, CPL>, SCORE_THREADS, 0));    \
             per_sm_of[dev_id] = std::max(1, occ);                                                                   \
         }                                                                                                           \
-        const int blocks = std::max(1, std::min(n_tiles, sm_count * per_sm_of[dev_id]));                            \
-        PC_LAUNCH((k_score<T, CPL>), dim3(blocks), dim3(SCORE_THREADS), smem, stream, k, hist_pos, valid, n_src, D.head_dim, scale, rope, \
-                                                                 pooled, scores, status);                          \
+        const int blocks = std::max(1, std::min((n_pairs + SCORE_WARPS - 1) / SCORE_WARPS, sm_count * per_sm_of[dev_id])); \
+        PC_LAUNCH((k_score<T, CPL>), dim3(blocks), dim3(SCORE_THREADS), 0, stream, k, hist_pos, valid, n_src, D.head_dim, scale, rope, \
+                  static_cast<const long long *>(fx), fx_scale, fx_clear, scores, status);                          \
     } break;
     switch (chunks / 32) {
         PC_SCORE_CASE(1) PC_SCORE_CASE(2) PC_SCORE_CASE(3) PC_SCORE_CASE(4) PC_SCORE_CASE(6) PC_SCORE_CASE(8)
@@ -475,21 +457,12 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
     return PC_OK;
 }
 
-template <typename T>
-pc_status launch_score(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q,
-                       const uint8_t *valid, float *scores, cudaStream_t stream) {
-    return enqueue_score<T>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_partial, ctx->qpool, ctx->status,
-                            src->history.k, src->history.pos, src->history.n_tokens, q, q_pos, n_q, valid, scores, stream,
-                            ctx);
-}
-
 }  // namespace
 
-extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q,
-                              const int32_t *budget, const uint8_t *valid, const float *scores_override, float *scores,
-                              int32_t *sel_idx, void *stream_) {
+pc_status pc_score_impl(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q, const int32_t *budget,
+                        const uint8_t *valid, const float *scores_override, float *scores, int32_t *sel_idx, void *q_rot_out,
+                        cudaStream_t stream) {
     if (!ctx || !src || !budget) return PC_ERR_INVALID_ARG;
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int n_frames = src->n_frames;
     if (n_frames < 0 || (n_frames > 0 && !src->frame_count)) return PC_ERR_INVALID_ARG;
     if (n_frames > PC_MAX_FRAMES) return PC_ERR_CAPACITY;
@@ -515,10 +488,23 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
             if (!q || !q_pos || n_q <= 0 || !scores) return PC_ERR_INVALID_ARG;
             if (!pc_aligned16(q) || !pc_aligned16(q_pos) || !pc_aligned16(scores)) return PC_ERR_INVALID_ARG;
             if (n_q > ctx->desc.max_q) return PC_ERR_CAPACITY;
+            const size_t row = (size_t)ctx->desc.n_kv_heads * ctx->desc.head_dim;
+            if (ctx->qpool_dirty) {          // an earlier call stopped between the query pass and the scoring kernel
+                PC_CUDA_TRY(cudaMemsetAsync(ctx->qpool_fx, 0, 2 * row * sizeof(long long), stream));
+                ctx->qpool_dirty = 0;
+            }
+            long long *fx = ctx->qpool_fx + (size_t)ctx->qpool_turn * row, *fx_next = ctx->qpool_fx + (size_t)(ctx->qpool_turn ^ 1) * row;
+            ctx->qpool_dirty = 1;
+            const float q_scale = pc_q_rot_scale(ctx->desc.head_dim);
             st = ctx->desc.dtype == PC_BF16
-                     ? launch_score<__nv_bfloat16>(ctx, src, q, q_pos, n_q, valid, scores, stream)
-                     : launch_score<float>(ctx, src, q, q_pos, n_q, valid, scores, stream);
+                     ? enqueue_score<__nv_bfloat16>(ctx->desc, ctx->sm_count, ctx->rope, fx, fx_next, ctx->status, src->history.k,
+                                                    src->history.pos, n_src, q, q_pos, n_q, valid, scores, q_rot_out, q_scale, stream, ctx)
+                     : enqueue_score<float>(ctx->desc, ctx->sm_count, ctx->rope, fx, fx_next, ctx->status, src->history.k,
+                                            src->history.pos, n_src, q, q_pos, n_q, valid, scores, nullptr, 1.0f, stream, ctx);
             if (st != PC_OK) return st;
+            ctx->qpool_dirty = 0;
+            ctx->qpool_turn ^= 1;
+            if (q_rot_out) ctx->q_rot_n = n_q;
         }
         select_on = scores;
     } else if (reinterpret_cast<uintptr_t>(scores_override) & 3) {      // read element by element: any float address will do
@@ -533,6 +519,13 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
     return PC_OK;
 }
 
+extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q,
+                              const int32_t *budget, const uint8_t *valid, const float *scores_override, float *scores,
+                              int32_t *sel_idx, void *stream_) {
+    return pc_score_impl(ctx, src, q, q_pos, n_q, budget, valid, scores_override, scores, sel_idx, nullptr,
+                         static_cast<cudaStream_t>(stream_));
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Scoring without a context and without any allocation.
 //
@@ -540,8 +533,8 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
 // was handed to its own arena at start-up and whose policy forbids driver allocations afterwards, or a
 // latency-critical thread that cannot take the device-wide synchronisation a cudaMalloc / cudaFree implies.  Such
 // callers cannot create a pc_ctx (pc_create allocates), so everything a context would hold for scoring — the rotary
-// table, the pooled query and its per-block partials — lives in one file-scope device array
-// of fixed size that every GPU loading this library carries until the process exits.
+// table and the fixed-point accumulator of the pooled query — lives in one file-scope device array of fixed size
+// that every GPU loading this library carries until the process exits.
 //
 // In host code the array's name is only a handle; the device address is obtained once per device with
 // cudaGetSymbolAddress while that device is current, and that pointer (never the symbol) is what kernels receive.
@@ -550,20 +543,23 @@ namespace {
 
 constexpr int STATIC_MAX_ROW = 1024;          // n_kv_heads * head_dim
 constexpr int STATIC_MAX_ROPE = 32768;        // rotary table entries: sum over axes of max_pos * pairs on that axis
+constexpr int STATIC_MAX_QROW = 12288;        // n_q_heads * head_dim: one row of the query pass's shared-memory slab
 constexpr int STATIC_MAX_DEVICES = PC_MAX_DEVICES;
 
-constexpr size_t STATIC_OFF_POOLED = 256;  /* first 256 bytes unused */                                                  // float [STATIC_MAX_ROW]
-constexpr size_t STATIC_OFF_PARTIAL = STATIC_OFF_POOLED + STATIC_MAX_ROW * sizeof(float);  // float [PC_QPOOL_BLOCKS][STATIC_MAX_ROW]
-constexpr size_t STATIC_OFF_ROPE = STATIC_OFF_PARTIAL + (size_t)PC_QPOOL_BLOCKS * STATIC_MAX_ROW * sizeof(float);
-constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);   // 790,784 bytes
+constexpr size_t STATIC_OFF_FX = 256;  /* first 256 bytes unused */                             // long long [STATIC_MAX_ROW]
+constexpr size_t STATIC_OFF_ROPE = STATIC_OFF_FX + STATIC_MAX_ROW * sizeof(long long);         // float2 [STATIC_MAX_ROPE]
+constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);    // 270,592 bytes
 
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
 
 // Rotary table in fp64, stored as fp32 (cos, sin): entry (axis a, position p, column m) = p * base^(-m / n_axis[a]).
-__global__ void __launch_bounds__(256) k_rope_table(float2 *__restrict__ tab, pc_rope_dev rope, double base, int total) {
+// The first `clear` 64-bit words of `fx` are set to zero as well (the accumulator of the pooled query).
+__global__ void __launch_bounds__(256) k_rope_table(float2 *__restrict__ tab, pc_rope_dev rope, double base, int total,
+                                                    long long *__restrict__ fx, int clear) {
     pc_grid_dep_launch();
     pc_grid_dep_wait();
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < clear) fx[e] = 0;
     if (e >= total) return;
     const int a = e >= rope.off[2] ? 2 : (e >= rope.off[1] ? 1 : 0);
     const int na = rope.n_axis[a], local = e - rope.off[a];
@@ -594,8 +590,7 @@ template <typename T>
 pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const void *hist_k, const int32_t *hist_pos,
                               int32_t n_src, const void *q, const int32_t *q_pos, int32_t n_q, const uint8_t *valid,
                               float *scores, int32_t *status, cudaStream_t stream) {
-    float *pooled = reinterpret_cast<float *>(base + STATIC_OFF_POOLED);
-    float *partial = reinterpret_cast<float *>(base + STATIC_OFF_PARTIAL);
+    long long *fx = reinterpret_cast<long long *>(base + STATIC_OFF_FX);
     float2 *tab = reinterpret_cast<float2 *>(base + STATIC_OFF_ROPE);
 
     pc_rope_dev rope;
@@ -607,16 +602,17 @@ pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const
         total += D.max_pos[a] * rope.n_axis[a];
     }
     rope.tab = tab;
-    // the array keeps whatever the last call left; the table, the partials and the pooled query are all rewritten before
-    // they are read, and nothing has to start at zero
-    PC_LAUNCH(k_rope_table, dim3((total + 255) / 256), dim3(256), 0, stream, tab, rope, D.rope_base, total);
+    // the array keeps whatever the last call left: the table is rewritten before it is read, and the accumulator of the
+    // pooled query, which must start at zero, is cleared by the same kernel
+    const int row = D.n_kv_heads * D.head_dim;
+    PC_LAUNCH(k_rope_table, dim3((std::max(total, row) + 255) / 256), dim3(256), 0, stream, tab, rope, D.rope_base, total, fx, row);
     PC_CUDA_TRY(cudaGetLastError());
 
     int sm_count = 0, dev = 0;
     PC_CUDA_TRY(cudaGetDevice(&dev));
     PC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    return enqueue_score<T>(D, sm_count, rope, partial, pooled, status, hist_k, hist_pos, n_src, q, q_pos, n_q,
-                            valid, scores, stream, nullptr);
+    return enqueue_score<T>(D, sm_count, rope, fx, nullptr, status, hist_k, hist_pos, n_src, q, q_pos, n_q, valid, scores, nullptr,
+                            1.0f, stream, nullptr);
 }
 
 }  // namespace
@@ -635,19 +631,18 @@ extern "C" pc_status pc_score_tokens_static(const pc_layer_desc *desc, const voi
     if (D.n_q_heads <= 0 || D.n_kv_heads <= 0 || D.n_q_heads % D.n_kv_heads) return PC_ERR_UNSUPPORTED;
     if (!(D.rope_base > 1.0)) return PC_ERR_INVALID_ARG;
     const int row = D.n_kv_heads * D.head_dim;
-    const int chunks = row / (D.dtype == PC_BF16 ? 8 : 4);
-    if (chunks % 32) return PC_ERR_UNSUPPORTED;
+    const int per = D.dtype == PC_BF16 ? 8 : 4;
+    if ((row / per) % 32 || (D.n_q_heads * D.head_dim / per) % 32) return PC_ERR_UNSUPPORTED;
     int64_t rope_entries = 0;
     for (int a = 0; a < 3; ++a) {
         if (D.max_pos[a] <= 0 || D.max_pos[a] > (1 << 20)) return PC_ERR_INVALID_ARG;
         rope_entries += (int64_t)D.max_pos[a] * ((D.head_dim / 2 - a + 2) / 3);
     }
-    if (row > STATIC_MAX_ROW || rope_entries > STATIC_MAX_ROPE ||
-        (size_t)D.n_q_heads * D.head_dim * sizeof(float) > 48 * 1024) {
+    if (row > STATIC_MAX_ROW || rope_entries > STATIC_MAX_ROPE || D.n_q_heads * D.head_dim > STATIC_MAX_QROW) {
         fprintf(stderr,
                 "packcache: pc_score_tokens_static: shape exceeds the fixed scratch (n_kv_heads*head_dim %d > %d, or "
-                "rotary table %lld > %d entries, or n_q_heads*head_dim > 12288)\n",
-                row, STATIC_MAX_ROW, (long long)rope_entries, STATIC_MAX_ROPE);
+                "rotary table %lld > %d entries, or n_q_heads*head_dim > %d)\n",
+                row, STATIC_MAX_ROW, (long long)rope_entries, STATIC_MAX_ROPE, STATIC_MAX_QROW);
         return PC_ERR_CAPACITY;
     }
     unsigned char *base = nullptr;

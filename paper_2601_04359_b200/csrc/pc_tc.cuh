@@ -12,41 +12,14 @@ constexpr int TILE_BYTES = 2 * HALF_BYTES;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: gives up after about one second, or at once when another thread of the CTA already gave up.
+// mbarrier helpers and the bounded wait are the library-wide ones (pc_common.cuh)
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) { pc_mbar_init(bar, count); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) { pc_mbar_expect_tx(bar, bytes); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) { pc_mbar_arrive(bar); }
+__device__ __forceinline__ uint64_t global_ns() { return pc_global_ns(); }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
-                                          int where = PC_WHERE_ATTN_WAIT) {
-    for (int i = 0; i < 2048; ++i)
-        if (mbar_try(bar, parity)) return true;
-    const uint64_t t0 = global_ns();
-    for (;;) {
-        if (mbar_try(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_ns() - t0 > 1000000000ull) {
-            *abort_flag = 1;
-            pc_flag(status, PC_ERR_TIMEOUT, where);
-            return false;
-        }
-    }
+                                          int where = PC_WHERE_ATTN_WAIT, uint32_t limit_us = 0) {
+    return pc_mbar_wait(bar, parity, abort_flag, status, where, limit_us);
 }
 
 // True in exactly one lane of a converged warp.  The compiler turns work predicated on elect.sync into single-issue
@@ -170,62 +143,6 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
 constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t IDESC_QK = IDESC_BASE;               // A, B K-major
 constexpr uint32_t IDESC_PV = IDESC_BASE | (1u << 16);  // B (V) MN-major
-
-// ---- CTA pairs (`cta_group::2`): two CTAs of a cluster run one multiply-add of M = 256 — each its own 128 rows of A and
-// of D, each holding half of B (N split) in its own shared memory.  The even CTA of the pair (cluster rank 0) issues.
-// arrive on a barrier that may live in the other CTA of the cluster (address from peer_addr)
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {   // own barrier, arrivals from the whole cluster
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
-                                                  int where = PC_WHERE_ATTN_WAIT) {
-    for (int i = 0; i < 2048; ++i)
-        if (mbar_try_cluster(bar, parity)) return true;
-    const uint64_t t0 = global_ns();
-    for (;;) {
-        if (mbar_try_cluster(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_ns() - t0 > 1000000000ull) {
-            *abort_flag = 1;
-            pc_flag(status, PC_ERR_TIMEOUT, where);
-            return false;
-        }
-    }
-}
-// TMA load of this CTA's share of a pair's operand; the bytes are counted on a barrier of the issuing (even) CTA
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t leader_bar) {
-    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(leader_bar) : "memory");
-}
-// commit of the pair's multiply-adds: one arrival on the barrier at this shared-memory offset in each of the two CTAs (two
-// commits, the second through the peer's cluster address; each tracks every multiply-add issued before it)
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer_addr(bar, 1)) : "memory");
-}
-__device__ __forceinline__ void mma_ss_pair(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void mma_ts_pair(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-                 ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
-}
-// instruction descriptor of a pair: M = 256 over the two CTAs, N = 128
-constexpr uint32_t IDESC_PAIR_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((256u >> 4) << 24);
-constexpr uint32_t IDESC_PAIR_QK = IDESC_PAIR_BASE;
-constexpr uint32_t IDESC_PAIR_PV = IDESC_PAIR_BASE | (1u << 16);
-// MN-major B operand one swizzle atom (64 elements) wide: 8-row groups 1024 B apart, no second atom
-__device__ __forceinline__ uint64_t desc_mnmajor64(uint32_t addr) {
-    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
-           ((uint64_t)2 << 61);
-}
 
 // ------------------------------------------------------------------------------------------------ tensor maps (host)
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,

@@ -120,7 +120,11 @@ extern "C" pc_status pc_window_append_masked(pc_window *w, const pc_segment *fra
     if (n_valid < 0 || n_valid > frame->n_tokens) return PC_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     pc_segment &A = w->buf[w->active];
-    if ((int64_t)A.n_tokens + n_valid > A.capacity || frame->n_tokens > w->scratch_capacity) return PC_ERR_CAPACITY;
+    // the grown buffer must fit the caller's score / index scratch as well (the next update scores every token of it), and
+    // the mask's row indices go through that index scratch
+    if ((int64_t)A.n_tokens + n_valid > A.capacity || (int64_t)A.n_tokens + n_valid > w->scratch_capacity ||
+        frame->n_tokens > w->scratch_capacity)
+        return PC_ERR_CAPACITY;
     if ((int)w->count.size() + 1 > PC_MAX_FRAMES) return PC_ERR_CAPACITY;
     if (n_valid > 0) {
         const size_t row = (size_t)w->ctx->desc.n_kv_heads * w->ctx->desc.head_dim * w->ctx->elem_size;
@@ -128,7 +132,7 @@ extern "C" pc_status pc_window_append_masked(pc_window *w, const pc_segment *fra
                   w->ctx->status);
         st = pc_launch_pack(w->ctx, frame->k, frame->v, frame->pos, w->sel_idx, n_valid, frame->n_tokens, 0,
                             static_cast<char *>(A.k) + (size_t)A.n_tokens * row, static_cast<char *>(A.v) + (size_t)A.n_tokens * row,
-                            A.pos + 4 * (size_t)A.n_tokens, stream);
+                            A.pos + 4 * (size_t)A.n_tokens, nullptr, stream);
         if (st != PC_OK) return st;
     }
     A.n_tokens += n_valid;

@@ -17,6 +17,7 @@ from paper_2601_04359_b200.device import DeviceLayer, dev, host, idev, make_ctx,
 pytestmark = pytest.mark.gpu
 
 BF16_ATOL = 2e-2
+BF16_KERNEL_ATOL = 4e-3   # what the kernel may add beyond the rounding of its bf16 output (see check_bf16_attention)
 F32_RTOL = 1e-4
 
 
@@ -32,9 +33,24 @@ def _ok(ctx):
     assert pc.pc_poll_status(ctx) == pc.PC_OK
 
 
+def bf16_ulp(x: np.ndarray) -> np.ndarray:
+    """Spacing of bfloat16 numbers at |x| (8 significant bits), floored at the spacing of 2^-6."""
+    return 2.0 ** (np.floor(np.log2(np.maximum(np.abs(x), 2.0 ** -6))) - 7)
+
+
+def check_bf16_attention(got: np.ndarray, want: np.ndarray):
+    """The stated bound (2e-2 max-abs) and a sharper element-wise one.  The output is a bf16 number, so half a spacing of
+    error comes from storing it: on the V outlier channels (values near 4, spacing 2^-5) that alone is 1.6e-2 and
+    nearly fills the stated bound.  What the kernel itself adds (bf16 rounding of the rotated operands and of the
+    probabilities) is bounded apart: |got - want| <= ulp_bf16(want) + 4e-3."""
+    err = np.abs(got - want)
+    assert err.max() <= BF16_ATOL
+    assert (err <= bf16_ulp(want) + BF16_KERNEL_ATOL).all(), float((err - bf16_ulp(want)).max())
+
+
 def _check_attention(cfg, got: np.ndarray, want: np.ndarray):
     if cfg.dtype == wl.BF16:
-        assert np.abs(got - want).max() <= BF16_ATOL
+        check_bf16_attention(got, want)
     else:
         scale = np.abs(want).max()
         assert np.abs(got - want).max() <= F32_RTOL * scale
@@ -172,43 +188,6 @@ def test_attention_key_ranges_merge_like_one_range(cluster):
     for o in outs[1:]:                       # the split only changes fp32 rounding order: at most a bf16 ulp or two
         assert (np.abs(o - outs[0]) <= 2.0 ** -6 * np.maximum(np.abs(outs[0]), 0.5)).all()
     ctx.close()
-
-
-# ------------------------------------------------------------------------------------------- CTA-pair kernel
-@pytest.mark.parametrize("shape", ["group4", "four_row_tiles"])
-def test_cta_pair_attention_gives_the_bits_of_the_single_cta_kernel(shape):
-    """The kernel that issues its multiply-adds for pairs of CTAs (each CTA holds half of every key / value tile) against
-    the oracle and, bit for bit, against the default kernel, for one to four key ranges with ragged segments."""
-    if shape == "group4":        # four query heads per KV head, two row tiles: eight query tiles per KV head
-        cfg = replace(wl.small_bf16(n_frames=3, grid=(12, 21), n_text=130, total=500, keep_full=1, seed=50), n_q_heads=32, n_kv_heads=8)
-    else:                        # three query heads per KV head, four row tiles (the last one ragged)
-        cfg = wl.small_bf16(n_frames=2, grid=(16, 25), n_text=37, total=400, keep_full=1, seed=51)
-    L = wl.make_layer(cfg, with_current=True)
-    D = DeviceLayer(L)
-    ctx = make_ctx(cfg)
-    segs = [(L.anchor_k, L.anchor_v, L.anchor_pos), (L.hist_k, L.hist_v, L.hist_pos), (L.cur_k, L.cur_v, L.q_pos)]
-    want, want_lse = oracle.attend(L.q, L.q_pos, segs, cfg.rope_base, want_lse=True)
-    for n in (1, 2, 3, 4):
-        pc.pc_set_kv_splits(ctx, n)
-        pc.pc_set_attend_impl(ctx, 0)
-        a, la = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos, want_lse=True)
-        a, la = a.clone(), la.clone()
-        pc.pc_set_attend_impl(ctx, 2)
-        b, lb = pc.pc_attend_frame(ctx, D.cache, D.current, D.q, D.q_pos, want_lse=True)
-        _ok(ctx)
-        assert torch.equal(a, b) and torch.equal(la, lb)
-        assert np.abs(host(b).astype(np.float64) - want).max() <= BF16_ATOL
-        assert np.abs(host(lb) - want_lse).max() <= 2e-2
-    # a shape whose query tiles per KV head do not divide by four runs the default kernel under the same setting
-    cfg3 = wl.small_bf16(n_frames=2, grid=(8, 9), seed=52)
-    L3 = wl.make_layer(cfg3)
-    D3 = DeviceLayer(L3)
-    ctx3 = make_ctx(cfg3)
-    a = pc.pc_attend_frame(ctx3, D3.cache, None, D3.q, D3.q_pos).clone()
-    pc.pc_set_attend_impl(ctx3, 2)
-    assert torch.equal(a, pc.pc_attend_frame(ctx3, D3.cache, None, D3.q, D3.q_pos))
-    _ok(ctx3)
-    ctx.close(); ctx3.close()
 
 
 # ------------------------------------------------------------------------------------------- prepared key set
@@ -477,12 +456,22 @@ def test_full_size_sampled_against_oracle(name):
 
     out, lse = pc.pc_attend_frame(ctx, dst, None, D.q, D.q_pos, want_lse=True)
     _ok(ctx)
-    rows = np.stack([rng.integers(0, cfg.n_q, size=96), rng.integers(0, cfg.n_q_heads, size=96)], axis=1).astype(np.int32)
-    rows[0] = (0, 0); rows[1] = (cfg.n_q - 1, cfg.n_q_heads - 1); rows[2] = (1007, 5); rows[3] = (896, 23)
+    if name == "lumos47":
+        # the benchmark's configuration: every (query, head) row, so that every (row tile, head, key range) of the launch
+        # the bench times is compared (the oracle takes about 11 s for them on 16 cores)
+        rows = np.stack(np.meshgrid(np.arange(cfg.n_q), np.arange(cfg.n_q_heads), indexing="ij"), axis=-1).reshape(-1, 2)
+        rows = rows.astype(np.int32)
+    else:
+        # one row of every (row tile, head) and a random sample on top
+        tiles = [(min(t * 128 + int(rng.integers(128)), cfg.n_q - 1), h) for t in range((cfg.n_q + 127) // 128)
+                 for h in range(cfg.n_q_heads)]
+        rand = np.stack([rng.integers(0, cfg.n_q, size=96), rng.integers(0, cfg.n_q_heads, size=96)], axis=1)
+        rows = np.concatenate([np.array(tiles), rand]).astype(np.int32)
+        rows[0] = (0, 0); rows[1] = (cfg.n_q - 1, cfg.n_q_heads - 1); rows[2] = (1007, 5); rows[3] = (896, 23)
     want, want_lse = oracle.attend(L.q, L.q_pos, [(L.anchor_k, L.anchor_v, L.anchor_pos), (wk, wv, wp)], rows=rows,
                                    want_lse=True)
     o = host(out)
-    assert np.abs(o[rows[:, 0], rows[:, 1]] - want).max() <= BF16_ATOL
+    check_bf16_attention(o[rows[:, 0], rows[:, 1]], want)
     assert np.abs(host(lse)[rows[:, 0], rows[:, 1]] - want_lse).max() <= 2e-2
     assert np.isfinite(o).all()
     ctx.close()
@@ -498,12 +487,14 @@ def test_full_cache_comparator_at_24_frames():
     out, lse = pc.pc_attend_frame(ctx, D.cache, None, D.q, D.q_pos, want_lse=True)
     _ok(ctx)
     rng = np.random.default_rng(2)
-    rows = np.stack([rng.integers(0, cfg.n_q, size=48), rng.integers(0, cfg.n_q_heads, size=48)], axis=1).astype(np.int32)
+    # one row of every (row tile, head), so that every tile / head / key-range combination of the launch is compared
+    rows = np.array([(min(t * 128 + int(rng.integers(128)), cfg.n_q - 1), h) for t in range((cfg.n_q + 127) // 128)
+                     for h in range(cfg.n_q_heads)], dtype=np.int32)
     rows[0] = (0, 0); rows[1] = (cfg.n_q - 1, cfg.n_q_heads - 1)
     want, want_lse = oracle.attend(L.q, L.q_pos, [(L.anchor_k, L.anchor_v, L.anchor_pos), (L.hist_k, L.hist_v, L.hist_pos)],
                                    rows=rows, want_lse=True)
     o = host(out)
-    assert np.abs(o[rows[:, 0], rows[:, 1]] - want).max() <= BF16_ATOL
+    check_bf16_attention(o[rows[:, 0], rows[:, 1]], want)
     assert np.abs(host(lse)[rows[:, 0], rows[:, 1]] - want_lse).max() <= 2e-2
     assert np.isfinite(o).all()
     ctx.close()
@@ -538,5 +529,5 @@ def test_layer_stack_cells_sampled(layer, frac, kind, param):
     rng = np.random.default_rng(layer)
     rows = np.stack([rng.integers(0, cfg.n_q, size=32), rng.integers(0, cfg.n_q_heads, size=32)], axis=1).astype(np.int32)
     want = oracle.attend(L.q, L.q_pos, [(L.anchor_k, L.anchor_v, L.anchor_pos), (wk, wv, wp)], rows=rows)
-    assert np.abs(host(out)[rows[:, 0], rows[:, 1]] - want).max() <= BF16_ATOL
+    check_bf16_attention(host(out)[rows[:, 0], rows[:, 1]], want)
     ctx.close()

@@ -1,7 +1,7 @@
 """Seeded random shapes through the whole path on the GPU, every stage against the oracle: head groupings from 2/2 to
 32/8, frames of 1 to 550 tokens, 0 to 200 text tokens, all four decay kernels, budgets from nothing to everything, with
-and without the current frame, 1-4 key ranges (or the automatic choice), both merge forms, the default and the CTA-pair
-attention kernel, and the attention mass where the tensor-core path takes the shape."""
+and without the current frame, 1-4 key ranges (or the automatic choice), both merge forms, the tensor-core and the
+CUDA-core attention kernel, and the attention mass where the tensor-core path takes the shape."""
 from __future__ import annotations
 
 from dataclasses import replace
@@ -35,7 +35,7 @@ def test_random_shapes_against_the_oracle(seed):
         cfg = replace(wl.small_bf16(n_frames=n_frames, grid=grid, n_text=n_text, total=total, kind=kind, param=DECAY[kind],
                                     keep_full=keep_full, seed=2000 + 10 * seed + case), n_q_heads=hq, n_kv_heads=hkv)
         with_cur, splits, cluster = bool(rng.integers(2)), int(rng.integers(0, 5)), bool(rng.integers(2))
-        impl = [0, 0, 2][rng.integers(3)]
+        impl = [0, 0, 1][rng.integers(3)]
         what = f"{cfg.name} heads {hq}/{hkv} text {n_text} budget {total}/{keep_full} decay {kind} current {with_cur} ranges {splits} " \
                f"cluster {cluster} impl {impl}"
         L = wl.make_layer(cfg, with_current=True)
@@ -67,12 +67,12 @@ def test_random_shapes_against_the_oracle(seed):
         assert pc.pc_poll_status(ctx) == pc.PC_OK, what
         assert np.abs(host(out).astype(np.float64) - want).max() <= 2e-2, what
         assert np.abs(host(lse) - want_lse).max() <= 2e-2, what
-        if hkv * cfg.head_dim % 256 == 0:
+        if hkv * cfg.head_dim % 256 == 0 and impl == 0:
             n_keys = sum(len(s[0]) for s in segs)
             got = host(pc.pc_attend_mass(ctx, lse, n_keys)).astype(np.float64)
             want_mass = oracle.attend_mass(L.q, L.q_pos, [(s[0], s[2]) for s in segs], cfg.rope_base)
             assert pc.pc_poll_status(ctx) == pc.PC_OK, what
-            assert (np.abs(got - want_mass) <= 1e-2 * want_mass + 1e-3 / n_keys).all(), what
+            assert (np.abs(got - want_mass) <= 2e-3 * want_mass + 1e-3 / n_keys).all(), what
         ctx.close()
 
 

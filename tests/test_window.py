@@ -280,6 +280,44 @@ def test_window_masked_append_matches_reference():
 
 
 @pytest.mark.gpu
+def test_masked_append_respects_the_smaller_buffer_like_append():
+    """Two history buffers of unequal size: the caller's score / index scratch has the size of the smaller one, so a
+    masked append that would grow the active (larger) buffer past it must be refused before anything is enqueued, as
+    the plain append is."""
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200.device import make_ctx, segment
+
+    cfg = wl.small_bf16(n_frames=4, grid=(8, 9), n_text=37, total=100, seed=14)
+    n = cfg.frame_tokens                                                     # 72 tokens per frame
+    L = wl.make_layer(cfg)
+    fr = _frames(cfg, 4, seed=15)
+    ctx = make_ctx(cfg)
+    mk = lambda cap: pc.Segment(torch.full((cap, cfg.n_kv_heads, cfg.head_dim), 5.0, dtype=torch.bfloat16, device="cuda"),
+                                torch.full((cap, cfg.n_kv_heads, cfg.head_dim), 5.0, dtype=torch.bfloat16, device="cuda"),
+                                torch.full((cap, 4), -3, dtype=torch.int32, device="cuda"), 0)
+    big, small = mk(4 * n), mk(2 * n + 10)                                   # scratch: 2n + 10 tokens
+    win = pc.Window(ctx, 8, pc.PC_HALFLIFE, 2.0, 10 ** 6, 0, segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype), big, small)
+    ones = torch.ones(n, dtype=torch.uint8, device="cuda")
+    seg = lambda f: segment(fr[f]["k"], fr[f]["v"], fr[f]["pos"], cfg.dtype)
+    win.append_masked(seg(0), ones, n)
+    win.append_masked(seg(1), ones, n)
+    guard = big.k[2 * n:].clone()
+    with pytest.raises(pc.PackCacheError) as e:                              # 3n > 2n + 10 although the buffer holds 4n
+        win.append_masked(seg(2), ones, n)
+    assert e.value.status == pc.PC_ERR_CAPACITY
+    with pytest.raises(pc.PackCacheError) as e:
+        win.append(seg(2))
+    assert e.value.status == pc.PC_ERR_CAPACITY
+    torch.cuda.synchronize()
+    assert torch.equal(big.k[2 * n:], guard) and win.state()[0].tolist() == [n, n]      # nothing was enqueued or counted
+    keep = torch.zeros(n, dtype=torch.uint8, device="cuda"); keep[:10] = 1
+    win.append_masked(seg(2), keep, 10)                                      # 2n + 10 still fits
+    assert pc.pc_poll_status(ctx) == pc.PC_OK and win.state()[0].tolist() == [n, n, 10]
+    win.close(); ctx.close()
+
+
+@pytest.mark.gpu
 def test_window_minimum_quota_matches_reference():
     import torch
     from paper_2601_04359_b200 import binding as pc
