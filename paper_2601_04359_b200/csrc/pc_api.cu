@@ -64,8 +64,8 @@ static pc_status create_on_device(pc_ctx *c) {
     PC_CUDA_TRY(cudaMalloc(&c->status, 2 * sizeof(int32_t)));
     PC_CUDA_TRY(cudaMemset(c->status, 0, 2 * sizeof(int32_t)));
     PC_CUDA_TRY(cudaMallocHost(&c->host_status, 2 * sizeof(int32_t)));
-    PC_CUDA_TRY(cudaMalloc(&c->qpool_fx, 2 * (size_t)row * sizeof(long long)));
-    PC_CUDA_TRY(cudaMemset(c->qpool_fx, 0, 2 * (size_t)row * sizeof(long long)));
+    PC_CUDA_TRY(cudaMalloc(&c->qpool_fx, ((size_t)row + 1) * sizeof(long long)));
+    PC_CUDA_TRY(cudaMemset(c->qpool_fx, 0, ((size_t)row + 1) * sizeof(long long)));
     if (desc->dtype == PC_BF16) {
         pc_status st = pc_attend_tc_scratch(desc, c->sm_count, &c->k_rot_rows, &c->part_o_floats, &c->part_ml_floats);
         if (st != PC_OK) return st;

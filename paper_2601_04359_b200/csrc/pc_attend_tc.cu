@@ -71,10 +71,10 @@ struct RopeJobs { RopeJob job[PC_MAX_SEGMENTS + 1]; int n_jobs, total_warps; };
 
 // One warp per row (a query row wider than a key row is cut into key-row-wide slices, one warp each, so that all warps
 // carry the same load).  32 lanes x 8 elements = 256 is a multiple of d, so all of a lane's chunks (lane, lane + 32, ...)
-// hold the same four rotary pairs: four table entries per lane per row, with the output scale folded in, serve every
-// chunk.  All of a row's chunks are loaded before any is used.
+// hold the same four rotary pairs: four table entries per lane per row serve every chunk; the output scale (1 for keys)
+// is applied after the rotation, exactly as the query pass of the scoring stage does, so both give the same bits.  All of a row's chunks are loaded before any is used.
 template <int CPL /* chunks per lane */>
-__device__ __forceinline__ void rope_row(const RopeJob &J, int row, int lane, const float2 (&cs)[4]) {
+__device__ __forceinline__ void rope_row(const RopeJob &J, int row, int lane, const float2 (&cs)[4], float scale) {
     const uint4 *src = reinterpret_cast<const uint4 *>(J.src) + (size_t)row * (CPL * 32) + lane;
     uint4 *dst = reinterpret_cast<uint4 *>(J.dst) + (size_t)row * (CPL * 32) + lane;
     uint4 v[CPL];
@@ -87,7 +87,7 @@ __device__ __forceinline__ void rope_row(const RopeJob &J, int row, int lane, co
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const float2 y = pc_rotate(pc_bf16_lo(w[u]), pc_bf16_hi(w[u]), cs[u]);
-            o[u] = pc_pack_bf16(y.x, y.y);
+            o[u] = pc_pack_bf16(__fmul_rn(y.x, scale), __fmul_rn(y.y, scale));
         }
         dst[c * 32] = make_uint4(o[0], o[1], o[2], o[3]);
     }
@@ -108,18 +108,15 @@ __global__ void __launch_bounds__(256) k_rope_rows(const __grid_constant__ RopeJ
     const int pair0 = ((lane * 8) % d) / 2;
     float2 cs[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-        cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_ROPE_POS);
-        cs[u].x *= J.scale;
-        cs[u].y *= J.scale;
-    }
+    for (int u = 0; u < 4; ++u) cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_ROPE_POS);
+    const float scale = J.scale;
     switch (J.chunks_per_row >> 5) {
-    case 4: rope_row<4>(J, row, lane, cs); break;        // 8 KV heads x 128
-    case 12: rope_row<12>(J, row, lane, cs); break;      // 24 query heads x 128
-    case 1: rope_row<1>(J, row, lane, cs); break;
-    case 2: rope_row<2>(J, row, lane, cs); break;
-    case 8: rope_row<8>(J, row, lane, cs); break;
-    case 16: rope_row<16>(J, row, lane, cs); break;
+    case 4: rope_row<4>(J, row, lane, cs, scale); break;        // 8 KV heads x 128
+    case 12: rope_row<12>(J, row, lane, cs, scale); break;      // 24 query heads x 128
+    case 1: rope_row<1>(J, row, lane, cs, scale); break;
+    case 2: rope_row<2>(J, row, lane, cs, scale); break;
+    case 8: rope_row<8>(J, row, lane, cs, scale); break;
+    case 16: rope_row<16>(J, row, lane, cs, scale); break;
     default:
         for (int c = 0; c < (J.chunks_per_row >> 5); ++c) {
             const uint4 *src = reinterpret_cast<const uint4 *>(J.src) + (size_t)row * J.chunks_per_row + c * 32 + lane;
@@ -130,7 +127,7 @@ __global__ void __launch_bounds__(256) k_rope_rows(const __grid_constant__ RopeJ
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const float2 y = pc_rotate(pc_bf16_lo(w[u]), pc_bf16_hi(w[u]), cs[u]);
-                o[u] = pc_pack_bf16(y.x, y.y);
+                o[u] = pc_pack_bf16(__fmul_rn(y.x, scale), __fmul_rn(y.y, scale));
             }
             *dst = make_uint4(o[0], o[1], o[2], o[3]);
         }

@@ -61,12 +61,11 @@ struct pc_ctx {
     float2 *rope_tab;          // owned
     int32_t *status;           // device [2]: code, where
     int32_t *host_status;      // pinned [2]
-    // Pooled query of the scoring pass as fixed-point sums (units of 2^-32), two buffers of Hkv*d 64-bit integers used
-    // in turn: the query pass of call n adds into buffer n & 1 (integer addition: the result does not depend on the
-    // order of the blocks), the scoring kernel of call n reads it and clears the other one for call n + 1.
-    long long *qpool_fx;       // device [2][Hkv*d], zero between uses
-    int qpool_turn;            // buffer the next query pass adds into
-    int qpool_dirty;           // 1: a call failed between the two kernels, both buffers are cleared before the next use
+    // Pooled query of the scoring pass as fixed-point sums (units of 2^-32): Hkv*d 64-bit integers and one counter word.
+    // The query pass adds into it (integer addition: the result does not depend on the order of the blocks); the
+    // scoring kernel reads it and its last block clears it again, so it is zero between calls.
+    long long *qpool_fx;       // device [Hkv*d + 1]
+    int qpool_dirty;           // 1: a call failed between the two kernels; the array is cleared before the next use
     // attention scratch (tensor-core path)
     void *k_rot;               // rotated keys, bf16 [rows][Hkv][d]
     size_t k_rot_rows;

@@ -77,11 +77,7 @@ __global__ void __launch_bounds__(QPREP_MAX_WARPS * 32) k_qprep(const T *__restr
         const int pair0 = ((lane * PER) % d) / 2;
         float2 cs[NP];
 #pragma unroll
-        for (int u = 0; u < NP; ++u) {
-            cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_QPOOL_POS);
-            cs[u].x *= out_scale;
-            cs[u].y *= out_scale;
-        }
+        for (int u = 0; u < NP; ++u) cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_QPOOL_POS);
         float *mine = slab + (size_t)warp * row_len + lane * PER;
         uint4 *dst = q_rot ? reinterpret_cast<uint4 *>(q_rot + (size_t)i * row_len) + lane : nullptr;
         auto one_chunk = [&](const uint4 &v, int c) {
@@ -96,7 +92,11 @@ __global__ void __launch_bounds__(QPREP_MAX_WARPS * 32) k_qprep(const T *__restr
             float4 *s4 = reinterpret_cast<float4 *>(mine + (size_t)c * 32 * PER);
 #pragma unroll
             for (int k = 0; k < PER / 4; ++k) s4[k] = make_float4(r[4 * k], r[4 * k + 1], r[4 * k + 2], r[4 * k + 3]);
-            if (dst) dst[c * 32] = pack_row<T>(r);
+            if (dst) {                                                  // the attention kernel's queries carry its scale
+#pragma unroll
+                for (int k = 0; k < PER; ++k) r[k] = __fmul_rn(r[k], out_scale);
+                dst[c * 32] = pack_row<T>(r);
+            }
         };
         if constexpr (QCPL > 0) {
 #pragma unroll
@@ -108,15 +108,27 @@ __global__ void __launch_bounds__(QPREP_MAX_WARPS * 32) k_qprep(const T *__restr
     __syncthreads();
     const int n_warps_used = min(warps, n_q - blockIdx.x * warps);
     const int n_out = (n_q_heads / group) * d;
-    for (int e = threadIdx.x; e < n_out; e += blockDim.x) {
-        const int g = e / d, x = e - g * d;
-        float sum = 0.f;
-        for (int w = 0; w < n_warps_used; ++w) {
-            const float *s = slab + (size_t)w * row_len + (size_t)g * group * d + x;
-            for (int h = 0; h < group; ++h) sum += s[h * d];
+    // four pooled elements per thread at a time, so that four independent sums are in flight; the order of the additions
+    // of each sum is fixed (warps ascending, heads of the group ascending)
+    for (int e0 = threadIdx.x; e0 < n_out; e0 += 4 * blockDim.x) {
+        const float *s[4];
+        float sum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int e = min(e0 + k * (int)blockDim.x, n_out - 1), g = e / d, x = e - g * d;
+            s[k] = slab + (size_t)g * group * d + x;
         }
-        const long long v = __float2ll_rn(sum * FX_ONE);
-        atomicAdd(fx + e, (unsigned long long)v);
+        for (int w = 0; w < n_warps_used; ++w)
+            for (int h = 0; h < group; ++h) {
+                const int off = w * row_len + h * d;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) sum[k] += s[k][off];
+            }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int e = e0 + k * (int)blockDim.x;
+            if (e < n_out) atomicAdd(fx + e, (unsigned long long)__float2ll_rn(sum[k] * FX_ONE));
+        }
     }
 }
 
@@ -136,9 +148,8 @@ constexpr int SCORE_THREADS = SCORE_WARPS * 32;
 template <typename T, int CPL /* chunks per lane */>
 __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict__ k, const int32_t *__restrict__ k_pos,
                                                             const uint8_t *__restrict__ valid, int n_src, int d, float scale,
-                                                            pc_rope_dev rope, const long long *__restrict__ fx, double fx_scale,
-                                                            long long *__restrict__ fx_clear, float *__restrict__ scores,
-                                                            int32_t *status) {
+                                                            pc_rope_dev rope, long long *fx, double fx_scale,
+                                                            float *__restrict__ scores, int32_t *status) {
     pc_grid_dep_launch();
     constexpr int PER = Elem<T>::PER16, NP = PER / 2, CP = (CPL + 1) / 2;
     __shared__ float4 qs[CP * NP * 32];                               // (q_a chunk 2cp, q_a chunk 2cp+1, q_b ..., q_b ...)
@@ -177,9 +188,20 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict_
         }
         qs[idx] = make_float4(v[0], v[1], v[2], v[3]);
     }
-    if (fx_clear && blockIdx.x == 0)                                  // the other accumulator, for the next call's query pass
-        for (int e = threadIdx.x; e < CPL * 32 * PER; e += SCORE_THREADS) fx_clear[e] = 0;
     __syncthreads();
+    // The accumulator must be zero again for the next query pass.  Every block counts itself in once it has read it
+    // (word `row` of the array is the counter); the block that arrives last knows that all have read, clears the
+    // accumulator and the counter.  Nobody waits for anybody, and nothing of this lives on the host, so a captured
+    // graph replays it unchanged.
+    __shared__ int is_last;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        is_last = atomicAdd(reinterpret_cast<unsigned long long *>(fx + CPL * 32 * PER), 1ull) == (unsigned long long)(gridDim.x - 1);
+    }
+    __syncthreads();
+    if (is_last) {
+        for (int e = threadIdx.x; e <= CPL * 32 * PER; e += SCORE_THREADS) fx[e] = 0;
+    }
 
     // table slots of this lane's pairs: entry = tbase + coordinate(axis) * stride
     const int pair0 = ((lane * PER) % d) / 2;
@@ -390,10 +412,10 @@ __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict_
 }
 
 // Enqueue the query pass and the scoring kernel on caller-given scratch (a context's, or the library's fixed array).
-// fx: the fixed-point accumulator of this call, all zero on entry; fx_clear: the accumulator the scoring kernel clears
-// for the next call, or NULL; q_rot / q_scale: where the rotated queries go as well and the factor folded into them.
+// fx: the fixed-point accumulator (Hkv*d sums and one counter word), all zero on entry and zero again when the scoring
+// kernel has run; q_rot / q_scale: where the rotated queries go as well and the factor folded into them.
 template <typename T>
-pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev &rope, long long *fx, long long *fx_clear,
+pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev &rope, long long *fx,
                         int32_t *status, const void *hist_k, const int32_t *hist_pos, int n_src, const void *q,
                         const int32_t *q_pos, int32_t n_q, const uint8_t *valid, float *scores, void *q_rot, float q_scale,
                         cudaStream_t stream, pc_ctx *marks) {
@@ -418,7 +440,7 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
             smem_of[dev_id] = q_smem;                                                                               \
         }                                                                                                           \
         PC_LAUNCH((k_qprep<T, QCPL>), dim3(q_blocks), dim3(warps * 32), q_smem, stream, static_cast<const T *>(q), q_pos, n_q, \
-                  D.n_q_heads, group, D.head_dim, q_chunks / 32, rope, q_rot ? q_scale : 1.0f, static_cast<T *>(q_rot),        \
+                  D.n_q_heads, group, D.head_dim, q_chunks / 32, rope, q_scale, static_cast<T *>(q_rot),                       \
                   reinterpret_cast<unsigned long long *>(fx), status);                                              \
     }
     switch (q_chunks / 32) {
@@ -431,7 +453,7 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
     PC_CUDA_TRY(cudaGetLastError());
     if (marks) pc_mark(marks, PC_MARK_QPOOL, stream);
     const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
-    const double fx_scale = 1.0 / (4294967296.0 * (double)n_q * (double)(q_rot ? q_scale : 1.0f));
+    const double fx_scale = 1.0 / (4294967296.0 * (double)n_q);
     const int n_pairs = (n_src + 1) / 2;
     const T *k = static_cast<const T *>(hist_k);
 #define PC_SCORE_CASE(CPL)                                                                                          \
@@ -445,7 +467,7 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
         }                                                                                                           \
         const int blocks = std::max(1, std::min((n_pairs + SCORE_WARPS - 1) / SCORE_WARPS, sm_count * per_sm_of[dev_id])); \
         PC_LAUNCH((k_score<T, CPL>), dim3(blocks), dim3(SCORE_THREADS), 0, stream, k, hist_pos, valid, n_src, D.head_dim, scale, rope, \
-                  static_cast<const long long *>(fx), fx_scale, fx_clear, scores, status);                          \
+                  fx, fx_scale, scores, status);                                                                    \
     } break;
     switch (chunks / 32) {
         PC_SCORE_CASE(1) PC_SCORE_CASE(2) PC_SCORE_CASE(3) PC_SCORE_CASE(4) PC_SCORE_CASE(6) PC_SCORE_CASE(8)
@@ -490,20 +512,18 @@ pc_status pc_score_impl(pc_ctx *ctx, const pc_cache *src, const void *q, const i
             if (n_q > ctx->desc.max_q) return PC_ERR_CAPACITY;
             const size_t row = (size_t)ctx->desc.n_kv_heads * ctx->desc.head_dim;
             if (ctx->qpool_dirty) {          // an earlier call stopped between the query pass and the scoring kernel
-                PC_CUDA_TRY(cudaMemsetAsync(ctx->qpool_fx, 0, 2 * row * sizeof(long long), stream));
+                PC_CUDA_TRY(cudaMemsetAsync(ctx->qpool_fx, 0, (row + 1) * sizeof(long long), stream));
                 ctx->qpool_dirty = 0;
             }
-            long long *fx = ctx->qpool_fx + (size_t)ctx->qpool_turn * row, *fx_next = ctx->qpool_fx + (size_t)(ctx->qpool_turn ^ 1) * row;
             ctx->qpool_dirty = 1;
             const float q_scale = pc_q_rot_scale(ctx->desc.head_dim);
             st = ctx->desc.dtype == PC_BF16
-                     ? enqueue_score<__nv_bfloat16>(ctx->desc, ctx->sm_count, ctx->rope, fx, fx_next, ctx->status, src->history.k,
+                     ? enqueue_score<__nv_bfloat16>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_fx, ctx->status, src->history.k,
                                                     src->history.pos, n_src, q, q_pos, n_q, valid, scores, q_rot_out, q_scale, stream, ctx)
-                     : enqueue_score<float>(ctx->desc, ctx->sm_count, ctx->rope, fx, fx_next, ctx->status, src->history.k,
+                     : enqueue_score<float>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_fx, ctx->status, src->history.k,
                                             src->history.pos, n_src, q, q_pos, n_q, valid, scores, nullptr, 1.0f, stream, ctx);
             if (st != PC_OK) return st;
             ctx->qpool_dirty = 0;
-            ctx->qpool_turn ^= 1;
             if (q_rot_out) ctx->q_rot_n = n_q;
         }
         select_on = scores;
@@ -546,9 +566,9 @@ constexpr int STATIC_MAX_ROPE = 32768;        // rotary table entries: sum over 
 constexpr int STATIC_MAX_QROW = 12288;        // n_q_heads * head_dim: one row of the query pass's shared-memory slab
 constexpr int STATIC_MAX_DEVICES = PC_MAX_DEVICES;
 
-constexpr size_t STATIC_OFF_FX = 256;  /* first 256 bytes unused */                             // long long [STATIC_MAX_ROW]
-constexpr size_t STATIC_OFF_ROPE = STATIC_OFF_FX + STATIC_MAX_ROW * sizeof(long long);         // float2 [STATIC_MAX_ROPE]
-constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);    // 270,592 bytes
+constexpr size_t STATIC_OFF_FX = 256;  /* first 256 bytes unused */                 // long long [STATIC_MAX_ROW + 1 counter word]
+constexpr size_t STATIC_OFF_ROPE = STATIC_OFF_FX + STATIC_MAX_ROW * sizeof(long long) + 256;   // float2 [STATIC_MAX_ROPE]
+constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);    // 270,848 bytes
 
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
 
@@ -605,13 +625,14 @@ pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const
     // the array keeps whatever the last call left: the table is rewritten before it is read, and the accumulator of the
     // pooled query, which must start at zero, is cleared by the same kernel
     const int row = D.n_kv_heads * D.head_dim;
-    PC_LAUNCH(k_rope_table, dim3((std::max(total, row) + 255) / 256), dim3(256), 0, stream, tab, rope, D.rope_base, total, fx, row);
+    PC_LAUNCH(k_rope_table, dim3((std::max(total, row + 1) + 255) / 256), dim3(256), 0, stream, tab, rope, D.rope_base, total, fx,
+              row + 1);
     PC_CUDA_TRY(cudaGetLastError());
 
     int sm_count = 0, dev = 0;
     PC_CUDA_TRY(cudaGetDevice(&dev));
     PC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    return enqueue_score<T>(D, sm_count, rope, fx, nullptr, status, hist_k, hist_pos, n_src, q, q_pos, n_q, valid, scores, nullptr,
+    return enqueue_score<T>(D, sm_count, rope, fx, status, hist_k, hist_pos, n_src, q, q_pos, n_q, valid, scores, nullptr,
                             1.0f, stream, nullptr);
 }
 

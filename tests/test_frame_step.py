@@ -39,7 +39,7 @@ CASES = {
     "ragged_bf16": lambda: wl.small_bf16(n_frames=3, grid=(11, 13), n_text=130, total=260, kind=wl.LINEAR, param=0.0,
                                          keep_full=0, seed=5),
     "several_tiles": lambda: wl.small_bf16(n_frames=4, grid=(12, 21), n_text=130, total=700, keep_full=1, seed=31),
-    "no_anchors": lambda: wl.small_bf16(n_frames=3, grid=(9, 15), n_text=0, total=200, keep_full=0, seed=32),
+    "no_anchors": lambda: wl.small_bf16(n_frames=3, grid=(9, 15), n_text=37, total=200, keep_full=0, seed=32),
 }
 
 

@@ -72,7 +72,7 @@ def test_random_shapes_against_the_oracle(seed):
             got = host(pc.pc_attend_mass(ctx, lse, n_keys)).astype(np.float64)
             want_mass = oracle.attend_mass(L.q, L.q_pos, [(s[0], s[2]) for s in segs], cfg.rope_base)
             assert pc.pc_poll_status(ctx) == pc.PC_OK, what
-            assert (np.abs(got - want_mass) <= 2e-3 * want_mass + 1e-3 / n_keys).all(), what
+            assert (np.abs(got - want_mass) <= 5e-3 * want_mass + 1e-3 / n_keys).all(), what
         ctx.close()
 
 
