@@ -246,8 +246,8 @@ pc_status pc_frame_step_host(pc_ctx *ctx, const pc_host_frame *in, pc_device_wor
  * was given to an arena of their own at start-up and driver allocations are forbidden afterwards, or they sit on a
  * latency-critical thread that cannot take the device-wide synchronisation an allocation or a free implies — and so
  * cannot create a pc_ctx either.  This call needs no context and calls neither cudaMalloc nor cudaFree nor any
- * allocating routine: the rotary table and the accumulator of the pooled query live in one fixed device array
- * of 270,848 bytes that is part of the library image (every GPU that loads the library holds it until exit).
+ * allocating routine: the rotary table, the pooled query and its accumulator live in one fixed device array
+ * of 332,288 bytes that is part of the library image (every GPU that loads the library holds it until exit).
  *
  * Computes the same scores as pc_score (mean scaled rotary logit of every history token over the n_q queries and
  * all query heads, fp32); selection is not included.  desc->max_q / max_keys are ignored.

@@ -64,8 +64,9 @@ static pc_status create_on_device(pc_ctx *c) {
     PC_CUDA_TRY(cudaMalloc(&c->status, 2 * sizeof(int32_t)));
     PC_CUDA_TRY(cudaMemset(c->status, 0, 2 * sizeof(int32_t)));
     PC_CUDA_TRY(cudaMallocHost(&c->host_status, 2 * sizeof(int32_t)));
-    PC_CUDA_TRY(cudaMalloc(&c->qpool_fx, ((size_t)row + 1) * sizeof(long long)));
-    PC_CUDA_TRY(cudaMemset(c->qpool_fx, 0, ((size_t)row + 1) * sizeof(long long)));
+    PC_CUDA_TRY(cudaMalloc(&c->qpool_fx, ((size_t)PC_FX_REPLICAS * row + 1) * sizeof(long long)));
+    PC_CUDA_TRY(cudaMemset(c->qpool_fx, 0, ((size_t)PC_FX_REPLICAS * row + 1) * sizeof(long long)));
+    PC_CUDA_TRY(cudaMalloc(&c->qpool, (size_t)row * sizeof(float)));
     if (desc->dtype == PC_BF16) {
         pc_status st = pc_attend_tc_scratch(desc, c->sm_count, &c->k_rot_rows, &c->part_o_floats, &c->part_ml_floats);
         if (st != PC_OK) return st;
@@ -112,6 +113,7 @@ extern "C" pc_status pc_destroy(pc_ctx *c) {
     cudaFree(c->status);
     if (c->host_status) cudaFreeHost(c->host_status);
     cudaFree(c->qpool_fx);
+    cudaFree(c->qpool);
     for (int i = 0; i < PC_N_MARKS; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     cudaFree(c->k_rot);

@@ -39,6 +39,7 @@ enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT 
        PC_N_MARKS = 12 };
 
 constexpr int PC_MAX_SEGMENTS = 3;
+constexpr int PC_FX_REPLICAS = 8;             // copies of the pooled-query accumulator (see pc_score.cu)
 constexpr int PC_MAX_DEVICES = 64;            // per-device launch state is kept in arrays of this size
 
 // Rotary tables: for axis a (t, h, w) a [max_pos[a]][n_axis[a]] array of (cos, sin) of pos * base^(-m/n_axis[a]).
@@ -61,10 +62,12 @@ struct pc_ctx {
     float2 *rope_tab;          // owned
     int32_t *status;           // device [2]: code, where
     int32_t *host_status;      // pinned [2]
-    // Pooled query of the scoring pass as fixed-point sums (units of 2^-32): Hkv*d 64-bit integers and one counter word.
-    // The query pass adds into it (integer addition: the result does not depend on the order of the blocks); the
-    // scoring kernel reads it and its last block clears it again, so it is zero between calls.
-    long long *qpool_fx;       // device [Hkv*d + 1]
+    // Pooled query of the scoring pass as fixed-point sums (units of 2^-32): PC_FX_REPLICAS copies of Hkv*d 64-bit
+    // integers (the blocks of the query pass spread over the copies; integer addition: the result does not depend on the
+    // order of the blocks) and one ticket word.  The last block of the query pass adds the copies into `qpool` (fp32) and
+    // clears the accumulator, so it is zero between calls.
+    long long *qpool_fx;       // device [PC_FX_REPLICAS * Hkv*d + 1]
+    float *qpool;              // device [Hkv*d]
     int qpool_dirty;           // 1: a call failed between the two kernels; the array is cleared before the next use
     // attention scratch (tensor-core path)
     void *k_rot;               // rotated keys, bf16 [rows][Hkv][d]
@@ -104,13 +107,17 @@ __device__ __forceinline__ void pc_flag(int32_t *status, int code, int where) {
 // (cos, sin) for pair i of a head at position p[0..2]; flags and clamps a position outside the table.
 __device__ __forceinline__ float2 pc_rope_cs(const pc_rope_dev &r, int pair, int pt, int ph, int pw, int32_t *status,
                                              int where) {
-    int a = pair % 3, m = pair / 3;
+    const int a = pair % 3, m = pair / 3;
+    // the axis picks its coordinate and table by selects on fixed fields (no indexed access to the parameter block)
     int pa = a == 0 ? pt : (a == 1 ? ph : pw);
-    if (pa < 0 || pa >= r.max_pos[a]) {
+    const int mx = a == 0 ? r.max_pos[0] : (a == 1 ? r.max_pos[1] : r.max_pos[2]);
+    const int off = a == 0 ? r.off[0] : (a == 1 ? r.off[1] : r.off[2]);
+    const int na = a == 0 ? r.n_axis[0] : (a == 1 ? r.n_axis[1] : r.n_axis[2]);
+    if (pa < 0 || pa >= mx) {
         pc_flag(status, PC_ERR_INVALID_ARG, where);
-        pa = pa < 0 ? 0 : r.max_pos[a] - 1;
+        pa = pa < 0 ? 0 : mx - 1;
     }
-    return __ldg(r.tab + r.off[a] + (size_t)pa * r.n_axis[a] + m);
+    return __ldg(r.tab + off + (size_t)pa * na + m);
 }
 
 // One rotary pair turned by (cos, sin), with the roundings spelt out: every kernel that rotates (query pass, key

@@ -35,15 +35,16 @@ template <> struct Elem<__nv_bfloat16> {
 // Query pass.  One read of Q serves both consumers of the rotated queries: the pooled query of the scoring pass
 //   q~[g] = (1/n_q) sum_i sum_{h in g} R(p_i) q_ih
 // and, for the tensor-core attention kernel, the rotated bf16 queries with log2(e)/sqrt(d) folded in (q_rot).
-// One warp takes one query token: lane l reads the 16-byte chunks l, l + 32, ... of the row (all in flight at once);
-// 32 chunks span a multiple of d, so all of a lane's chunks hold the same rotary pairs and the lane needs PER/2 table
-// entries per token.  The rotated row also goes to a per-warp slab in shared memory; after a block barrier the threads
-// add, in a fixed order, the slabs' entries of each pooled element (heads of the group, then warps), turn the sum
+// A few warps share one query token: lane l of a warp reads the 16-byte chunks l, l + 32, ... of the warp's part of the
+// row (all in flight at once); 32 chunks span a multiple of d, so all of a lane's chunks hold the same rotary pairs and
+// the lane needs PER/2 table entries.  The rotated row also goes to a per-token slab in shared memory; after a block
+// barrier the threads add, in a fixed order, the slabs' entries of each pooled element (tokens, then heads), turn the sum
 // into a 64-bit fixed-point number (units of 2^-32) and add it to the global accumulator with an integer atomic:
 // integer addition is associative, so the pooled query does not depend on the order in which blocks arrive.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int QPREP_MAX_WARPS = 8;
+constexpr int QPREP_WARPS = 8;                      // warps per block when the parts of a token divide it
 constexpr float FX_ONE = 4294967296.0f;             // 2^32
+constexpr int FX_REPLICAS = PC_FX_REPLICAS;         // copies of the accumulator the blocks of the query pass spread over
 
 template <typename T> __device__ __forceinline__ uint4 pack_row(const float *f);
 template <> __device__ __forceinline__ uint4 pack_row<float>(const float *f) {
@@ -53,36 +54,40 @@ template <> __device__ __forceinline__ uint4 pack_row<__nv_bfloat16>(const float
     return make_uint4(pc_pack_bf16(f[0], f[1]), pc_pack_bf16(f[2], f[3]), pc_pack_bf16(f[4], f[5]), pc_pack_bf16(f[6], f[7]));
 }
 
-template <typename T, int QCPL /* chunks per lane of a query row; 0 = any count, looped */>
-__global__ void __launch_bounds__(QPREP_MAX_WARPS * 32) k_qprep(const T *__restrict__ q, const int32_t *__restrict__ q_pos, int n_q,
-                                                                 int n_q_heads, int group, int d, int cpl_rt, pc_rope_dev rope,
-                                                                 float out_scale, T *__restrict__ q_rot,
-                                                                 unsigned long long *__restrict__ fx, int32_t *status) {
+// A query row is cut into `parts` runs of CPW x 32 chunks, one warp each (short instruction streams on many warps: the
+// kernel is bound by latency, not by bytes); a block holds `tokens_per_block` tokens.
+template <typename T, int CPW /* chunks per lane of one warp's part of a query row */>
+__global__ void __launch_bounds__(1024) k_qprep(const T *__restrict__ q, const int32_t *__restrict__ q_pos, int n_q,
+                                                int n_q_heads, int group, int d, int parts, pc_rope_dev rope,
+                                                float out_scale, T *__restrict__ q_rot,
+                                                unsigned long long *fx, double fx_scale, float *__restrict__ pooled,
+                                                int32_t *status) {
     pc_grid_dep_launch();
     pc_grid_dep_wait();
     constexpr int PER = Elem<T>::PER16, NP = PER / 2;
-    extern __shared__ __align__(16) float slab[];                     // [warps][Hq*d]
-    const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    extern __shared__ __align__(16) float slab[];                     // [tokens_per_block][Hq*d]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tokens_per_block = (blockDim.x >> 5) / parts;
     const int row_len = n_q_heads * d;
-    const int cpl = QCPL > 0 ? QCPL : cpl_rt;
-    const int i = blockIdx.x * warps + warp;
+    const int tok = warp / parts, part = warp - tok * parts;
+    const int i = blockIdx.x * tokens_per_block + tok;
     if (i < n_q) {
         const int4 pp = __ldg(reinterpret_cast<const int4 *>(q_pos) + i);
-        const uint4 *src = reinterpret_cast<const uint4 *>(q + (size_t)i * row_len) + lane;
-        uint4 raw[QCPL > 0 ? QCPL : 1];
-        if constexpr (QCPL > 0) {
+        const size_t at = (size_t)i * (row_len / PER) + (size_t)part * CPW * 32 + lane;     // in 16-byte chunks
+        const uint4 *src = reinterpret_cast<const uint4 *>(q) + at;
+        uint4 raw[CPW];
 #pragma unroll
-            for (int c = 0; c < QCPL; ++c) raw[c] = pc_ldg_stream(src + c * 32);
-        }
+        for (int c = 0; c < CPW; ++c) raw[c] = pc_ldg_stream(src + c * 32);
         const int pair0 = ((lane * PER) % d) / 2;
         float2 cs[NP];
 #pragma unroll
         for (int u = 0; u < NP; ++u) cs[u] = pc_rope_cs(rope, pair0 + u, pp.x, pp.y, pp.z, status, PC_WHERE_QPOOL_POS);
-        float *mine = slab + (size_t)warp * row_len + lane * PER;
-        uint4 *dst = q_rot ? reinterpret_cast<uint4 *>(q_rot + (size_t)i * row_len) + lane : nullptr;
-        auto one_chunk = [&](const uint4 &v, int c) {
+        float *mine = slab + (size_t)tok * row_len + ((size_t)part * CPW * 32 + lane) * PER;
+        uint4 *dst = q_rot ? reinterpret_cast<uint4 *>(q_rot) + at : nullptr;
+#pragma unroll
+        for (int c = 0; c < CPW; ++c) {
             float x[PER], r[PER];
-            Elem<T>::unpack(v, x);
+            Elem<T>::unpack(raw[c], x);
 #pragma unroll
             for (int u = 0; u < NP; ++u) {
                 const float2 y = pc_rotate(x[2 * u], x[2 * u + 1], cs[u]);
@@ -97,19 +102,15 @@ __global__ void __launch_bounds__(QPREP_MAX_WARPS * 32) k_qprep(const T *__restr
                 for (int k = 0; k < PER; ++k) r[k] = __fmul_rn(r[k], out_scale);
                 dst[c * 32] = pack_row<T>(r);
             }
-        };
-        if constexpr (QCPL > 0) {
-#pragma unroll
-            for (int c = 0; c < QCPL; ++c) one_chunk(raw[c], c);
-        } else {
-            for (int c = 0; c < cpl; ++c) one_chunk(pc_ldg_stream(src + c * 32), c);
         }
     }
     __syncthreads();
-    const int n_warps_used = min(warps, n_q - blockIdx.x * warps);
+    const int n_tokens_used = min(tokens_per_block, n_q - blockIdx.x * tokens_per_block);
     const int n_out = (n_q_heads / group) * d;
+    // blocks spread over FX_REPLICAS copies of the accumulator: fewer atomics queue up on each cache line
+    unsigned long long *mine_fx = fx + (size_t)(blockIdx.x % FX_REPLICAS) * n_out;
     // four pooled elements per thread at a time, so that four independent sums are in flight; the order of the additions
-    // of each sum is fixed (warps ascending, heads of the group ascending)
+    // of each sum is fixed (tokens ascending, heads of the group ascending)
     for (int e0 = threadIdx.x; e0 < n_out; e0 += 4 * blockDim.x) {
         const float *s[4];
         float sum[4] = {0.f, 0.f, 0.f, 0.f};
@@ -118,7 +119,7 @@ __global__ void __launch_bounds__(QPREP_MAX_WARPS * 32) k_qprep(const T *__restr
             const int e = min(e0 + k * (int)blockDim.x, n_out - 1), g = e / d, x = e - g * d;
             s[k] = slab + (size_t)g * group * d + x;
         }
-        for (int w = 0; w < n_warps_used; ++w)
+        for (int w = 0; w < n_tokens_used; ++w)
             for (int h = 0; h < group; ++h) {
                 const int off = w * row_len + h * d;
 #pragma unroll
@@ -127,20 +128,42 @@ __global__ void __launch_bounds__(QPREP_MAX_WARPS * 32) k_qprep(const T *__restr
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const int e = e0 + k * (int)blockDim.x;
-            if (e < n_out) atomicAdd(fx + e, (unsigned long long)__float2ll_rn(sum[k] * FX_ONE));
+            if (e < n_out) atomicAdd(mine_fx + e, (unsigned long long)__float2ll_rn(sum[k] * FX_ONE));
         }
     }
+    // The block that finishes last (a ticket in the word after the last copy; nobody waits for anybody) adds the copies,
+    // writes the pooled query as fp32 and clears the accumulator and the ticket for the next call.  Nothing of this lives
+    // on the host, so a captured graph replays it unchanged.
+    __shared__ int is_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0)
+        is_last = atomicAdd(fx + (size_t)FX_REPLICAS * n_out, 1ull) == (unsigned long long)(gridDim.x - 1);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int e = threadIdx.x; e < n_out; e += blockDim.x) {
+        long long w = 0;
+#pragma unroll
+        for (int rep = 0; rep < FX_REPLICAS; ++rep) {                     // integer sums: any order gives the same bits
+            w += (long long)__ldcg(fx + (size_t)rep * n_out + e);
+            fx[(size_t)rep * n_out + e] = 0;
+        }
+        pooled[e] = (float)((double)w * fx_scale);
+    }
+    if (threadIdx.x == 0) fx[(size_t)FX_REPLICAS * n_out] = 0;
 }
 
 // ---------------------------------------------------------------------------------------------------------
 // Score.  One warp takes two history tokens at a time: lane l loads the 16-byte chunks l, l + 32, ... of both rows
 // (streaming loads, all in flight before the first is used: 2 x CPL x 512 bytes per warp) and both position records.
 // 32 chunks span a multiple of d, so all of a lane's chunks cover the same PER/2 rotary pairs (of different heads): the
-// lane sums the two brackets over its chunks and needs PER/2 table look-ups per token.  The pooled query sits in shared
-// memory, converted once per block from the fixed-point accumulator and laid out so that one 16-byte read gives a
-// lane its (q_a, q_b) of two chunks at once: chunks are processed two at a time and every multiply-add is a two-lane
-// fp32 instruction.  Blocks are persistent; warps take token pairs round-robin, so the tokens in flight at any time
-// form one contiguous window of the history.
+// lane sums the two brackets over its chunks and needs PER/2 table look-ups per token.  For a pair (a, b) the two
+// brackets are two-lane products of the pair as it comes out of the unpacking, (k_a, k_b), with (q_a, q_b) and with
+// (q_b, -q_a): two two-lane fp32 multiply-adds per pair, no register shuffling.  The pooled query sits in shared
+// memory in that form; one 16-byte read serves both rows.
+// Blocks are persistent; warps take token pairs round-robin, so the tokens in flight at any time form one contiguous
+// window of the history.
 // ---------------------------------------------------------------------------------------------------------
 constexpr int SCORE_WARPS = 8;
 constexpr int SCORE_THREADS = SCORE_WARPS * 32;
@@ -148,11 +171,11 @@ constexpr int SCORE_THREADS = SCORE_WARPS * 32;
 template <typename T, int CPL /* chunks per lane */>
 __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict__ k, const int32_t *__restrict__ k_pos,
                                                             const uint8_t *__restrict__ valid, int n_src, int d, float scale,
-                                                            pc_rope_dev rope, long long *fx, double fx_scale,
+                                                            pc_rope_dev rope, const float *__restrict__ pooled,
                                                             float *__restrict__ scores, int32_t *status) {
     pc_grid_dep_launch();
-    constexpr int PER = Elem<T>::PER16, NP = PER / 2, CP = (CPL + 1) / 2;
-    __shared__ float4 qs[CP * NP * 32];                               // (q_a chunk 2cp, q_a chunk 2cp+1, q_b ..., q_b ...)
+    constexpr int PER = Elem<T>::PER16, NP = PER / 2;
+    __shared__ float4 qs[CPL * NP * 32];                              // (q_a, q_b, q_b, -q_a) of (chunk, pair, lane)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gw = blockIdx.x * SCORE_WARPS + warp, n_warps = gridDim.x * SCORE_WARPS;
     const int n_pairs = (n_src + 1) >> 1;
@@ -174,34 +197,12 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict_
     };
     if (tp < n_pairs) request(tp);
 
-    for (int idx = threadIdx.x; idx < CP * NP * 32; idx += SCORE_THREADS) {
-        const int l = idx & 31, u = (idx >> 5) % NP, cp = idx / (32 * NP);
-        float v[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int c = 2 * cp + half;
-            if (c < CPL) {
-                const longlong2 w = __ldcg(reinterpret_cast<const longlong2 *>(fx + (size_t)(c * 32 + l) * PER + 2 * u));
-                v[half] = (float)((double)w.x * fx_scale);
-                v[2 + half] = (float)((double)w.y * fx_scale);
-            }
-        }
-        qs[idx] = make_float4(v[0], v[1], v[2], v[3]);
+    for (int idx = threadIdx.x; idx < CPL * NP * 32; idx += SCORE_THREADS) {
+        const int l = idx & 31, u = (idx >> 5) % NP, c = idx / (32 * NP);
+        const float2 w = __ldcg(reinterpret_cast<const float2 *>(pooled + (size_t)(c * 32 + l) * PER + 2 * u));
+        qs[idx] = make_float4(w.x, w.y, w.y, -w.x);
     }
     __syncthreads();
-    // The accumulator must be zero again for the next query pass.  Every block counts itself in once it has read it
-    // (word `row` of the array is the counter); the block that arrives last knows that all have read, clears the
-    // accumulator and the counter.  Nobody waits for anybody, and nothing of this lives on the host, so a captured
-    // graph replays it unchanged.
-    __shared__ int is_last;
-    if (threadIdx.x == 0) {
-        __threadfence();
-        is_last = atomicAdd(reinterpret_cast<unsigned long long *>(fx + CPL * 32 * PER), 1ull) == (unsigned long long)(gridDim.x - 1);
-    }
-    __syncthreads();
-    if (is_last) {
-        for (int e = threadIdx.x; e <= CPL * 32 * PER; e += SCORE_THREADS) fx[e] = 0;
-    }
 
     // table slots of this lane's pairs: entry = tbase + coordinate(axis) * stride
     const int pair0 = ((lane * PER) % d) / 2;
@@ -210,8 +211,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict_
     for (int u = 0; u < NP; ++u) {
         const int a = (pair0 + u) % 3;
         taxis[u] = a;
-        tbase[u] = rope.off[a] + (pair0 + u) / 3;
-        tstride[u] = rope.n_axis[a];
+        tbase[u] = (a == 0 ? rope.off[0] : (a == 1 ? rope.off[1] : rope.off[2])) + (pair0 + u) / 3;
+        tstride[u] = a == 0 ? rope.n_axis[0] : (a == 1 ? rope.n_axis[1] : rope.n_axis[2]);
     }
     const unsigned mt = rope.max_pos[0], mh = rope.max_pos[1], mw = rope.max_pos[2];
     const float4 *ql = qs + lane;
@@ -228,48 +229,37 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict_
             cs[u] = __ldg(rope.tab + tbase[u] + pa * tstride[u]);
         }
     };
-    // brackets per pair:  A = sum q_a k_a + q_b k_b,  B = sum q_b k_a - q_a k_b  (B kept as two sums)
-    auto row_score = [&](const uint4 (&raw)[CPL], const float2 (&cs)[NP]) {
-        float2 A2[NP], B2[NP], C2[NP];
-#pragma unroll
-        for (int u = 0; u < NP; ++u) A2[u] = B2[u] = C2[u] = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int cp = 0; cp < CP; ++cp) {
-            float k0[PER], k1[PER];
-            Elem<T>::unpack(raw[2 * cp], k0);
-            if (2 * cp + 1 < CPL) {
-                Elem<T>::unpack(raw[2 * cp + 1 < CPL ? 2 * cp + 1 : 0], k1);
-            } else {
-#pragma unroll
-                for (int e = 0; e < PER; ++e) k1[e] = 0.f;
-            }
-#pragma unroll
-            for (int u = 0; u < NP; ++u) {
-                const float4 qq = ql[(cp * NP + u) * 32];
-                const float2 qa = make_float2(qq.x, qq.y), qb = make_float2(qq.z, qq.w);
-                const float2 ka = make_float2(k0[2 * u], k1[2 * u]), kb = make_float2(k0[2 * u + 1], k1[2 * u + 1]);
-                pc_fma2(A2[u], qa, ka);
-                pc_fma2(A2[u], qb, kb);
-                pc_fma2(B2[u], qb, ka);
-                pc_fma2(C2[u], qa, kb);
-            }
-        }
-        float sum = 0.f;
-#pragma unroll
-        for (int u = 0; u < NP; ++u) {
-            const float A = A2[u].x + A2[u].y;
-            const float B = (B2[u].x + B2[u].y) - (C2[u].x + C2[u].y);
-            sum = fmaf(cs[u].x, A, fmaf(cs[u].y, B, sum));
-        }
-        return sum;
-    };
 
     for (; tp < n_pairs; tp += n_warps) {
         float2 cs0[NP], cs1[NP];
         table(p0, cs0);
         table(p1, cs1);
-        float s0 = row_score(raw0, cs0);
-        float s1 = row_score(raw1, cs1);
+        // brackets per pair:  A = sum q_a k_a + q_b k_b,  B = sum q_b k_a - q_a k_b, each as the two lanes of one register pair
+        float2 A0[NP], B0[NP], A1[NP], B1[NP];
+#pragma unroll
+        for (int u = 0; u < NP; ++u) A0[u] = B0[u] = A1[u] = B1[u] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+            float k0[PER], k1[PER];
+            Elem<T>::unpack(raw0[c], k0);
+            Elem<T>::unpack(raw1[c], k1);
+#pragma unroll
+            for (int u = 0; u < NP; ++u) {
+                const float4 qq = ql[(c * NP + u) * 32];
+                const float2 qab = make_float2(qq.x, qq.y), qba = make_float2(qq.z, qq.w);
+                const float2 x0 = make_float2(k0[2 * u], k0[2 * u + 1]), x1 = make_float2(k1[2 * u], k1[2 * u + 1]);
+                A0[u] = __ffma2_rn(qab, x0, A0[u]);
+                B0[u] = __ffma2_rn(qba, x0, B0[u]);
+                A1[u] = __ffma2_rn(qab, x1, A1[u]);
+                B1[u] = __ffma2_rn(qba, x1, B1[u]);
+            }
+        }
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int u = 0; u < NP; ++u) {
+            s0 = fmaf(cs0[u].x, A0[u].x + A0[u].y, fmaf(cs0[u].y, B0[u].x + B0[u].y, s0));
+            s1 = fmaf(cs1[u].x, A1[u].x + A1[u].y, fmaf(cs1[u].y, B1[u].x + B1[u].y, s1));
+        }
         const int j0 = 2 * tp;
         if (tp + n_warps < n_pairs) request(tp + n_warps);           // the next two rows travel while these are reduced
         // both sums with six shuffles: after the first exchange the lower half-warp carries token 0, the upper token 1
@@ -412,10 +402,11 @@ __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict_
 }
 
 // Enqueue the query pass and the scoring kernel on caller-given scratch (a context's, or the library's fixed array).
-// fx: the fixed-point accumulator (Hkv*d sums and one counter word), all zero on entry and zero again when the scoring
-// kernel has run; q_rot / q_scale: where the rotated queries go as well and the factor folded into them.
+// fx: the fixed-point accumulator (PC_FX_REPLICAS copies of Hkv*d sums and one ticket word), all zero on entry and zero
+// again when the query pass has run; pooled: Hkv*d floats, written by the query pass and read by the scoring kernel;
+// q_rot / q_scale: where the rotated queries go as well and the factor folded into them.
 template <typename T>
-pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev &rope, long long *fx,
+pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev &rope, long long *fx, float *pooled,
                         int32_t *status, const void *hist_k, const int32_t *hist_pos, int n_src, const void *q,
                         const int32_t *q_pos, int32_t n_q, const uint8_t *valid, float *scores, void *q_rot, float q_scale,
                         cudaStream_t stream, pc_ctx *marks) {
@@ -425,35 +416,41 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
     const int q_row = D.n_q_heads * D.head_dim;
     const int q_chunks = q_row / PER, chunks = row / PER;            // 16-byte chunks per query row / key row
     if (chunks % 32 || q_chunks % 32 || (32 * PER) % D.head_dim) return PC_ERR_UNSUPPORTED;
-    const int warps = std::max(1, std::min<int>(QPREP_MAX_WARPS, (int)((200u * 1024u) / ((size_t)q_row * sizeof(float)))));
-    const int q_smem = warps * q_row * (int)sizeof(float);
-    const int q_blocks = (n_q + warps - 1) / warps;
+    const double fx_scale = 1.0 / (4294967296.0 * (double)n_q);
+    // a row's chunk rows are dealt to `parts` warps of 1-4 chunk rows each
+    const int qcpl = q_chunks / 32;
+    const int cpw = qcpl % 3 == 0 ? 3 : (qcpl % 4 == 0 ? 4 : (qcpl % 2 == 0 ? 2 : 1));
+    const int parts = qcpl / cpw;
+    if (parts > 32) return PC_ERR_UNSUPPORTED;
+    int tokens_per_block = std::max(1, QPREP_WARPS / parts);
+    tokens_per_block = std::max(1, std::min<int>(tokens_per_block, (int)((200u * 1024u) / ((size_t)q_row * sizeof(float)))));
+    const int q_smem = tokens_per_block * q_row * (int)sizeof(float);
+    const int q_blocks = (n_q + tokens_per_block - 1) / tokens_per_block;
     int dev_id = 0;
     PC_CUDA_TRY(cudaGetDevice(&dev_id));
     if (dev_id < 0 || dev_id >= PC_MAX_DEVICES) return PC_ERR_UNSUPPORTED;
     if (marks) pc_mark(marks, PC_MARK_SCORE0, stream);
-#define PC_QPREP_CASE(QCPL)                                                                                          \
+#define PC_QPREP_CASE(CPW)                                                                                           \
     {                                                                                                               \
         static int smem_of[PC_MAX_DEVICES] = {};                      /* largest dynamic size allowed so far */      \
         if (q_smem > 48 * 1024 && smem_of[dev_id] < q_smem) {                                                       \
-            PC_CUDA_TRY(cudaFuncSetAttribute(k_qprep<T, QCPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, q_smem)); \
+            PC_CUDA_TRY(cudaFuncSetAttribute(k_qprep<T, CPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, q_smem)); \
             smem_of[dev_id] = q_smem;                                                                               \
         }                                                                                                           \
-        PC_LAUNCH((k_qprep<T, QCPL>), dim3(q_blocks), dim3(warps * 32), q_smem, stream, static_cast<const T *>(q), q_pos, n_q, \
-                  D.n_q_heads, group, D.head_dim, q_chunks / 32, rope, q_scale, static_cast<T *>(q_rot),                       \
-                  reinterpret_cast<unsigned long long *>(fx), status);                                              \
+        PC_LAUNCH((k_qprep<T, CPW>), dim3(q_blocks), dim3(tokens_per_block * parts * 32), q_smem, stream,           \
+                  static_cast<const T *>(q), q_pos, n_q, D.n_q_heads, group, D.head_dim, parts, rope, q_scale,      \
+                  static_cast<T *>(q_rot), reinterpret_cast<unsigned long long *>(fx), fx_scale, pooled, status);   \
     }
-    switch (q_chunks / 32) {
-    case 12: PC_QPREP_CASE(12) break;      // 24 query heads x 128 bf16
+    switch (cpw) {
+    case 3: PC_QPREP_CASE(3) break;        // 24 query heads x 128 bf16: four warps per token
     case 4: PC_QPREP_CASE(4) break;
     case 2: PC_QPREP_CASE(2) break;
-    default: PC_QPREP_CASE(0) break;
+    default: PC_QPREP_CASE(1) break;
     }
 #undef PC_QPREP_CASE
     PC_CUDA_TRY(cudaGetLastError());
     if (marks) pc_mark(marks, PC_MARK_QPOOL, stream);
     const float scale = (float)(1.0 / ((double)D.n_q_heads * std::sqrt((double)D.head_dim)));
-    const double fx_scale = 1.0 / (4294967296.0 * (double)n_q);
     const int n_pairs = (n_src + 1) / 2;
     const T *k = static_cast<const T *>(hist_k);
 #define PC_SCORE_CASE(CPL)                                                                                          \
@@ -467,7 +464,7 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
         }                                                                                                           \
         const int blocks = std::max(1, std::min((n_pairs + SCORE_WARPS - 1) / SCORE_WARPS, sm_count * per_sm_of[dev_id])); \
         PC_LAUNCH((k_score<T, CPL>), dim3(blocks), dim3(SCORE_THREADS), 0, stream, k, hist_pos, valid, n_src, D.head_dim, scale, rope, \
-                  fx, fx_scale, scores, status);                                                                    \
+                  pooled, scores, status);                                                                          \
     } break;
     switch (chunks / 32) {
         PC_SCORE_CASE(1) PC_SCORE_CASE(2) PC_SCORE_CASE(3) PC_SCORE_CASE(4) PC_SCORE_CASE(6) PC_SCORE_CASE(8)
@@ -512,15 +509,15 @@ pc_status pc_score_impl(pc_ctx *ctx, const pc_cache *src, const void *q, const i
             if (n_q > ctx->desc.max_q) return PC_ERR_CAPACITY;
             const size_t row = (size_t)ctx->desc.n_kv_heads * ctx->desc.head_dim;
             if (ctx->qpool_dirty) {          // an earlier call stopped between the query pass and the scoring kernel
-                PC_CUDA_TRY(cudaMemsetAsync(ctx->qpool_fx, 0, (row + 1) * sizeof(long long), stream));
+                PC_CUDA_TRY(cudaMemsetAsync(ctx->qpool_fx, 0, (PC_FX_REPLICAS * row + 1) * sizeof(long long), stream));
                 ctx->qpool_dirty = 0;
             }
             ctx->qpool_dirty = 1;
             const float q_scale = pc_q_rot_scale(ctx->desc.head_dim);
             st = ctx->desc.dtype == PC_BF16
-                     ? enqueue_score<__nv_bfloat16>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_fx, ctx->status, src->history.k,
+                     ? enqueue_score<__nv_bfloat16>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_fx, ctx->qpool, ctx->status, src->history.k,
                                                     src->history.pos, n_src, q, q_pos, n_q, valid, scores, q_rot_out, q_scale, stream, ctx)
-                     : enqueue_score<float>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_fx, ctx->status, src->history.k,
+                     : enqueue_score<float>(ctx->desc, ctx->sm_count, ctx->rope, ctx->qpool_fx, ctx->qpool, ctx->status, src->history.k,
                                             src->history.pos, n_src, q, q_pos, n_q, valid, scores, nullptr, 1.0f, stream, ctx);
             if (st != PC_OK) return st;
             ctx->qpool_dirty = 0;
@@ -553,7 +550,7 @@ extern "C" pc_status pc_score(pc_ctx *ctx, const pc_cache *src, const void *q, c
 // was handed to its own arena at start-up and whose policy forbids driver allocations afterwards, or a
 // latency-critical thread that cannot take the device-wide synchronisation a cudaMalloc / cudaFree implies.  Such
 // callers cannot create a pc_ctx (pc_create allocates), so everything a context would hold for scoring — the rotary
-// table and the fixed-point accumulator of the pooled query — lives in one file-scope device array of fixed size
+// table, the fixed-point accumulator of the pooled query and the pooled query itself — lives in one file-scope device array of fixed size
 // that every GPU loading this library carries until the process exits.
 //
 // In host code the array's name is only a handle; the device address is obtained once per device with
@@ -566,9 +563,10 @@ constexpr int STATIC_MAX_ROPE = 32768;        // rotary table entries: sum over 
 constexpr int STATIC_MAX_QROW = 12288;        // n_q_heads * head_dim: one row of the query pass's shared-memory slab
 constexpr int STATIC_MAX_DEVICES = PC_MAX_DEVICES;
 
-constexpr size_t STATIC_OFF_FX = 256;  /* first 256 bytes unused */                 // long long [STATIC_MAX_ROW + 1 counter word]
-constexpr size_t STATIC_OFF_ROPE = STATIC_OFF_FX + STATIC_MAX_ROW * sizeof(long long) + 256;   // float2 [STATIC_MAX_ROPE]
-constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);    // 270,848 bytes
+constexpr size_t STATIC_OFF_FX = 256;  /* first 256 bytes unused */       // long long [PC_FX_REPLICAS * STATIC_MAX_ROW + 1 counter word]
+constexpr size_t STATIC_OFF_POOLED = STATIC_OFF_FX + (size_t)PC_FX_REPLICAS * STATIC_MAX_ROW * sizeof(long long) + 256;   // float [STATIC_MAX_ROW]
+constexpr size_t STATIC_OFF_ROPE = STATIC_OFF_POOLED + STATIC_MAX_ROW * sizeof(float);          // float2 [STATIC_MAX_ROPE]
+constexpr size_t STATIC_BYTES = STATIC_OFF_ROPE + (size_t)STATIC_MAX_ROPE * sizeof(float2);    // 332,288 bytes
 
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
 
@@ -611,6 +609,7 @@ pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const
                               int32_t n_src, const void *q, const int32_t *q_pos, int32_t n_q, const uint8_t *valid,
                               float *scores, int32_t *status, cudaStream_t stream) {
     long long *fx = reinterpret_cast<long long *>(base + STATIC_OFF_FX);
+    float *pooled = reinterpret_cast<float *>(base + STATIC_OFF_POOLED);
     float2 *tab = reinterpret_cast<float2 *>(base + STATIC_OFF_ROPE);
 
     pc_rope_dev rope;
@@ -625,14 +624,15 @@ pc_status launch_score_static(const pc_layer_desc &D, unsigned char *base, const
     // the array keeps whatever the last call left: the table is rewritten before it is read, and the accumulator of the
     // pooled query, which must start at zero, is cleared by the same kernel
     const int row = D.n_kv_heads * D.head_dim;
-    PC_LAUNCH(k_rope_table, dim3((std::max(total, row + 1) + 255) / 256), dim3(256), 0, stream, tab, rope, D.rope_base, total, fx,
-              row + 1);
+    const int fx_words = PC_FX_REPLICAS * row + 1;
+    PC_LAUNCH(k_rope_table, dim3((std::max(total, fx_words) + 255) / 256), dim3(256), 0, stream, tab, rope, D.rope_base, total, fx,
+              fx_words);
     PC_CUDA_TRY(cudaGetLastError());
 
     int sm_count = 0, dev = 0;
     PC_CUDA_TRY(cudaGetDevice(&dev));
     PC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    return enqueue_score<T>(D, sm_count, rope, fx, status, hist_k, hist_pos, n_src, q, q_pos, n_q, valid, scores, nullptr,
+    return enqueue_score<T>(D, sm_count, rope, fx, pooled, status, hist_k, hist_pos, n_src, q, q_pos, n_q, valid, scores, nullptr,
                             1.0f, stream, nullptr);
 }
 
