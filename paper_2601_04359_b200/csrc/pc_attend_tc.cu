@@ -3,7 +3,8 @@
 // Launch sequence of pc_launch_attend_tc:
 //   k_rope_rows   rotates K of every segment (3D rotary tables, from the stored positions) into a bf16 scratch whose
 //                 segments start on 128-row boundaries, and rotates Q with log2(e)/sqrt(d) folded in.
-//   k_attend_tc   one CTA = two 128-row query tiles that share a KV head (grouped-query packing) x one KV range.
+//   k_attend_tc   persistent CTAs (one per SM) share the line of (item, key tile) steps evenly; an item = two 128-row
+//                 query tiles that share a KV head (grouped-query packing).
 //                 Warp 0 lane 0 drives TMA (K and V tiles, 128B swizzle, two stages each), warp 1 lane 0 issues
 //                 tcgen05.mma: S_t = Q_t K^T (both operands K-major in shared memory) into TMEM, and
 //                 O_t += P_t V with P_t read from TMEM and V MN-major in shared memory.  Warps 4-7 / 8-11 are the
@@ -40,11 +41,15 @@ constexpr int SM_ML = SM_BAR + 256;                       // (max, sum) of both 
 constexpr int SM_TOTAL = SM_ML + 2 * TILE * 8;
 constexpr int SM_ALLOC = SM_TOTAL + 1024;                 // slack for manual alignment
 
-enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PHALF = 11 /* [tile][half] */,
+enum { BAR_Q = 0, BAR_QFREE = 1, BAR_KEMPTY = 2, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PHALF = 11 /* [tile][half] */,
        BAR_DONE = 15, N_BARS = 16 };
 
 struct TcParams {
     int n_q, n_q_heads, group, n_tb, tiles_per_g, pairs_per_g, n_splits, n_kv_tiles;
+    int n_items;      // (KV head, pair of query tiles)
+    int persistent;   // 1: n_cta CTAs share the line of (item, key tile) steps evenly; 0: CTA (item, s) takes one of n_splits ranges
+    int n_cta;
+    int part_stride;  // partial slots reserved per item (most parts any item has)
     int n_seg;
     int cluster;      // 1: the KV ranges of one item form a thread-block cluster and merge through shared memory
     uint32_t wait_us; // limit of every bounded wait in microseconds (0 = about one second)
@@ -143,6 +148,49 @@ __device__ __forceinline__ void kv_tile_info(const TcParams &P, int jt, int &seg
     n_valid = min(TILE, P.seg_n[seg] - local * TILE);
 }
 
+// ---- work decomposition.  The (item, key tile) pairs of a call form one line of n_items * n_kv_tiles steps, item-major.
+// A CTA takes a contiguous run of it.  Persistent form: n_cta CTAs (one per SM) share the line evenly, so a CTA's run
+// usually crosses from one item into the next; set-up (barriers, tensor memory) is paid once per CTA, the next item's
+// queries and first keys arrive under the current item's last steps, and all SMs finish together.  Split form: CTA
+// (item, s) takes the s-th of n_splits equal ranges of one item (used when the caller fixes the number of key ranges, and
+// by the cluster merge).  The part of an item one CTA works on is a "unit"; an item's units are numbered by "part".
+__device__ __forceinline__ void cta_run(const TcParams &P, int c, long long &g0, long long &g1) {
+    if (P.persistent) {
+        const long long T = (long long)P.n_items * P.n_kv_tiles;
+        g0 = T * c / P.n_cta;
+        g1 = T * (c + 1) / P.n_cta;
+    } else {
+        const int item = c / P.n_splits, s = c % P.n_splits;
+        g0 = (long long)item * P.n_kv_tiles + (long long)P.n_kv_tiles * s / P.n_splits;
+        g1 = (long long)item * P.n_kv_tiles + (long long)P.n_kv_tiles * (s + 1) / P.n_splits;
+    }
+}
+// persistent form: the CTA whose run holds step x
+__device__ __forceinline__ int cta_of_step(const TcParams &P, long long x) {
+    const long long T = (long long)P.n_items * P.n_kv_tiles;
+    return (int)(((x + 1) * P.n_cta + T - 1) / T) - 1;
+}
+// number of parts of an item, and the part the unit of CTA c is
+__device__ __forceinline__ void item_parts(const TcParams &P, int item, int c, int &part, int &parts) {
+    if (P.persistent) {
+        const int first = cta_of_step(P, (long long)item * P.n_kv_tiles);
+        const int last = cta_of_step(P, (long long)item * P.n_kv_tiles + P.n_kv_tiles - 1);
+        part = c - first;
+        parts = last - first + 1;
+    } else {
+        part = c % P.n_splits;
+        parts = P.n_splits;
+    }
+}
+struct Unit { int item, jb, n_j; };   // key tiles jb .. jb + n_j - 1 of an item
+__device__ __forceinline__ Unit unit_at(const TcParams &P, long long g, long long g1) {
+    Unit u;
+    u.item = (int)(g / P.n_kv_tiles);
+    u.jb = (int)(g - (long long)u.item * P.n_kv_tiles);
+    u.n_j = (int)min((long long)(P.n_kv_tiles - u.jb), g1 - g);
+    return u;
+}
+
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
             const __grid_constant__ CUtensorMap map_v0, const __grid_constant__ CUtensorMap map_v1,
@@ -157,19 +205,14 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     auto bar = [&](int i) { return bar0 + 8u * i; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // work item
-    const int item = blockIdx.x / P.n_splits, split = blockIdx.x % P.n_splits;
-    const int g = item / P.pairs_per_g, pair = item % P.pairs_per_g;
-    const int n_tiles_q = min(2, P.tiles_per_g - 2 * pair);            // 1 when the head group has an odd tile count
-    const int jt0 = (int)(((long long)P.n_kv_tiles * split) / P.n_splits);
-    const int jt1 = (int)(((long long)P.n_kv_tiles * (split + 1)) / P.n_splits);
-    const int n_j = jt1 - jt0;
+    long long G0, G1;
+    cta_run(P, (int)blockIdx.x, G0, G1);           // this CTA's run of steps (never empty: the host sizes the grid so)
 
     if (threadIdx.x == 0) {
         mbar_init(bar(BAR_Q), 1);
+        mbar_init(bar(BAR_QFREE), 1);
+        mbar_init(bar(BAR_KEMPTY), 1);
         for (int s = 0; s < KV_STAGES; ++s) {
-            mbar_init(bar(BAR_KFULL + s), 1);
-            mbar_init(bar(BAR_KEMPTY + s), 1);
             mbar_init(bar(BAR_VFULL + s), 1);
             mbar_init(bar(BAR_VEMPTY + s), 1);
         }
@@ -191,42 +234,57 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    pc_grid_dep_wait();   // barriers and TMEM are set up; from here on the rotated K / Q of the pre-pass are read
+    pc_grid_dep_wait();   // barriers and TMEM are set up; from here on the rotated K / Q are read
 
+    // Steps are counted through the whole run (gs): ring stages and barrier phases follow gs, so a unit boundary is an
+    // ordinary step for the key / value pipeline.  Both query tiles always run; a unit whose head group has an odd tile
+    // count loads its one tile twice and the second copy's result is dropped.
     // the softmax warps hold a whole 128-column score row per thread: registers move from warps 0-3 to warps 4-11
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         reg_dealloc<72>();
         if (lane == 0) {
-            // The first K tile rides with the query tiles.  After that V(j) and K(j+1) always travel together: they are
-            // needed at the same point (top of step j) and their stages are released at the same point (end of step j),
-            // so one full / empty barrier pair serves both and the issuer has one wait and one commit less per step.
-            mbar_expect_tx(bar(BAR_Q), (n_tiles_q + (n_j > 0 ? 1 : 0)) * TILE_BYTES + P.extra_tx);
-            for (int t = 0; t < n_tiles_q; ++t) {
-                const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
-                tma_load_2d(base + SM_Q + t * TILE_BYTES, &map_q, h * TILE, tb * TILE, bar(BAR_Q));
-                tma_load_2d(base + SM_Q + t * TILE_BYTES + HALF_BYTES, &map_q, h * TILE + 64, tb * TILE, bar(BAR_Q));
-            }
-            if (n_j > 0) {
-                tma_load_2d(base + SM_K, &map_k, g * TILE, jt0 * TILE, bar(BAR_Q));
-                tma_load_2d(base + SM_K + HALF_BYTES, &map_k, g * TILE + 64, jt0 * TILE, bar(BAR_Q));
-            }
+            // A unit's query tiles arrive on BAR_Q once the last QK^T of the unit before has completed (BAR_QFREE); the
+            // run's first K tile rides with the first queries.  After that V(step) and K(step + 1) always travel together:
+            // they are needed at the same point and their stages are released at the same point, so one full / empty
+            // barrier pair serves both.  K(step + 1) may be the first tile of the next unit.
             bool alive = true;
-            for (int j = 0; j < n_j && alive; ++j) {
-                const int st = j % KV_STAGES, use = j / KV_STAGES, kst = (j + 1) % KV_STAGES;
-                int seg, local, n_valid;
-                kv_tile_info(P, jt0 + j, seg, local, n_valid);
-                const CUtensorMap *mv = seg == 0 ? &map_v0 : (seg == 1 ? &map_v1 : &map_v2);
-                if (use > 0) alive = mbar_wait(bar(BAR_VEMPTY + st), (use - 1) & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
-                else if (j == 1) alive = mbar_wait(bar(BAR_KEMPTY + 0), 0, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);   // K(2) lands where K(0) was
+            int gs = 0, un = 0;
+            for (long long g = G0; g < G1 && alive; ++un) {
+                const Unit U = unit_at(P, g, G1);
+                g += U.n_j;
+                const int kvh = U.item / P.pairs_per_g, pair = U.item % P.pairs_per_g;
+                const int n_tiles_q = min(2, P.tiles_per_g - 2 * pair);
+                if (un > 0) alive = mbar_wait(bar(BAR_QFREE), (un - 1) & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
                 if (!alive) break;
-                const bool more = j + 1 < n_j;
-                mbar_expect_tx(bar(BAR_VFULL + st), (more ? 2 : 1) * TILE_BYTES);
-                tma_load_2d(base + SM_V + st * TILE_BYTES, mv, g * TILE, local * TILE, bar(BAR_VFULL + st));
-                tma_load_2d(base + SM_V + st * TILE_BYTES + HALF_BYTES, mv, g * TILE + 64, local * TILE, bar(BAR_VFULL + st));
-                if (more) {
-                    tma_load_2d(base + SM_K + kst * TILE_BYTES, &map_k, g * TILE, (jt0 + j + 1) * TILE, bar(BAR_VFULL + st));
-                    tma_load_2d(base + SM_K + kst * TILE_BYTES + HALF_BYTES, &map_k, g * TILE + 64, (jt0 + j + 1) * TILE, bar(BAR_VFULL + st));
+                mbar_expect_tx(bar(BAR_Q), (2 + (un == 0 ? 1 : 0)) * TILE_BYTES + (un == 0 ? P.extra_tx : 0u));
+                for (int t = 0; t < 2; ++t) {
+                    const int T = 2 * pair + min(t, n_tiles_q - 1), tb = T / P.group, h = kvh * P.group + T % P.group;
+                    tma_load_2d(base + SM_Q + t * TILE_BYTES, &map_q, h * TILE, tb * TILE, bar(BAR_Q));
+                    tma_load_2d(base + SM_Q + t * TILE_BYTES + HALF_BYTES, &map_q, h * TILE + 64, tb * TILE, bar(BAR_Q));
+                }
+                if (un == 0) {
+                    tma_load_2d(base + SM_K, &map_k, kvh * TILE, U.jb * TILE, bar(BAR_Q));
+                    tma_load_2d(base + SM_K + HALF_BYTES, &map_k, kvh * TILE + 64, U.jb * TILE, bar(BAR_Q));
+                }
+                for (int j = 0; j < U.n_j && alive; ++j, ++gs) {
+                    const int st = gs % KV_STAGES, use = gs / KV_STAGES, kst = (gs + 1) % KV_STAGES;
+                    int seg, local, n_valid;
+                    kv_tile_info(P, U.jb + j, seg, local, n_valid);
+                    const CUtensorMap *mv = seg == 0 ? &map_v0 : (seg == 1 ? &map_v1 : &map_v2);
+                    if (use > 0) alive = mbar_wait(bar(BAR_VEMPTY + st), (use - 1) & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
+                    else if (gs == 1) alive = mbar_wait(bar(BAR_KEMPTY), 0, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);   // K(2) lands where K(0) was
+                    if (!alive) break;
+                    const bool in_unit = j + 1 < U.n_j, more = in_unit || g < G1;
+                    mbar_expect_tx(bar(BAR_VFULL + st), (more ? 2 : 1) * TILE_BYTES);
+                    tma_load_2d(base + SM_V + st * TILE_BYTES, mv, kvh * TILE, local * TILE, bar(BAR_VFULL + st));
+                    tma_load_2d(base + SM_V + st * TILE_BYTES + HALF_BYTES, mv, kvh * TILE + 64, local * TILE, bar(BAR_VFULL + st));
+                    if (more) {
+                        // the next step's keys: the next tile of this item, or the first tile of the next item
+                        const int nk = in_unit ? kvh : (U.item + 1) / P.pairs_per_g, nj = in_unit ? U.jb + j + 1 : 0;
+                        tma_load_2d(base + SM_K + kst * TILE_BYTES, &map_k, nk * TILE, nj * TILE, bar(BAR_VFULL + st));
+                        tma_load_2d(base + SM_K + kst * TILE_BYTES + HALF_BYTES, &map_k, nk * TILE + 64, nj * TILE, bar(BAR_VFULL + st));
+                    }
                 }
             }
             if (*abort_flag) {
@@ -242,7 +300,6 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         reg_dealloc<72>();
         const bool lead = elect_one();
         const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-        bool alive = mbar_wait(bar(BAR_Q), 0, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
         auto issue_qk = [&](int t, int st) {
             const uint32_t qa = base + SM_Q + t * TILE_BYTES, ka = base + SM_K + st * TILE_BYTES;
 #pragma unroll
@@ -251,38 +308,55 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
                 if (lead) mma_ss(tm + t * TILE, desc_kmajor(qa + off), desc_kmajor(ka + off), IDESC_QK, ks > 0);
             }
         };
-        if (alive && n_j > 0) {
+        bool alive = mbar_wait(bar(BAR_Q), 0, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
+        int gs = 0, un = 0;
+        if (alive) {
             tc_fence_after();
-            for (int t = 0; t < n_tiles_q; ++t) {
+            for (int t = 0; t < 2; ++t) {
                 issue_qk(t, 0);
                 if (lead) tc_commit(bar(BAR_SFULL + t));
             }
-            if (lead) tc_commit(bar(BAR_KEMPTY + 0));
+            if (lead) tc_commit(bar(BAR_KEMPTY));
+            if (unit_at(P, G0, G1).n_j == 1 && lead) tc_commit(bar(BAR_QFREE));      // that was the first unit's only QK^T
         }
-        for (int j = 0; j < n_j && alive; ++j) {
-            const int st = j % KV_STAGES, use = j / KV_STAGES;
-            const int nst = (j + 1) % KV_STAGES;
-            alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);      // V(j) and K(j+1)
-            for (int t = 0; t < n_tiles_q && alive; ++t) {
-                const uint32_t va = base + SM_V + st * TILE_BYTES;
-                // P arrives in two halves of 64 keys: the first PV steps run while the rest is exponentiated
-                for (int hf = 0; hf < 2 && alive; ++hf) {
-                    alive = mbar_wait(bar(BAR_PHALF + 2 * t + hf), j & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
-                    if (!alive) break;
-                    tc_fence_after();
+        for (long long g = G0; g < G1 && alive; ++un) {
+            const Unit U = unit_at(P, g, G1);
+            g += U.n_j;
+            const int next_n_j = g < G1 ? unit_at(P, g, G1).n_j : 0;
+            for (int j = 0; j < U.n_j && alive; ++j, ++gs) {
+                const int st = gs % KV_STAGES, use = gs / KV_STAGES, nst = (gs + 1) % KV_STAGES;
+                alive = mbar_wait(bar(BAR_VFULL + st), use & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);      // V(step) and K(step + 1)
+                const bool in_unit = j + 1 < U.n_j, more = in_unit || next_n_j > 0;
+                for (int t = 0; t < 2 && alive; ++t) {
+                    const uint32_t va = base + SM_V + st * TILE_BYTES;
+                    // P arrives in two halves of 64 keys: the first PV steps run while the rest is exponentiated
+                    for (int hf = 0; hf < 2 && alive; ++hf) {
+                        alive = mbar_wait(bar(BAR_PHALF + 2 * t + hf), gs & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
+                        if (!alive) break;
+                        tc_fence_after();
 #pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4) {   // 16 keys per step: P columns advance by 8 (two bf16 per column)
-                        const int ks = hf * 4 + k4;
-                        if (lead)
-                            mma_ts(tm + 256 + t * TILE, tm + t * TILE + ks * 8, desc_mnmajor(va + ks * 2048), IDESC_PV, (j > 0 || ks > 0));
+                        for (int k4 = 0; k4 < 4; ++k4) {   // 16 keys per step: P columns advance by 8 (two bf16 per column)
+                            const int ks = hf * 4 + k4;
+                            if (lead)
+                                mma_ts(tm + 256 + t * TILE, tm + t * TILE + ks * 8, desc_mnmajor(va + ks * 2048), IDESC_PV, (j > 0 || ks > 0));
+                        }
                     }
+                    if (!alive) break;
+                    if (more) {
+                        if (!in_unit && t == 0) {           // the next unit's queries must be in before its first QK^T
+                            alive = mbar_wait(bar(BAR_Q), (un + 1) & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us);
+                            if (!alive) break;
+                            tc_fence_after();
+                        }
+                        issue_qk(t, nst);
+                    }
+                    if (lead) tc_commit(bar(BAR_SFULL + t));          // S_t of the next step ready, and / or O_t of this unit final
                 }
-                if (!alive) break;
-                if (j + 1 < n_j) issue_qk(t, nst);
-                if (lead) tc_commit(bar(BAR_SFULL + t));          // S_t(j+1) ready, or after the last tile: O_t final
-            }
-            if (alive && lead) {
-                tc_commit(bar(BAR_VEMPTY + st));            // PV(j) and QK(j+1) are behind this: V stage st and K stage nst are free
+                if (alive && lead) {
+                    // the QK^T just issued were the last of their unit: its query tiles may be overwritten
+                    if (more && (in_unit ? j + 2 == U.n_j : next_n_j == 1)) tc_commit(bar(BAR_QFREE));
+                    tc_commit(bar(BAR_VEMPTY + st));        // PV(step) and QK(step + 1) are behind this: V stage st and K stage nst are free
+                }
             }
         }
         // make sure nothing of ours is still running on the tensor core before TMEM is freed
@@ -300,134 +374,140 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const uint32_t s_addr = tmem + lane_addr + t * TILE;
         const uint32_t o_addr = tmem + lane_addr + 256 + t * TILE;
-        float m_used = -INFINITY, l = 0.f;
-        bool alive = t < n_tiles_q;
-        for (int j = 0; j < n_j && alive; ++j) {
-            int seg, local, n_valid;
-            kv_tile_info(P, jt0 + j, seg, local, n_valid);
-            alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), j & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us));
-            if (!alive) break;
-            tc_fence_after();
-            // the whole score row of this thread: one TMEM pass
-            uint32_t sv[128];
-            tmem_ld32(s_addr, sv);
-            tmem_ld32(s_addr + 32, sv + 32);
-            tmem_ld32(s_addr + 64, sv + 64);
-            tmem_ld32(s_addr + 96, sv + 96);
-            tmem_wait_ld();
-            if (n_valid < TILE) {                        // ragged last tile of a segment: keys past its end score -inf
+        bool alive = true;
+        int gs = 0;
+        for (long long g = G0; g < G1 && alive;) {
+            const Unit U = unit_at(P, g, G1);
+            g += U.n_j;
+            const int kvh = U.item / P.pairs_per_g, pair = U.item % P.pairs_per_g;
+            const int n_tiles_q = min(2, P.tiles_per_g - 2 * pair);
+            float m_used = -INFINITY, l = 0.f;
+            for (int j = 0; j < U.n_j && alive; ++j, ++gs) {
+                int seg, local, n_valid;
+                kv_tile_info(P, U.jb + j, seg, local, n_valid);
+                alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), gs & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us));
+                if (!alive) break;
+                tc_fence_after();
+                // the whole score row of this thread: one TMEM pass
+                uint32_t sv[128];
+                tmem_ld32(s_addr, sv);
+                tmem_ld32(s_addr + 32, sv + 32);
+                tmem_ld32(s_addr + 64, sv + 64);
+                tmem_ld32(s_addr + 96, sv + 96);
+                tmem_wait_ld();
+                if (n_valid < TILE) {                        // ragged last tile of a segment: keys past its end score -inf
 #pragma unroll
-                for (int i = 0; i < TILE; ++i)
-                    if (i >= n_valid) sv[i] = 0xFF800000u;
-            }
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                    for (int i = 0; i < TILE; ++i)
+                        if (i >= n_valid) sv[i] = 0xFF800000u;
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < TILE; i += 4) {
-                mx0 = fmaxf(mx0, __uint_as_float(sv[i]));
-                mx1 = fmaxf(mx1, __uint_as_float(sv[i + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(sv[i + 2]));
-                mx3 = fmaxf(mx3, __uint_as_float(sv[i + 3]));
-            }
-            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            // lazy rescale: move the reference maximum only when it grew by more than the threshold
-            const bool grow = mx > m_used + RESCALE_THRESHOLD;
-            if (__any_sync(0xffffffffu, grow)) {
-                const float m_new = fmaxf(m_used, mx);
-                const float corr = fast_exp2(m_used - m_new);       // 0 on the first tile (m_used = -inf)
-                l *= corr;
-                if (j > 0) {
-                    uint32_t v[32];
+                for (int i = 0; i < TILE; i += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(sv[i]));
+                    mx1 = fmaxf(mx1, __uint_as_float(sv[i + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(sv[i + 2]));
+                    mx3 = fmaxf(mx3, __uint_as_float(sv[i + 3]));
+                }
+                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                // lazy rescale: move the reference maximum only when it grew by more than the threshold
+                const bool grow = mx > m_used + RESCALE_THRESHOLD;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float m_new = fmaxf(m_used, mx);
+                    const float corr = fast_exp2(m_used - m_new);       // 0 on the first tile (m_used = -inf)
+                    l *= corr;
+                    if (j > 0) {
+                        uint32_t v[32];
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        tmem_ld32(o_addr + c * 32, v);
-                        tmem_wait_ld();
+                        for (int c = 0; c < 4; ++c) {
+                            tmem_ld32(o_addr + c * 32, v);
+                            tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
-                        tmem_st32(o_addr + c * 32, v);
+                            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * corr);
+                            tmem_st32(o_addr + c * 32, v);
+                        }
+                    }
+                    m_used = m_new;
+                }
+                // p = 2^(s - m) as bf16 pairs, written over the S columns; the row sum runs on two-lane adds
+                const float2 neg_m = make_float2(-m_used, -m_used);
+                float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) {
+                        float2 x = add2(make_float2(__uint_as_float(sv[c * 32 + 2 * i]), __uint_as_float(sv[c * 32 + 2 * i + 1])), neg_m);
+                        float2 y = add2(make_float2(__uint_as_float(sv[c * 32 + 2 * i + 2]), __uint_as_float(sv[c * 32 + 2 * i + 3])), neg_m);
+                        x.x = fast_exp2(x.x); x.y = fast_exp2(x.y);
+                        y.x = fast_exp2(y.x); y.y = fast_exp2(y.y);
+                        la = add2(la, x);
+                        lb = add2(lb, y);
+                        pk[i] = pc_pack_bf16(x.x, x.y);
+                        pk[i + 1] = pc_pack_bf16(y.x, y.y);
+                    }
+                    tmem_st16(s_addr + c * 16, pk);
+                    if (c & 1) {                               // keys 0-63, then 64-127, handed to the tensor core
+                        tmem_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar(BAR_PHALF + 2 * t + (c >> 1)));
                     }
                 }
-                m_used = m_new;
+                l += (la.x + la.y) + (lb.x + lb.y);
             }
-            // p = 2^(s - m) as bf16 pairs, written over the S columns; the row sum runs on two-lane adds
-            const float2 neg_m = make_float2(-m_used, -m_used);
-            float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    float2 x = add2(make_float2(__uint_as_float(sv[c * 32 + 2 * i]), __uint_as_float(sv[c * 32 + 2 * i + 1])), neg_m);
-                    float2 y = add2(make_float2(__uint_as_float(sv[c * 32 + 2 * i + 2]), __uint_as_float(sv[c * 32 + 2 * i + 3])), neg_m);
-                    x.x = fast_exp2(x.x); x.y = fast_exp2(x.y);
-                    y.x = fast_exp2(y.x); y.y = fast_exp2(y.y);
-                    la = add2(la, x);
-                    lb = add2(lb, y);
-                    pk[i] = pc_pack_bf16(x.x, x.y);
-                    pk[i + 1] = pc_pack_bf16(y.x, y.y);
-                }
-                tmem_st16(s_addr + c * 16, pk);
-                if (c & 1) {                               // keys 0-63, then 64-127, handed to the tensor core
-                    tmem_wait_st();
-                    tc_fence_before();
-                    mbar_arrive(bar(BAR_PHALF + 2 * t + (c >> 1)));
-                }
-            }
-            l += (la.x + la.y) + (lb.x + lb.y);
-        }
-        // epilogue: O_t is final once the last PV has committed
-        if (alive && n_j > 0) alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), n_j & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us));
-        if (alive && n_j > 0) {
-            tc_fence_after();
-            const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
-            const int row = tb * TILE + r;
-            uint32_t v[32];
-            if (P.n_splits == 1) {
-                const float inv = 1.f / l;
-                __nv_bfloat16 *orow = P.out + ((size_t)row * P.n_q_heads + h) * TILE;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    tmem_ld32(o_addr + c * 32, v);
-                    tmem_wait_ld();
+            // epilogue of the unit: O_t is final once the last PV has committed.  The same commit may also carry the first
+            // scores of the next unit; its phase is then waited for a second time at the top of the loop, which returns at once.
+            if (alive) alive = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + t), gs & 1, abort_flag, P.status, PC_WHERE_ATTN_WAIT, P.wait_us));
+            if (alive && t < n_tiles_q) {
+                tc_fence_after();
+                int part, parts;
+                item_parts(P, U.item, (int)blockIdx.x, part, parts);
+                const int T = 2 * pair + t, tb = T / P.group, h = kvh * P.group + T % P.group;
+                const int row = tb * TILE + r;
+                // the thread's whole O row leaves TMEM in one pass (four loads in flight, one wait): at a unit boundary the
+                // tensor core idles until O is free again, so the read-out is on the critical path
+                uint32_t v[128];
+                tmem_ld32(o_addr, v);
+                tmem_ld32(o_addr + 32, v + 32);
+                tmem_ld32(o_addr + 64, v + 64);
+                tmem_ld32(o_addr + 96, v + 96);
+                tmem_wait_ld();
+                if (parts == 1) {
+                    const float inv = 1.f / l;
+                    __nv_bfloat16 *orow = P.out + ((size_t)row * P.n_q_heads + h) * TILE;
                     if (row < P.n_q) {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
+                        for (int i = 0; i < 16; ++i) {
                             uint4 w;
                             w.x = pc_pack_bf16(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
                             w.y = pc_pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
                             w.z = pc_pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
                             w.w = pc_pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
-                            *reinterpret_cast<uint4 *>(orow + c * 32 + i * 8) = w;
+                            *reinterpret_cast<uint4 *>(orow + i * 8) = w;
                         }
                     }
-                }
-                if (P.lse && row < P.n_q) P.lse[(size_t)row * P.n_q_heads + h] = (m_used + log2f(l)) * 0.6931471805599453f;
-            } else if (P.cluster) {
-                // Stage O (un-normalised, fp32) and (max, sum) in shared memory that no multiply-add reads any more:
-                // tile 0 over both query tiles (every QK^T has completed once this tile's last PV has), tile 1 over the
-                // key stages (its own last PV is the last multiply-add of the CTA).
-                const uint32_t stage = base + (t == 0 ? SM_Q : SM_K);
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    tmem_ld32(o_addr + c * 32, v);
-                    tmem_wait_ld();
+                    if (P.lse && row < P.n_q) P.lse[(size_t)row * P.n_q_heads + h] = (m_used + log2f(l)) * 0.6931471805599453f;
+                } else if (P.cluster) {
+                    // (split form, one unit per CTA) Stage O (un-normalised, fp32) and (max, sum) in shared memory that no
+                    // multiply-add reads any more: tile 0 over both query tiles (every QK^T has completed once this tile's
+                    // last PV has), tile 1 over the key stages (its own last PV is the last multiply-add of the CTA).
+                    const uint32_t stage = base + (t == 0 ? SM_Q : SM_K);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) sts128(stage + stage_off(c * 8 + i, r), v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                }
-                *reinterpret_cast<float2 *>(gen + SM_ML + (t * TILE + r) * 8) = make_float2(m_used, l);
-            } else {
-                // Partial tile layout: 16-byte unit (c4, r) = columns 4*c4..4*c4+3 of row r at unit c4*128 + r, so the 32 rows
-                // of a warp store 512 contiguous bytes per instruction (a row-major tile would touch 32 lines per store).
-                const size_t tile_slot = (size_t)blockIdx.x * 2 + t;
-                uint4 *ptile = reinterpret_cast<uint4 *>(P.part_o) + tile_slot * (TILE * TILE / 4) + r;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    tmem_ld32(o_addr + c * 32, v);
-                    tmem_wait_ld();
+                    for (int i = 0; i < 32; ++i) sts128(stage + stage_off(i, r), v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    *reinterpret_cast<float2 *>(gen + SM_ML + (t * TILE + r) * 8) = make_float2(m_used, l);
+                } else {
+                    // Partial tile layout: 16-byte unit (c4, r) = columns 4*c4..4*c4+3 of row r at unit c4*128 + r, so the 32 rows
+                    // of a warp store 512 contiguous bytes per instruction (a row-major tile would touch 32 lines per store).
+                    const size_t tile_slot = ((size_t)U.item * P.part_stride + part) * 2 + t;
+                    uint4 *ptile = reinterpret_cast<uint4 *>(P.part_o) + tile_slot * (TILE * TILE / 4) + r;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        ptile[(c * 8 + i) * TILE] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    for (int i = 0; i < 32; ++i) ptile[i * TILE] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    *reinterpret_cast<float2 *>(P.part_ml + (tile_slot * TILE + r) * 2) = make_float2(m_used, l);
                 }
-                *reinterpret_cast<float2 *>(P.part_ml + (tile_slot * TILE + r) * 2) = make_float2(m_used, l);
+            }
+            if (alive && g < G1) {
+                // the next unit's first PV overwrites O: every read of it above must have completed (the loads have: each is
+                // followed by its wait), and the tensor core must see that before the P of the next step is handed over
+                tc_fence_before();
             }
         }
     }
@@ -441,6 +521,9 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
         // Merge the KV ranges of this item across the cluster: CTA `rank` finishes every n_splits-th row of the two
         // tiles, reading each peer's staged O and (max, sum) through distributed shared memory.  Sixteen threads share
         // a row (two 16-byte units each), so a row's 256 output bytes leave as two 128-byte runs.
+        const int item = (int)blockIdx.x / P.n_splits;
+        const int kvh = item / P.pairs_per_g, pair = item % P.pairs_per_g;
+        const int n_tiles_q = min(2, P.tiles_per_g - 2 * pair);
         cluster_sync_all();                        // every CTA's staging is complete and visible
         if (warp >= 4) {
             const int S = P.n_splits, my = (int)cluster_rank();
@@ -451,7 +534,7 @@ k_attend_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ C
             for (int R = my + slot * S; R < 2 * TILE; R += 16 * S) {
                 const int t = R >> 7, r = R & (TILE - 1);
                 if (t >= n_tiles_q) break;
-                const int T = 2 * pair + t, tb = T / P.group, h = g * P.group + T % P.group;
+                const int T = 2 * pair + t, tb = T / P.group, h = kvh * P.group + T % P.group;
                 const int row = tb * TILE + r;
                 if (row >= P.n_q) continue;
                 float mk[MAX_SPLITS], lk[MAX_SPLITS], m = -INFINITY;
@@ -500,12 +583,15 @@ __global__ void __launch_bounds__(256) k_combine(const TcParams P) {
     const int item = g * P.pairs_per_g + (T >> 1), t = T & 1;
     const int r = quad * 32 + lane, row = tb * TILE + r;
     if (row >= P.n_q) return;
+    int part0, n_parts;
+    item_parts(P, item, 0, part0, n_parts);
+    if (n_parts < 2) return;                      // the one CTA that had the whole item wrote its output itself
     float2 ml[MAX_SPLITS];
     float4 o[MAX_SPLITS][4];
 #pragma unroll
     for (int s = 0; s < MAX_SPLITS; ++s)
-        if (s < P.n_splits) {
-            const size_t tile_slot = ((size_t)item * P.n_splits + s) * 2 + t;
+        if (s < n_parts) {
+            const size_t tile_slot = ((size_t)item * P.part_stride + s) * 2 + t;
             ml[s] = __ldcg(reinterpret_cast<const float2 *>(P.part_ml) + tile_slot * TILE + r);
             const float4 *pt = reinterpret_cast<const float4 *>(P.part_o) + tile_slot * (TILE * TILE / 4) + r;
 #pragma unroll
@@ -514,14 +600,14 @@ __global__ void __launch_bounds__(256) k_combine(const TcParams P) {
     float m = -INFINITY;
 #pragma unroll
     for (int s = 0; s < MAX_SPLITS; ++s)
-        if (s < P.n_splits) m = fmaxf(m, ml[s].x);
+        if (s < n_parts) m = fmaxf(m, ml[s].x);
     float l = 0.f;
     float4 acc[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int s = 0; s < MAX_SPLITS; ++s)
-        if (s < P.n_splits) {
+        if (s < n_parts) {
             const float sc = exp2f(ml[s].x - m);
             l = fmaf(ml[s].y, sc, l);
 #pragma unroll
@@ -625,7 +711,7 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     P.n_kv_tiles = tiles;
     P.n_seg = n_seg;
     const int n_items = D.n_kv_heads * P.pairs_per_g;
-    P.n_splits = ctx->kv_splits > 0 ? std::min(ctx->kv_splits, tiles) : choose_splits(n_items, tiles, ctx->sm_count);
+    P.n_items = n_items;
     P.out = static_cast<__nv_bfloat16 *>(out);
     P.lse = lse;
     P.part_o = ctx->part_o;
@@ -633,7 +719,29 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
     P.status = ctx->status;
     P.wait_us = ctx->wait_limit_us;
     P.extra_tx = ctx->test_extra_tx;
-    if (P.n_splits > 1 && !ctx->cluster_merge && (size_t)n_items * P.n_splits * 2 * TILE * TILE > ctx->part_o_floats) return PC_ERR_CAPACITY;
+    // Persistent form unless the caller fixed the number of key ranges or asked for the cluster merge: one CTA per SM, but
+    // never so many that an item is cut into more than MAX_SPLITS parts (a CTA's run is at least a third of an item).
+    const long long T = (long long)n_items * tiles;
+    P.persistent = (ctx->kv_splits == 0 && !ctx->cluster_merge) ? 1 : 0;
+    if (P.persistent) {
+        P.n_cta = (int)std::min<long long>(std::min<long long>(ctx->sm_count, (long long)n_items * (MAX_SPLITS - 1)), T);
+        int most = 1;
+        for (int i = 0; i < n_items; ++i) {        // the kernel's own rule (cta_of_step), evaluated for every item
+            const long long x0 = (long long)i * tiles, x1 = x0 + tiles - 1;
+            const int first = (int)(((x0 + 1) * P.n_cta + T - 1) / T) - 1, last = (int)(((x1 + 1) * P.n_cta + T - 1) / T) - 1;
+            most = std::max(most, last - first + 1);
+        }
+        if (most > MAX_SPLITS) P.persistent = 0;
+        P.part_stride = most;
+        P.n_splits = most;
+    }
+    if (!P.persistent) {
+        P.n_splits = ctx->kv_splits > 0 ? std::min(ctx->kv_splits, tiles) : choose_splits(n_items, tiles, ctx->sm_count);
+        P.n_cta = n_items * P.n_splits;
+        P.part_stride = P.n_splits;
+    }
+    P.cluster = (!P.persistent && P.n_splits > 1 && ctx->cluster_merge) ? 1 : 0;
+    if (P.part_stride > 1 && !P.cluster && (size_t)n_items * P.part_stride * 2 * TILE * TILE > ctx->part_o_floats) return PC_ERR_CAPACITY;
 
     CUtensorMap mq, mk, mv[PC_MAX_SEGMENTS];
     bool ok = make_map(&mq, q_rot, (uint64_t)n_q, (uint64_t)D.n_q_heads * D.head_dim) &&
@@ -652,10 +760,9 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
         PC_CUDA_TRY(cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC));
         attr_set[ctx->device] = true;
     }
-    P.cluster = (P.n_splits > 1 && ctx->cluster_merge) ? 1 : 0;
     if (P.cluster) {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(n_items * P.n_splits);
+        cfg.gridDim = dim3(P.n_cta);
         cfg.blockDim = dim3(TC_THREADS);
         cfg.dynamicSmemBytes = SM_ALLOC;
         cfg.stream = stream;
@@ -668,11 +775,11 @@ pc_status pc_launch_attend_tc(pc_ctx *ctx, int n_seg, const pc_segment *segs, co
         cfg.numAttrs = 1;
         PC_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_attend_tc, mq, mk, mv[0], mv[1], mv[2], P));
     } else {
-        PC_LAUNCH(k_attend_tc, dim3(n_items * P.n_splits), dim3(TC_THREADS), SM_ALLOC, stream, mq, mk, mv[0], mv[1], mv[2], P);
+        PC_LAUNCH(k_attend_tc, dim3(P.n_cta), dim3(TC_THREADS), SM_ALLOC, stream, mq, mk, mv[0], mv[1], mv[2], P);
     }
     PC_CUDA_TRY(cudaGetLastError());
     pc_mark(ctx, PC_MARK_ATTEND, stream);
-    if (P.n_splits > 1 && !P.cluster) {
+    if (P.part_stride > 1 && !P.cluster) {
         PC_LAUNCH(k_combine, dim3(P.n_tb * D.n_q_heads * 4), dim3(256), 0, stream, P);
         PC_CUDA_TRY(cudaGetLastError());
         pc_mark(ctx, PC_MARK_COMBINE, stream);
