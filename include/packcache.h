@@ -318,6 +318,37 @@ pc_status pc_window_append_masked(pc_window *w, const pc_segment *frame, const u
 pc_status pc_window_update(pc_window *w, const void *q, const int32_t *q_pos, int32_t n_q, const float *scores_override,
                            int32_t *regime, void *stream);
 
+/* Update and attention in one call: what pc_window_update (without an override) followed by pc_attend_frame over the
+ * window's cache give, bit for bit, through the fused frame step (pc_frame_step) whenever the update packs.
+ *   q, q_pos device; out device [n_q][Hq][d]; lse device or NULL; regime host out or NULL. */
+pc_status pc_window_step(pc_window *w, const void *q, const int32_t *q_pos, int32_t n_q, void *out, float *lse,
+                         int32_t *regime, void *stream);
+
+/* The same step with its per-frame inputs and its output in HOST memory, the cache staying resident on the device
+ * (Fig. 6c: in the steady state a frame brings only its own keys, values and queries; Eq. 3: the cache itself is
+ * bounded): copies the frame that was just finished (its K, V, positions; n_frame may be 0) to the end of the active
+ * history buffer and the new frame's queries and positions into the workspace, runs pc_window_step, copies the
+ * output back and waits for the stream.  Pinned host memory keeps the copies asynchronous.  All arguments are checked
+ * before anything is enqueued.  Errors: as pc_window_append and pc_window_step. */
+typedef struct {
+    const void *frame_k, *frame_v; /* host [n_frame][Hkv][d]: the frame to append as the newest history frame */
+    const int32_t *frame_pos;      /* host [n_frame][4], in the shifted frame of reference (pc_window_state) */
+    int32_t n_frame;
+    const void *q;                 /* host [n_q][Hq][d] */
+    const int32_t *q_pos;          /* host [n_q][4] */
+    int32_t n_q;
+    void *out;                     /* host out [n_q][Hq][d] */
+} pc_host_window_step;
+
+typedef struct {
+    void *q;        /* device [>= n_q][Hq][d] */
+    int32_t *q_pos; /* device [>= n_q][4] */
+    void *out;      /* device [>= n_q][Hq][d] */
+} pc_window_step_workspace;
+
+pc_status pc_window_step_host(pc_window *w, const pc_host_window_step *in, const pc_window_step_workspace *ws,
+                              int32_t *regime, void *stream);
+
 /* The current cache as a pc_cache for pc_attend_frame (frame_count points into the window: valid until the next
  * append / update / destroy). */
 pc_status pc_window_cache(pc_window *w, pc_cache *out);

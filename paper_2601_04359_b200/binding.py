@@ -26,7 +26,7 @@ EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact"
            "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge",
            "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_append_masked", "pc_window_update", "pc_window_cache",
            "pc_window_state", "pc_attend_prepare", "pc_attend_prepared", "pc_attend_mass", "pc_frame_step",
-           "pc_forget_anchors", "pc_set_wait_limit_us", "pc_test_expect_extra_bytes"]
+           "pc_forget_anchors", "pc_set_wait_limit_us", "pc_test_expect_extra_bytes", "pc_window_step", "pc_window_step_host"]
 
 
 class pc_layer_desc(C.Structure):
@@ -58,6 +58,15 @@ class pc_host_frame(C.Structure):
                 ("anchor_v", C.c_void_p), ("anchor_pos", C.c_void_p), ("n_anchor", C.c_int32), ("hist_k", C.c_void_p),
                 ("hist_v", C.c_void_p), ("hist_pos", C.c_void_p), ("n_frames", C.c_int32),
                 ("frame_count", C.POINTER(C.c_int32)), ("out", C.c_void_p)]
+
+
+class pc_host_window_step(C.Structure):
+    _fields_ = [("frame_k", C.c_void_p), ("frame_v", C.c_void_p), ("frame_pos", C.c_void_p), ("n_frame", C.c_int32),
+                ("q", C.c_void_p), ("q_pos", C.c_void_p), ("n_q", C.c_int32), ("out", C.c_void_p)]
+
+
+class pc_window_step_workspace(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("q_pos", C.c_void_p), ("out", C.c_void_p)]
 
 
 class pc_device_workspace(C.Structure):
@@ -122,6 +131,10 @@ def load() -> C.CDLL:
     lib.pc_window_append.argtypes = [C.c_void_p, C.POINTER(pc_segment), C.c_void_p]
     lib.pc_window_append_masked.argtypes = [C.c_void_p, C.POINTER(pc_segment), C.c_void_p, C.c_int32, C.c_void_p]
     lib.pc_window_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int32), C.c_void_p]
+    lib.pc_window_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32),
+                                   C.c_void_p]
+    lib.pc_window_step_host.argtypes = [C.c_void_p, C.POINTER(pc_host_window_step), C.POINTER(pc_window_step_workspace),
+                                        C.POINTER(C.c_int32), C.c_void_p]
     lib.pc_window_cache.argtypes = [C.c_void_p, C.POINTER(pc_cache)]
     lib.pc_window_state.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int64),
                                     C.POINTER(C.c_int32)]
@@ -410,6 +423,29 @@ class Window:
         regime = C.c_int32(-1)
         _check(load().pc_window_update(self.handle, _ptr(q), _ptr(q_pos), 0 if q is None else q.shape[0],
                                        _ptr(scores_override), C.byref(regime), _stream(stream)), "pc_window_update")
+        return regime.value
+
+    def step(self, q: torch.Tensor, q_pos: torch.Tensor, out: Optional[torch.Tensor] = None,
+             lse: Optional[torch.Tensor] = None, stream=None):
+        """Update and attention in one call; returns (regime, out)."""
+        if out is None:
+            out = torch.empty_like(q)
+        regime = C.c_int32(-1)
+        _check(load().pc_window_step(self.handle, _ptr(q), _ptr(q_pos), q.shape[0], _ptr(out), _ptr(lse), C.byref(regime),
+                                     _stream(stream)), "pc_window_step")
+        return regime.value, out
+
+    def step_host(self, frame: Optional[dict], q: torch.Tensor, q_pos: torch.Tensor, out: torch.Tensor, ws: dict,
+                  stream=None) -> int:
+        """frame: pinned CPU tensors k, v, pos of the frame to append (or None); q, q_pos, out: pinned CPU tensors;
+        ws: device tensors q, q_pos, out.  Blocks until ``out`` holds the result; returns the regime."""
+        n = 0 if frame is None else frame["k"].shape[0]
+        h = pc_host_window_step(_ptr(frame["k"]) if n else None, _ptr(frame["v"]) if n else None,
+                                _ptr(frame["pos"]) if n else None, n, _ptr(q), _ptr(q_pos), q.shape[0], _ptr(out))
+        wsp = pc_window_step_workspace(_ptr(ws["q"]), _ptr(ws["q_pos"]), _ptr(ws["out"]))
+        regime = C.c_int32(-1)
+        _check(load().pc_window_step_host(self.handle, C.byref(h), C.byref(wsp), C.byref(regime), _stream(stream)),
+               "pc_window_step_host")
         return regime.value
 
     def state(self):

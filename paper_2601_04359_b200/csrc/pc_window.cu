@@ -1,5 +1,6 @@
 // Cache window: the Fill / Pack / Slide regimes (Sec. 3.4, Fig. 6) and the temporal rebase (Eq. 9) as a host-side state
 // machine around pc_plan_budget, pc_score and pc_compact; its one kernel turns a cache mask (Eq. 1) into row indices.
+#include <algorithm>
 #include <vector>
 
 #include "pc_common.cuh"
@@ -140,22 +141,31 @@ extern "C" pc_status pc_window_append_masked(pc_window *w, const pc_segment *fra
     return PC_OK;
 }
 
-extern "C" pc_status pc_window_update(pc_window *w, const void *q, const int32_t *q_pos, int32_t n_q,
-                                      const float *scores_override, int32_t *regime, void *stream) {
-    if (!w) return PC_ERR_INVALID_ARG;
+namespace {
+
+// What an update has to do, worked out on the host before anything is enqueued.
+struct WindowPlan {
+    bool fill;               // everything still fits: nothing to do
+    pc_cache src;            // source of the pack: the active buffer past the frames that leave
+    const int32_t *budget;   // quotas of the frames that stay (points into the window's plan)
+    int stay, left;          // frames that stay / leave (beyond the window, or starved by the plan at the old end)
+    int64_t n_sel;           // tokens kept
+    int32_t delta_t;         // temporal rebase (Eq. 9)
+    const float *scores_override;
+};
+
+pc_status window_plan(pc_window *w, const float *scores_override, WindowPlan *pl) {
     const int n_frames = (int)w->count.size();
     const int drop = std::max(0, n_frames - w->p.window);          // frames beyond the window leave first (FIFO)
     int64_t dropped_tokens = 0, kept_tokens = 0;
     for (int f = 0; f < n_frames; ++f) (f < drop ? dropped_tokens : kept_tokens) += w->count[f];
-    if (drop == 0 && kept_tokens <= w->p.budget.total) {           // Fill: everything still fits
-        if (regime) *regime = PC_WINDOW_FILL;
-        return PC_OK;
-    }
+    pl->fill = drop == 0 && kept_tokens <= w->p.budget.total;      // Fill: everything still fits
+    if (pl->fill) return PC_OK;
     const int kept = n_frames - drop;
     pc_segment &A = w->buf[w->active], &B = w->buf[w->active ^ 1];
     const size_t row = (size_t)w->ctx->desc.n_kv_heads * w->ctx->desc.head_dim * w->ctx->elem_size;
     // source: the active buffer past the dropped frames
-    pc_cache src;
+    pc_cache &src = pl->src;
     src.anchors = w->anchors;
     src.history.k = static_cast<char *>(A.k) + (size_t)dropped_tokens * row;
     src.history.v = static_cast<char *>(A.v) + (size_t)dropped_tokens * row;
@@ -172,37 +182,124 @@ extern "C" pc_status pc_window_update(pc_window *w, const void *q, const int32_t
     int lead = 0;
     int64_t lead_tokens = 0;
     while (lead < kept && w->budget[lead] == 0) lead_tokens += src.frame_count[lead++];
-    const int32_t *budget = w->budget.data() + lead;
-    const int left = drop + lead, stay = kept - lead;
+    pl->budget = w->budget.data() + lead;
+    pl->left = drop + lead;
+    pl->stay = kept - lead;
     src.history.k = static_cast<char *>(src.history.k) + (size_t)lead_tokens * row;
     src.history.v = static_cast<char *>(src.history.v) + (size_t)lead_tokens * row;
     src.history.pos += 4 * (size_t)lead_tokens;
     src.history.n_tokens -= (int32_t)lead_tokens;
     src.history.capacity -= (int32_t)lead_tokens;
-    src.n_frames = stay;
+    src.n_frames = pl->stay;
     src.frame_count += lead;
-    if (scores_override) scores_override += lead_tokens;
-    int64_t n_sel = 0;
-    for (int f = 0; f < stay; ++f) n_sel += budget[f];
-    if (n_sel > B.capacity) return PC_ERR_CAPACITY;
-    const int32_t delta_t = w->p.rebase ? left * w->p.t_step : 0;  // Eq. 9: t falls by the number of frames that left
-    if (stay > 0) {
-        st = pc_score(w->ctx, &src, q, q_pos, n_q, budget, nullptr, scores_override, w->scores, w->sel_idx, stream);
+    pl->scores_override = scores_override ? scores_override + lead_tokens : nullptr;
+    pl->n_sel = 0;
+    for (int f = 0; f < pl->stay; ++f) pl->n_sel += pl->budget[f];
+    if (pl->n_sel > B.capacity) return PC_ERR_CAPACITY;
+    pl->delta_t = w->p.rebase ? pl->left * w->p.t_step : 0;        // Eq. 9: t falls by the number of frames that left
+    return PC_OK;
+}
+
+// the other buffer becomes the active one and holds what was kept
+void window_commit(pc_window *w, const WindowPlan &pl) {
+    pc_segment &A = w->buf[w->active], &B = w->buf[w->active ^ 1];
+    B.n_tokens = (int32_t)pl.n_sel;
+    A.n_tokens = 0;
+    w->active ^= 1;
+    w->count.assign(pl.budget, pl.budget + pl.stay);
+    w->t_shift += pl.delta_t;
+}
+
+}  // namespace
+
+extern "C" pc_status pc_window_update(pc_window *w, const void *q, const int32_t *q_pos, int32_t n_q,
+                                      const float *scores_override, int32_t *regime, void *stream) {
+    if (!w) return PC_ERR_INVALID_ARG;
+    WindowPlan pl;
+    pc_status st = window_plan(w, scores_override, &pl);
+    if (st != PC_OK) return st;
+    if (pl.fill) {
+        if (regime) *regime = PC_WINDOW_FILL;
+        return PC_OK;
+    }
+    if (pl.stay > 0) {
+        st = pc_score(w->ctx, &pl.src, q, q_pos, n_q, pl.budget, nullptr, pl.scores_override, w->scores, w->sel_idx, stream);
         if (st != PC_OK) return st;
         pc_cache dst;
         dst.anchors = w->anchors;
-        dst.history = B;
-        dst.n_frames = stay;
-        dst.frame_count = budget;
-        st = pc_compact(w->ctx, &src, w->sel_idx, budget, delta_t, &dst, stream);
+        dst.history = w->buf[w->active ^ 1];
+        dst.n_frames = pl.stay;
+        dst.frame_count = pl.budget;
+        st = pc_compact(w->ctx, &pl.src, w->sel_idx, pl.budget, pl.delta_t, &dst, stream);
         if (st != PC_OK) return st;
     }
-    B.n_tokens = (int32_t)n_sel;
-    A.n_tokens = 0;
-    w->active ^= 1;
-    w->count.assign(budget, budget + stay);
-    w->t_shift += delta_t;
-    if (regime) *regime = left ? PC_WINDOW_SLIDE : PC_WINDOW_PACK;
+    window_commit(w, pl);
+    if (regime) *regime = pl.left ? PC_WINDOW_SLIDE : PC_WINDOW_PACK;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_window_step(pc_window *w, const void *q, const int32_t *q_pos, int32_t n_q, void *out, float *lse,
+                                    int32_t *regime, void *stream) {
+    if (!w) return PC_ERR_INVALID_ARG;
+    WindowPlan pl;
+    pc_status st = window_plan(w, nullptr, &pl);
+    if (st != PC_OK) return st;
+    if (pl.fill || pl.stay == 0) {
+        if (!pl.fill) window_commit(w, pl);
+        pc_cache cache;
+        cache.anchors = w->anchors;
+        cache.history = w->buf[w->active];
+        cache.n_frames = (int32_t)w->count.size();
+        cache.frame_count = w->count.data();
+        st = pc_attend_frame(w->ctx, &cache, nullptr, q, q_pos, n_q, out, lse, stream);
+        if (st != PC_OK) return st;
+        if (regime) *regime = pl.fill ? PC_WINDOW_FILL : (pl.left ? PC_WINDOW_SLIDE : PC_WINDOW_PACK);
+        return PC_OK;
+    }
+    pc_cache dst;
+    dst.anchors = w->anchors;
+    dst.history = w->buf[w->active ^ 1];
+    dst.n_frames = pl.stay;
+    dst.frame_count = pl.budget;
+    st = pc_frame_step(w->ctx, &pl.src, pl.budget, pl.delta_t, &dst, q, q_pos, n_q, w->scores, w->sel_idx, out, lse, stream);
+    if (st != PC_OK) return st;
+    window_commit(w, pl);
+    if (regime) *regime = pl.left ? PC_WINDOW_SLIDE : PC_WINDOW_PACK;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_window_step_host(pc_window *w, const pc_host_window_step *in, const pc_window_step_workspace *ws,
+                                         int32_t *regime, void *stream_) {
+    if (!w || !in || !ws) return PC_ERR_INVALID_ARG;
+    if (!in->q || !in->q_pos || !in->out || in->n_q <= 0 || in->n_frame < 0) return PC_ERR_INVALID_ARG;
+    if (!ws->q || !ws->q_pos || !ws->out) return PC_ERR_INVALID_ARG;
+    if (in->n_frame > 0 && (!in->frame_k || !in->frame_v || !in->frame_pos)) return PC_ERR_INVALID_ARG;
+    if (in->n_q > w->ctx->desc.max_q) return PC_ERR_CAPACITY;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const pc_layer_desc &D = w->ctx->desc;
+    const size_t row = (size_t)D.n_kv_heads * D.head_dim * w->ctx->elem_size;
+    const size_t qrow = (size_t)D.n_q_heads * D.head_dim * w->ctx->elem_size;
+    pc_segment &A = w->buf[w->active];
+    const int n = in->n_frame;
+    if (n > 0) {
+        if ((int64_t)A.n_tokens + n > A.capacity || (int64_t)A.n_tokens + n > w->scratch_capacity) return PC_ERR_CAPACITY;
+        if ((int)w->count.size() + 1 > PC_MAX_FRAMES) return PC_ERR_CAPACITY;
+    }
+    // every argument is checked: from here on work is enqueued.  The finished frame goes straight to the end of the
+    // active history buffer (no staging copy); the queries follow, so their copy overlaps nothing it depends on.
+    if (n > 0) {
+        PC_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(A.k) + (size_t)A.n_tokens * row, in->frame_k, (size_t)n * row, cudaMemcpyHostToDevice, stream));
+        PC_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(A.v) + (size_t)A.n_tokens * row, in->frame_v, (size_t)n * row, cudaMemcpyHostToDevice, stream));
+        PC_CUDA_TRY(cudaMemcpyAsync(A.pos + 4 * (size_t)A.n_tokens, in->frame_pos, (size_t)n * 16, cudaMemcpyHostToDevice, stream));
+        A.n_tokens += n;
+        w->count.push_back(n);
+    }
+    PC_CUDA_TRY(cudaMemcpyAsync(ws->q, in->q, (size_t)in->n_q * qrow, cudaMemcpyHostToDevice, stream));
+    PC_CUDA_TRY(cudaMemcpyAsync(ws->q_pos, in->q_pos, (size_t)in->n_q * 16, cudaMemcpyHostToDevice, stream));
+    pc_status st = pc_window_step(w, ws->q, ws->q_pos, in->n_q, ws->out, nullptr, regime, stream);
+    if (st != PC_OK) return st;
+    PC_CUDA_TRY(cudaMemcpyAsync(in->out, ws->out, (size_t)in->n_q * qrow, cudaMemcpyDeviceToHost, stream));
+    PC_CUDA_TRY(cudaStreamSynchronize(stream));
     return PC_OK;
 }
 

@@ -51,7 +51,8 @@ def test_two_gloo_ranks_shard_layers_and_take_the_slowest_time():
     for rank, gathered, slowest in got:
         assert gathered == [[0, 1, 2, 3], [4, 5, 6, 7]]                # disjoint, seeded per rank
         assert slowest == 15.0                                         # every rank reports the maximum
-    assert bench.job_ms_per_frame(15.0, world) == 7.5                  # two replicas finish two frames per step
+    # a frame's latency is the slowest rank's step; what two replicas add is throughput, reported apart from it
+    assert abs(bench.replica_frames_per_s(15.0, world) - 2000.0 / 15.0) < 1e-9
     assert bench.max_over_ranks(3.0, None) == 3.0
 
 

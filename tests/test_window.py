@@ -353,3 +353,63 @@ def test_window_minimum_quota_matches_reference():
         assert np.array_equal(host(cache.history.k)[:k], ref.k) and np.array_equal(cache.history.pos.cpu().numpy()[:k], ref.pos)
     assert ref.t_shift > 0
     win.close(); ctx.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rebase", [False, True])
+def test_window_step_from_host_buffers_reproduces_the_device_side_window(rebase):
+    """The resident-cache step (frame and queries in pinned host memory, cache on the device, update and attention
+    fused) against the separate device-side calls (append, update, attend) on a second window fed the same frames:
+    regimes, token counts, shift, packed cache and attention output must agree bit for bit through Fill, Pack and
+    Slide, and the output must match the oracle over the reference window's cache."""
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200.device import dev, host, idev, make_ctx, segment
+    from .test_gpu_parity import check_bf16_attention
+
+    cfg = wl.small_bf16(n_frames=6, grid=(9, 15), n_text=37, total=300, kind=wl.HALFLIFE, param=2.0, keep_full=1, seed=21)
+    n, W, total = cfg.frame_tokens, 3, 300
+    L = wl.make_layer(cfg)
+    fr = _frames(cfg, 6, seed=22)
+    cap = total + 2 * n
+    mk = lambda: pc.Segment(torch.full((cap, cfg.n_kv_heads, cfg.head_dim), 5.0, dtype=torch.bfloat16, device="cuda"),
+                            torch.full((cap, cfg.n_kv_heads, cfg.head_dim), 5.0, dtype=torch.bfloat16, device="cuda"),
+                            torch.full((cap, 4), -3, dtype=torch.int32, device="cuda"), 0)
+    anchors = segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype)
+    ctx_a, ctx_b = make_ctx(cfg, max_keys=cfg.n_anchor + cap), make_ctx(cfg, max_keys=cfg.n_anchor + cap)
+    win_a = pc.Window(ctx_a, W, pc.PC_HALFLIFE, 2.0, total, 1, anchors, mk(), mk(), rebase=rebase)
+    win_b = pc.Window(ctx_b, W, pc.PC_HALFLIFE, 2.0, total, 1, anchors, mk(), mk(), rebase=rebase)
+    td = torch.bfloat16
+    pin = lambda a, dt=None: (torch.from_numpy(np.ascontiguousarray(a)).to(dt) if dt else torch.from_numpy(np.ascontiguousarray(a))).pin_memory()
+    ws = {"q": torch.empty((n, cfg.n_q_heads, cfg.head_dim), dtype=td, device="cuda"),
+          "q_pos": torch.empty((n, 4), dtype=torch.int32, device="cuda"),
+          "out": torch.empty((n, cfg.n_q_heads, cfg.head_dim), dtype=td, device="cuda")}
+    out_host = torch.empty((n, cfg.n_q_heads, cfg.head_dim), dtype=td).pin_memory()
+    seen = set()
+    for f in range(6):
+        shift = win_a.state()[1]
+        pos = fr[f]["pos"].copy(); pos[:, 0] -= shift                       # frames arrive in the shifted frame of reference
+        qpos = fr[f + 1]["pos"].copy(); qpos[:, 0] -= shift
+        # (a) device-side calls
+        win_a.append(segment(fr[f]["k"], fr[f]["v"], pos, cfg.dtype))
+        qd, qpd = dev(fr[f + 1]["q"], cfg.dtype), idev(qpos)
+        regime_a = win_a.update(qd, qpd)
+        out_a = pc.pc_attend_frame(ctx_a, win_a.cache(), None, qd, qpd)
+        # (b) one call from host buffers: the frame, the queries and their positions in, the output back
+        regime_b = win_b.step_host({"k": pin(fr[f]["k"], td), "v": pin(fr[f]["v"], td), "pos": pin(pos)},
+                                   pin(fr[f + 1]["q"], td), pin(qpos), out_host, ws)
+        assert regime_a == regime_b and pc.pc_poll_status(ctx_a) == pc.PC_OK and pc.pc_poll_status(ctx_b) == pc.PC_OK
+        seen.add(regime_a)
+        ca, sa, _ = win_a.state(); cb, sb, _ = win_b.state()
+        assert ca.tolist() == cb.tolist() and sa == sb
+        A, B = win_a.cache(), win_b.cache()
+        m = int(ca.sum())
+        assert torch.equal(A.history.k[:m], B.history.k[:m]) and torch.equal(A.history.v[:m], B.history.v[:m])
+        assert torch.equal(A.history.pos[:m], B.history.pos[:m])
+        assert torch.equal(out_a.cpu(), out_host)
+        want = oracle.attend(fr[f + 1]["q"], qpos, [(L.anchor_k, L.anchor_v, L.anchor_pos),
+                                                   (host(B.history.k)[:m], host(B.history.v)[:m], B.history.pos.cpu().numpy()[:m])],
+                             cfg.rope_base)
+        check_bf16_attention(out_host.float().numpy().astype(np.float64), want)
+    assert seen == {pc.PC_WINDOW_FILL, pc.PC_WINDOW_PACK, pc.PC_WINDOW_SLIDE}
+    win_a.close(); win_b.close(); ctx_a.close(); ctx_b.close()
