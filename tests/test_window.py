@@ -413,3 +413,38 @@ def test_window_step_from_host_buffers_reproduces_the_device_side_window(rebase)
         check_bf16_attention(out_host.float().numpy().astype(np.float64), want)
     assert seen == {pc.PC_WINDOW_FILL, pc.PC_WINDOW_PACK, pc.PC_WINDOW_SLIDE}
     win_a.close(); win_b.close(); ctx_a.close(); ctx_b.close()
+
+
+@pytest.mark.gpu
+def test_sliding_window_comparator_is_a_window_of_one_frame():
+    """The sliding-window comparator of the latency curves attends to the anchors and the newest frame.  That is the
+    cache window with W = 1 and room for a whole frame: after every update it must hold exactly the newest frame's
+    rows, and attention over it must give the bits of attention over (anchors, that frame)."""
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200.device import dev, idev, make_ctx, segment
+
+    cfg = wl.small_bf16(n_frames=4, grid=(9, 15), n_text=37, total=10 ** 6, keep_full=0, seed=23)
+    n = cfg.frame_tokens
+    L = wl.make_layer(cfg)
+    fr = _frames(cfg, 4, seed=24)
+    ctx, ctx2 = make_ctx(cfg), make_ctx(cfg)
+    mk = lambda: pc.Segment(torch.zeros((2 * n, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((2 * n, cfg.n_kv_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda"),
+                            torch.zeros((2 * n, 4), dtype=torch.int32, device="cuda"), 0)
+    anchors = segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype)
+    win = pc.Window(ctx, 1, pc.PC_HALFLIFE, 2.0, n, 1, anchors, mk(), mk())           # one frame, kept whole
+    for f in range(4):
+        newest = segment(fr[f]["k"], fr[f]["v"], fr[f]["pos"], cfg.dtype)
+        win.append(newest)
+        q, qp = dev(fr[f + 1]["q"], cfg.dtype), idev(fr[f + 1]["pos"])
+        regime, out = win.step(q, qp)
+        assert regime == (pc.PC_WINDOW_FILL if f == 0 else pc.PC_WINDOW_SLIDE)
+        cache = win.cache()
+        assert win.state()[0].tolist() == [n]
+        assert torch.equal(cache.history.k[:n], newest.k) and torch.equal(cache.history.v[:n], newest.v)
+        assert torch.equal(cache.history.pos[:n], newest.pos)
+        want = pc.pc_attend_frame(ctx2, pc.Cache(anchors, newest, np.array([n], np.int32)), None, q, qp)
+        assert torch.equal(out, want)
+        assert pc.pc_poll_status(ctx) == pc.PC_OK and pc.pc_poll_status(ctx2) == pc.PC_OK
+    win.close(); ctx.close(); ctx2.close()
