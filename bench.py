@@ -306,28 +306,27 @@ def run_cuda(args):
         for k, v in pc.pc_get_timing(ctxs[i % N_LAYERS]).items():
             if v >= 0:
                 acc[k].append(v)
-    # what the event marks add by themselves under the same conditions: the same marks around a selection of eight
-    # tokens enqueued right behind a frame step, so that it meets a busy stream as the step's own kernels do
-    cal = make_ctx(cfg, max_keys=1024, max_q=128)
-    pc.pc_set_timing(cal, True)
-    tiny = pc.Cache(pc.Segment.empty(), pc.Segment(layers[0].cache.history.k, layers[0].cache.history.v,
-                                                   layers[0].cache.history.pos, 8), np.array([8], np.int32))
-    tiny_scores = torch.zeros(8, dtype=torch.float32, device="cuda")
-    tiny_sel = torch.empty(8, dtype=torch.int32, device="cuda")
-    for c in ctxs:
-        pc.pc_set_timing(c, False)
-    pair = []
-    for i in range(40):
-        step(i)
-        pc.pc_score(cal, tiny, None, None, np.array([4], np.int32), scores_override=tiny_scores, sel_idx=tiny_sel, stream=stream)
-        v = pc.pc_get_timing(cal)["select"]
-        if i >= 5 and v >= 0:
-            pair.append(v)
-    cal.close()
-    for c in ctxs:
-        pc.pc_set_timing(c, False)
     kern_ms = {k: (float(np.mean(v)) if v else None) for k, v in acc.items()}
-    pair_ms = float(np.median(pair)) if pair else None
+    # An event between two kernels drains the stream, so the kernel behind it starts from an idle GPU and its span
+    # overstates it.  With the mark in front of a kernel left out, the span of that kernel and the one before it, minus the
+    # earlier kernel's own span, is the kernel's duration as it runs in the untimed step (launch overlapped as there).
+    plan = {"score": (["QPOOL"], "SCORE0", "SCORE", "qpool"), "select": (["SCORE"], "QPOOL", "SELECT", "score"),
+            "pack": (["SELECT", "PACK0"], "SCORE", "PACK", "select"), "attend": (["PACK", "ATT0"], "PACK0", "ATTEND", "pack"),
+            "combine": (["ATTEND"], "ATT0", "COMBINE", "attend")}
+    pipelined = {}
+    for name, (skip, a, b_, before) in plan.items():
+        for c in ctxs:
+            pc.pc_set_timing_skip(c, skip)
+        spans = []
+        for i in range(min(args.steps, 100)):
+            step(i)
+            v = pc.pc_get_span(ctxs[i % N_LAYERS], a, b_)
+            if i >= 3 and v >= 0:
+                spans.append(v)
+        pipelined[name] = (float(np.mean(spans)) - kern_ms[before]) if spans and kern_ms[before] else None
+    for c in ctxs:
+        pc.pc_set_timing_skip(c, [])
+        pc.pc_set_timing(c, False)
 
     # ---- the same frame through the three separate calls (pc_score, pc_compact, pc_attend_frame: eight launches)
     for i in range(3):
@@ -493,12 +492,13 @@ def run_cuda(args):
     score_bytes = cfg.n_src * (row + 16 + 4)
     pack_bytes = n_sel * (5 * row + 32 + 4)          # K and V rows read, K, V and rotated K written, positions, index
     hbm = lambda nbytes, ms: (nbytes / (ms * 1e-3) / 1e9) if ms else None
-    net = lambda ms: (ms - pair_ms) if (ms and pair_ms and ms > pair_ms) else None
 
-    def hbm_entry(nbytes, ms):
-        return {"GBps": hbm(nbytes, ms), "bytes": nbytes, "frac": (hbm(nbytes, ms) or 0) / peaks["hbm_gbs"],
-                "GBps_net_of_event_pair": hbm(nbytes, net(ms)), "frac_net_of_event_pair": (hbm(nbytes, net(ms)) or 0) / peaks["hbm_gbs"]}
+    def hbm_entry(nbytes, ms, ms_pipe):
+        return {"GBps": hbm(nbytes, ms), "bytes": nbytes, "frac": (hbm(nbytes, ms) or 0) / peaks["hbm_gbs"], "ms": ms,
+                "GBps_pipelined": hbm(nbytes, ms_pipe), "frac_pipelined": (hbm(nbytes, ms_pipe) or 0) / peaks["hbm_gbs"],
+                "ms_pipelined": ms_pipe}
     both_ms = (kern_ms["score"] + kern_ms["pack"]) if kern_ms["score"] and kern_ms["pack"] else None
+    both_pipe = (pipelined["score"] + pipelined["pack"]) if pipelined.get("score") and pipelined.get("pack") else None
     stages = {k: (round(v, 5) if v is not None else None) for k, v in kern_ms.items()}
     line = {
         "metric": METRIC, "value": ms_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -526,7 +526,7 @@ def run_cuda(args):
                      "peak_source": f"{peaks['source']} (burst; sustained {peaks['bf16_tflops_sustained']})",
                      "flops_per_launch": flops, "ms_per_launch": att_ms},
         "kernels_ms": stages,
-        "event_pair_ms": pair_ms,
+        "kernels_ms_pipelined": {k: (round(v, 5) if v is not None else None) for k, v in pipelined.items()},
         "separate_calls": {"ms_per_frame": sep_ms, "what": "the same frame through pc_score, pc_compact and pc_attend_frame "
                            "(eight launches: Q read twice, rotary pre-pass over anchors and packed history)"},
         "late4": late,
@@ -539,21 +539,16 @@ def run_cuda(args):
                         "mode": "cache window in the Slide regime (pc_window_append + pc_window_step): append the newest frame, "
                                 "drop the oldest, re-plan, score and re-select from packed + new, pack, attend (same keys attended)"},
         "hbm_kernels": {
-            "score": hbm_entry(score_bytes, kern_ms["score"]),
-            "pack": hbm_entry(pack_bytes, kern_ms["pack"]),
-            "score_plus_pack": hbm_entry(score_bytes + pack_bytes, both_ms) if both_ms else None,
-            "how": "bytes / duration between the library's CUDA event marks around the kernel; 'net_of_event_pair' subtracts "
-                   "event_pair_ms, the same marks around a selection of eight tokens behind a frame step (what the pair and "
-                   "the launch overlap it breaks cost by themselves, plus that near-empty kernel); score_plus_pack subtracts it "
-                   "once per kernel.  A plain streaming read of the score kernel's bytes, timed by an event pair per launch on "
-                   "this GPU, reaches 0.69 of the copy peak (0.90 back to back), so `frac` by itself cannot reach 0.70",
+            "score": hbm_entry(score_bytes, kern_ms["score"], pipelined.get("score")),
+            "pack": hbm_entry(pack_bytes, kern_ms["pack"], pipelined.get("pack")),
+            "score_plus_pack": hbm_entry(score_bytes + pack_bytes, both_ms, both_pipe) if both_ms else None,
+            "how": "bytes / kernel duration.  `frac`: between the library's CUDA event marks around the kernel alone; an event "
+                   "between two kernels drains the stream, so this span also holds a launch from an idle GPU (a plain "
+                   "streaming read of the score kernel's bytes timed that way reaches 0.69 of the copy peak on this GPU, "
+                   "0.90 back to back).  `frac_pipelined`: the mark in front of the kernel left out, the common span of the "
+                   "kernel and the one before it minus that kernel's own span: the duration as in the untimed step",
             "peak": peaks["hbm_gbs"], "peak_source": peaks["source"]},
     }
-    if both_ms and pair_ms:
-        sp = line["hbm_kernels"]["score_plus_pack"]
-        nb = score_bytes + pack_bytes
-        sp["GBps_net_of_event_pair"] = hbm(nb, both_ms - 2 * pair_ms)
-        sp["frac_net_of_event_pair"] = sp["GBps_net_of_event_pair"] / peaks["hbm_gbs"]
     if world == 1 and not args.no_cpu_baseline:
         import oracle
         t0 = time.perf_counter()

@@ -393,6 +393,19 @@ enum { PC_STAGE_QPOOL = 0 /* the query pass */, PC_STAGE_SCORE = 1, PC_STAGE_SEL
        PC_STAGE_ATTEND = 5, PC_STAGE_COMBINE = 6, PC_STAGE_MASS = 7, PC_N_STAGES = 8 };
 pc_status pc_set_timing(pc_ctx *ctx, int32_t on);
 pc_status pc_get_timing(pc_ctx *ctx, float *ms);
+/* The marks themselves, for finer measurements.  An event between two kernels drains the stream: the kernel behind it
+ * starts from an idle GPU instead of overlapping its launch with the tail of the kernel before, so a span of one
+ * kernel overstates it by a few microseconds.  pc_set_timing_skip leaves out the marks whose bits are set (bit i = mark
+ * i); pc_get_span gives the time between any two recorded marks, -1 if either is missing.  With the mark between two
+ * kernels left out, their common span minus the first kernel's own span is the second kernel's duration as it runs in
+ * the untimed sequence.  Marks: a scoring call records SCORE0, QPOOL (after the query pass), SCORE (after the scoring
+ * kernel), SELECT; a pack PACK0, PACK; an attention call ATT0, ROPE (only when a rotary pre-pass ran), ATTEND, COMBINE;
+ * pc_attend_mass MASS0, MASS. */
+enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT = 3, PC_MARK_PACK0 = 4, PC_MARK_PACK = 5,
+       PC_MARK_ATT0 = 6, PC_MARK_ROPE = 7, PC_MARK_ATTEND = 8, PC_MARK_COMBINE = 9, PC_MARK_MASS0 = 10, PC_MARK_MASS = 11,
+       PC_N_MARKS = 12 };
+pc_status pc_set_timing_skip(pc_ctx *ctx, uint32_t mark_mask);
+pc_status pc_get_span(pc_ctx *ctx, int32_t mark_a, int32_t mark_b, float *ms);
 
 const char *pc_status_string(pc_status s);
 

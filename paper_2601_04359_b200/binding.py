@@ -26,7 +26,8 @@ EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact"
            "pc_frame_step_host", "pc_status_string", "pc_score_tokens_static", "pc_set_cluster_merge",
            "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_append_masked", "pc_window_update", "pc_window_cache",
            "pc_window_state", "pc_attend_prepare", "pc_attend_prepared", "pc_attend_mass", "pc_frame_step",
-           "pc_forget_anchors", "pc_set_wait_limit_us", "pc_test_expect_extra_bytes", "pc_window_step", "pc_window_step_host"]
+           "pc_forget_anchors", "pc_set_wait_limit_us", "pc_test_expect_extra_bytes", "pc_window_step", "pc_window_step_host", "pc_set_timing_skip",
+           "pc_get_span"]
 
 
 class pc_layer_desc(C.Structure):
@@ -113,6 +114,8 @@ def load() -> C.CDLL:
     lib.pc_set_cluster_merge.argtypes = [C.c_void_p, C.c_int32]
     lib.pc_set_timing.argtypes = [C.c_void_p, C.c_int32]
     lib.pc_get_timing.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
+    lib.pc_set_timing_skip.argtypes = [C.c_void_p, C.c_uint32]
+    lib.pc_get_span.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_float)]
     lib.pc_frame_step_host.argtypes = [C.c_void_p, C.POINTER(pc_host_frame), C.POINTER(pc_device_workspace),
                                        C.POINTER(pc_budget_params), C.c_int32, C.c_void_p]
     lib.pc_score_tokens_static.argtypes = [C.POINTER(pc_layer_desc), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
@@ -358,6 +361,25 @@ def pc_get_timing(ctx: Context) -> dict:
     ms = (C.c_float * len(STAGES))()
     _check(load().pc_get_timing(ctx.handle, ms), "pc_get_timing")
     return {name: float(ms[i]) for i, name in enumerate(STAGES)}
+
+
+MARKS = {"SCORE0": 0, "QPOOL": 1, "SCORE": 2, "SELECT": 3, "PACK0": 4, "PACK": 5, "ATT0": 6, "ROPE": 7, "ATTEND": 8,
+         "COMBINE": 9, "MASS0": 10, "MASS": 11}
+
+
+def pc_set_timing_skip(ctx: Context, marks: Sequence[str]) -> None:
+    """Leave out the named event marks (see MARKS) from now on."""
+    mask = 0
+    for m in marks:
+        mask |= 1 << MARKS[m]
+    _check(load().pc_set_timing_skip(ctx.handle, mask), "pc_set_timing_skip")
+
+
+def pc_get_span(ctx: Context, a: str, b: str) -> float:
+    """Milliseconds between two recorded marks of the most recent calls, -1 if either is missing."""
+    ms = C.c_float(-1.0)
+    _check(load().pc_get_span(ctx.handle, MARKS[a], MARKS[b], C.byref(ms)), "pc_get_span")
+    return float(ms.value)
 
 
 def pc_frame_step_host(ctx: Context, host: dict, ws_src: Cache, ws_dst: Cache, ws: dict, kind: int, param: float,

@@ -192,6 +192,22 @@ extern "C" pc_status pc_get_timing(pc_ctx *c, float *ms) {
     return PC_OK;
 }
 
+extern "C" pc_status pc_set_timing_skip(pc_ctx *c, uint32_t mark_mask) {
+    if (!c) return PC_ERR_INVALID_ARG;
+    c->ev_skip = mark_mask;
+    c->ev_mask = 0;
+    return PC_OK;
+}
+
+extern "C" pc_status pc_get_span(pc_ctx *c, int32_t a, int32_t b, float *ms) {
+    if (!c || !ms || a < 0 || b < 0 || a >= PC_N_MARKS || b >= PC_N_MARKS) return PC_ERR_INVALID_ARG;
+    *ms = -1.f;
+    if (!((c->ev_mask >> a) & 1u) || !((c->ev_mask >> b) & 1u)) return PC_OK;
+    PC_CUDA_TRY(cudaEventSynchronize(c->ev[b]));
+    PC_CUDA_TRY(cudaEventElapsedTime(ms, c->ev[a], c->ev[b]));
+    return PC_OK;
+}
+
 extern "C" pc_status pc_poll_status(pc_ctx *c, void *stream) {
     if (!c) return PC_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

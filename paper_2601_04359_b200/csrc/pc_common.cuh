@@ -33,11 +33,6 @@ enum {
     PC_WHERE_MASS_WAIT = 10,
 };
 
-// event marks: score call 0-3, pack 4-5, attend 6-9, attention mass 10-11
-enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT = 3, PC_MARK_PACK0 = 4, PC_MARK_PACK = 5,
-       PC_MARK_ATT0 = 6, PC_MARK_ROPE = 7, PC_MARK_ATTEND = 8, PC_MARK_COMBINE = 9, PC_MARK_MASS0 = 10, PC_MARK_MASS = 11,
-       PC_N_MARKS = 12 };
-
 constexpr int PC_MAX_SEGMENTS = 3;
 constexpr int PC_FX_REPLICAS = 8;             // copies of the pooled-query accumulator (see pc_score.cu)
 constexpr int PC_MAX_DEVICES = 64;            // per-device launch state is kept in arrays of this size
@@ -94,6 +89,7 @@ struct pc_ctx {
     // optional per-kernel timing (benchmarks): events at the boundaries of the kernels of each call
     int timing_on;
     unsigned ev_mask;
+    unsigned ev_skip;          // marks that are not recorded (see pc_set_timing_skip)
     cudaEvent_t ev[PC_N_MARKS];
     float *part_o;             // split-KV partial outputs
     float *part_ml;            // split-KV partial (max, sum)
@@ -234,6 +230,10 @@ inline cudaError_t pc_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
 #define PC_LAUNCH(kernel, grid, block, smem, stream, ...) PC_CUDA_TRY(pc_launch(kernel, grid, block, smem, stream, __VA_ARGS__))
 
 inline void pc_mark(pc_ctx *c, int idx, cudaStream_t s) {
+    if ((c->ev_skip >> idx) & 1u) {
+        c->ev_mask &= ~(1u << idx);
+        return;
+    }
     if (c->timing_on && c->ev[idx] && cudaEventRecord(c->ev[idx], s) == cudaSuccess) c->ev_mask |= 1u << idx;
 }
 
