@@ -223,10 +223,12 @@ def test_prepared_attention_equals_attend_frame_over_several_passes(cfg_name):
 
 
 # ------------------------------------------------------------------------------------------- CUDA graph
-def test_frame_step_replays_from_a_cuda_graph():
-    """Three layers' frame steps (score, select, pack, attend: eight kernels each, launched with programmatic
-    dependencies) captured once into a CUDA graph.  A replay must give the bits of the eager calls, also after the
-    inputs were overwritten in place (a new frame's queries and history in the same buffers)."""
+@pytest.mark.parametrize("fused", [False, True])
+def test_frame_step_replays_from_a_cuda_graph(fused):
+    """Three layers' frame steps (score, select, pack, attend, launched with programmatic dependencies: eight kernels
+    each through the three separate calls, six through the fused step with one context per layer) captured once into a
+    CUDA graph.  A replay must give the bits of the eager calls, also after the inputs were overwritten in place (a
+    new frame's queries and history in the same buffers)."""
     cfgs = [wl.small_bf16(n_frames=4, grid=(12, 21), n_text=130, total=500, keep_full=1, seed=30 + i) for i in range(3)]
     Ls = [wl.make_layer(c) for c in cfgs]
     Ds = [DeviceLayer(L) for L in Ls]
@@ -239,11 +241,16 @@ def test_frame_step_replays_from_a_cuda_graph():
     dsts = [D.empty_packed(n_sel) for D in Ds]
     outs = [torch.empty_like(D.q) for D in Ds]
 
+    ctxs = [ctx] + [make_ctx(cfg) for _ in Ds[1:]]
+
     def frame(stream):
-        for D, dst, out in zip(Ds, dsts, outs):
-            pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget, scores=scores, sel_idx=sel, stream=stream)
-            pc.pc_compact(ctx, D.cache, sel, budget, 0, dst, stream=stream)
-            pc.pc_attend_frame(ctx, dst, None, D.q, D.q_pos, out=out, stream=stream)
+        for D, dst, out, c in zip(Ds, dsts, outs, ctxs):
+            if fused:
+                pc.pc_frame_step(c, D.cache, budget, 0, dst, D.q, D.q_pos, scores=scores, sel_idx=sel, out=out, stream=stream)
+            else:
+                pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget, scores=scores, sel_idx=sel, stream=stream)
+                pc.pc_compact(ctx, D.cache, sel, budget, 0, dst, stream=stream)
+                pc.pc_attend_frame(ctx, dst, None, D.q, D.q_pos, out=out, stream=stream)
 
     frame(torch.cuda.current_stream())                              # warm-up: one-time attribute and occupancy queries
     torch.cuda.synchronize()
@@ -255,7 +262,8 @@ def test_frame_step_replays_from_a_cuda_graph():
         o.zero_()
     graph.replay()
     torch.cuda.synchronize()
-    _ok(ctx)
+    for c in ctxs:
+        _ok(c)
     for o, e in zip(outs, eager):
         assert torch.equal(o, e)
     want = oracle.attend(Ls[1].q, Ls[1].q_pos, [(Ls[1].anchor_k, Ls[1].anchor_v, Ls[1].anchor_pos),
@@ -276,11 +284,13 @@ def test_frame_step_replays_from_a_cuda_graph():
     replayed = [o.clone() for o in outs]
     frame(torch.cuda.current_stream())
     torch.cuda.synchronize()
-    _ok(ctx)
+    for c in ctxs:
+        _ok(c)
     for o, e in zip(outs, replayed):
         assert torch.equal(o, e)
     assert not torch.equal(replayed[0], eager[0])
-    ctx.close()
+    for c in ctxs:
+        c.close()
 
 
 # ------------------------------------------------------------------------------------------- select
