@@ -148,3 +148,40 @@ def test_fused_step_at_the_benchmark_size_matches_the_separate_calls():
         assert _same(scores, scores0) and _same(sel[:n_sel], sel0[:n_sel]) and _same(dst.history.k, dst0.history.k)
         assert _same(dst.history.pos, dst0.history.pos) and _same(out, out0) and _same(lse, lse0)
     ref_ctx.close(); ctx.close()
+
+
+def test_fused_step_rejects_bad_arguments_before_enqueueing_anything():
+    """Host-detectable errors return at once: a destination that is too small, a null output, too many queries for
+    the context, a budget above a frame's tokens; none of them leaves a device-side status or touches the outputs."""
+    cfg = wl.small_bf16(n_frames=3, grid=(8, 9), total=100, seed=42)
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    b = cfg.budget
+    budget = pc.pc_plan_budget(b.kind, b.param, b.total, b.keep_full, L.frame_count)
+    n_sel = int(budget.sum())
+    ctx = make_ctx(cfg)
+    out = torch.full_like(D.q, 7.0)
+    small = D.empty_packed(n_sel - 1)
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_frame_step(ctx, D.cache, budget, 0, small, D.q, D.q_pos, out=out)
+    assert e.value.status == pc.PC_ERR_CAPACITY
+    dst = D.empty_packed(n_sel, poison=3.0)
+    over = budget.copy(); over[0] = L.frame_count[0] + 1
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_frame_step(ctx, D.cache, over, 0, D.empty_packed(int(over.sum())), D.q, D.q_pos, out=out)
+    assert e.value.status == pc.PC_ERR_BUDGET
+    tight = make_ctx(cfg, max_q=cfg.n_q - 1)
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_frame_step(tight, D.cache, budget, 0, dst, D.q, D.q_pos, out=out)
+    assert e.value.status == pc.PC_ERR_CAPACITY
+    lib = pc.load()
+    import ctypes as C
+    cs, cd = D.cache.c(), dst.c()
+    bud = np.ascontiguousarray(budget, np.int32)
+    st = lib.pc_frame_step(ctx.handle, C.byref(cs), bud.ctypes.data_as(C.POINTER(C.c_int32)), 0, C.byref(cd), D.q.data_ptr(),
+                           D.q_pos.data_ptr(), cfg.n_q, None, None, None, None, None)          # no output buffer
+    assert st == pc.PC_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert pc.pc_poll_status(ctx) == pc.PC_OK and pc.pc_poll_status(tight) == pc.PC_OK
+    assert (out == 7.0).all() and (host(dst.history.k) == 3.0).all()
+    ctx.close(); tight.close()
