@@ -486,7 +486,10 @@ def run_cuda(args):
     peaks = _peaks()
     n_keys = cfg.n_anchor + n_sel
     flops = 4.0 * cfg.n_q * n_keys * cfg.head_dim * cfg.n_q_heads
-    att_ms = kern_ms["attend"]
+    # the attention kernel's duration as it runs in the untimed step (the mark in front of it left out); its span between
+    # two marks of its own, which also holds a launch from an idle GPU, rides along
+    att_span_ms = kern_ms["attend"]
+    att_ms = pipelined.get("attend") or att_span_ms
     achieved = flops / (att_ms * 1e-3) / 1e12
     row = cfg.n_kv_heads * cfg.head_dim * 2
     score_bytes = cfg.n_src * (row + 16 + 4)
@@ -524,7 +527,13 @@ def run_cuda(args):
         "roofline": {"kernel": "k_attend_tc", "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
                      "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": attend_traffic(),
                      "peak_source": f"{peaks['source']} (burst; sustained {peaks['bf16_tflops_sustained']})",
-                     "flops_per_launch": flops, "ms_per_launch": att_ms},
+                     "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                     "flops_per_launch": flops, "ms_per_launch": att_ms, "ms_per_launch_single_kernel_span": att_span_ms,
+                     "frac_by_single_kernel_span": flops / (att_span_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                     "how": "flops / the kernel's mean duration by CUDA events on the launching stream: the event mark in front "
+                            "of the kernel left out, span of the pack kernel and this one minus the pack kernel's own span (the "
+                            "duration as in the untimed step); the kernel runs inside a long power-capped step, for which the "
+                            "sustained peak is the like-for-like denominator, the burst peak the conservative one used for frac"},
         "kernels_ms": stages,
         "kernels_ms_pipelined": {k: (round(v, 5) if v is not None else None) for k, v in pipelined.items()},
         "separate_calls": {"ms_per_frame": sep_ms, "what": "the same frame through pc_score, pc_compact and pc_attend_frame "
