@@ -285,14 +285,30 @@ extern "C" pc_status pc_window_step_host(pc_window *w, const pc_host_window_step
         if ((int64_t)A.n_tokens + n > A.capacity || (int64_t)A.n_tokens + n > w->scratch_capacity) return PC_ERR_CAPACITY;
         if ((int)w->count.size() + 1 > PC_MAX_FRAMES) return PC_ERR_CAPACITY;
     }
-    // every argument is checked: from here on work is enqueued.  The finished frame goes straight to the end of the
-    // active history buffer (no staging copy); the queries follow, so their copy overlaps nothing it depends on.
+    // The plan of the step is tried on the window as it will be with the frame appended (host arithmetic only); if it
+    // cannot be made (budget, capacity of the other buffer), the window is left as it was and nothing is enqueued.
     if (n > 0) {
-        PC_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(A.k) + (size_t)A.n_tokens * row, in->frame_k, (size_t)n * row, cudaMemcpyHostToDevice, stream));
-        PC_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(A.v) + (size_t)A.n_tokens * row, in->frame_v, (size_t)n * row, cudaMemcpyHostToDevice, stream));
-        PC_CUDA_TRY(cudaMemcpyAsync(A.pos + 4 * (size_t)A.n_tokens, in->frame_pos, (size_t)n * 16, cudaMemcpyHostToDevice, stream));
         A.n_tokens += n;
         w->count.push_back(n);
+    }
+    {
+        WindowPlan trial;
+        const pc_status st = window_plan(w, nullptr, &trial);
+        if (st != PC_OK) {
+            if (n > 0) {
+                A.n_tokens -= n;
+                w->count.pop_back();
+            }
+            return st;
+        }
+    }
+    // every argument is checked: from here on work is enqueued.  The finished frame goes straight to the end of the
+    // active history buffer (no staging copy); the queries follow.
+    if (n > 0) {
+        const size_t at = (size_t)(A.n_tokens - n);
+        PC_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(A.k) + at * row, in->frame_k, (size_t)n * row, cudaMemcpyHostToDevice, stream));
+        PC_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(A.v) + at * row, in->frame_v, (size_t)n * row, cudaMemcpyHostToDevice, stream));
+        PC_CUDA_TRY(cudaMemcpyAsync(A.pos + 4 * at, in->frame_pos, (size_t)n * 16, cudaMemcpyHostToDevice, stream));
     }
     PC_CUDA_TRY(cudaMemcpyAsync(ws->q, in->q, (size_t)in->n_q * qrow, cudaMemcpyHostToDevice, stream));
     PC_CUDA_TRY(cudaMemcpyAsync(ws->q_pos, in->q_pos, (size_t)in->n_q * 16, cudaMemcpyHostToDevice, stream));

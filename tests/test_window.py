@@ -448,3 +448,43 @@ def test_sliding_window_comparator_is_a_window_of_one_frame():
         assert torch.equal(out, want)
         assert pc.pc_poll_status(ctx) == pc.PC_OK and pc.pc_poll_status(ctx2) == pc.PC_OK
     win.close(); ctx.close(); ctx2.close()
+
+
+@pytest.mark.gpu
+def test_window_step_from_host_buffers_leaves_the_window_alone_when_the_plan_fails():
+    """The step's plan is tried before anything is enqueued: when it cannot be made (here the two frames that are to be
+    kept whole exceed the token budget), the call returns the error, the frame is not appended and no buffer is touched;
+    the window goes on working."""
+    import torch
+    from paper_2601_04359_b200 import binding as pc
+    from paper_2601_04359_b200.device import make_ctx, segment
+
+    cfg = wl.small_bf16(n_frames=3, grid=(8, 9), n_text=37, total=100, keep_full=2, seed=25)
+    n = cfg.frame_tokens                                                     # 72 tokens per frame, budget 100, 2 frames whole
+    L = wl.make_layer(cfg)
+    fr = _frames(cfg, 3, seed=26)
+    ctx = make_ctx(cfg)
+    td = torch.bfloat16
+    mk = lambda: pc.Segment(torch.full((4 * n, cfg.n_kv_heads, cfg.head_dim), 5.0, dtype=td, device="cuda"),
+                            torch.full((4 * n, cfg.n_kv_heads, cfg.head_dim), 5.0, dtype=td, device="cuda"),
+                            torch.full((4 * n, 4), -3, dtype=torch.int32, device="cuda"), 0)
+    a, b = mk(), mk()
+    win = pc.Window(ctx, 4, pc.PC_HALFLIFE, 2.0, 100, 2, segment(L.anchor_k, L.anchor_v, L.anchor_pos, cfg.dtype), a, b)
+    pin = lambda x, dt=None: (torch.from_numpy(np.ascontiguousarray(x)).to(dt) if dt else torch.from_numpy(np.ascontiguousarray(x))).pin_memory()
+    ws = {"q": torch.empty((n, cfg.n_q_heads, cfg.head_dim), dtype=td, device="cuda"),
+          "q_pos": torch.empty((n, 4), dtype=torch.int32, device="cuda"),
+          "out": torch.empty((n, cfg.n_q_heads, cfg.head_dim), dtype=td, device="cuda")}
+    out_host = torch.full((n, cfg.n_q_heads, cfg.head_dim), 9.0, dtype=td).pin_memory()
+    frame = lambda f, m=n: {"k": pin(fr[f]["k"][:m], td), "v": pin(fr[f]["v"][:m], td), "pos": pin(fr[f]["pos"][:m])}
+    assert win.step_host(frame(0), pin(fr[1]["q"], td), pin(fr[1]["pos"]), out_host, ws) == pc.PC_WINDOW_FILL
+    first_out = out_host.clone()
+    before = (win.state()[0].tolist(), a.k.clone(), b.k.clone())
+    with pytest.raises(pc.PackCacheError) as e:                             # 72 + 72 kept whole > 100
+        win.step_host(frame(1), pin(fr[2]["q"], td), pin(fr[2]["pos"]), out_host, ws)
+    assert e.value.status == pc.PC_ERR_BUDGET
+    torch.cuda.synchronize()
+    assert win.state()[0].tolist() == before[0] == [n] and torch.equal(a.k, before[1]) and torch.equal(b.k, before[2])
+    assert torch.equal(out_host, first_out) and pc.pc_poll_status(ctx) == pc.PC_OK
+    assert win.step_host(frame(1, 20), pin(fr[2]["q"], td), pin(fr[2]["pos"]), out_host, ws) == pc.PC_WINDOW_FILL     # 92 fit
+    assert win.state()[0].tolist() == [n, 20] and pc.pc_poll_status(ctx) == pc.PC_OK
+    win.close(); ctx.close()
