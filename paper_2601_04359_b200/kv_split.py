@@ -8,8 +8,8 @@ numbers and therefore keep the same tokens; pack and attention are then rank-loc
 the concatenation of the ranks' outputs.  This module is argument marshalling and one collective; scoring, selection,
 packing and attention run in the library's kernels.
 
-Not measured on several GPUs (this build only ever had one): the logic is covered by a world-size-2 ``gloo`` test on
-CPU and by a one-GPU test that runs the ranks' slices one after the other and adds their scores.
+Not measured on several GPUs: the logic is covered by a world-size-2 ``gloo`` test on CPU and by a one-GPU test that
+runs the ranks' slices one after the other and adds their scores.
 """
 from __future__ import annotations
 

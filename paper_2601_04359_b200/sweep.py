@@ -12,7 +12,7 @@ cumulative curve of Fig. 1; TOTAL and LAST of Tab. 2 are the last total and the 
 the budget x decay grid of the 28-layer configuration (budget 10 / 25 / 50 / 100 % of the history, decay linear or
 half-life 2 / 4 / 8) over the depth of the generation: per-frame time at sampled depths, the total over all 47 frames
 and the last four.  `--layers` only scales a per-layer time to a stack of identical layers; `--stack N` times one frame
-through N distinct layers.  `--markdown` prints the tables in the form the benchmark spec keeps.
+through N distinct layers.  `--markdown` also prints the two tables as markdown.
 """
 from __future__ import annotations
 
