@@ -197,12 +197,12 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------------------------- CUDA arm
-def attend_traffic():
+def attend_traffic(rec=None, src=None):
     """DRAM bytes of one k_attend_tc launch from the ncu capture recorded under profiles/, or None when the kernel's
     source has changed since that capture (the record carries the git blob id of the file it was taken on)."""
     import hashlib
-    rec = os.path.join(ROOT, "profiles", "attend_dram_traffic.json")
-    src = os.path.join(ROOT, "paper_2601_04359_b200", "csrc", "pc_attend_tc.cu")
+    rec = rec or os.path.join(ROOT, "profiles", "attend_dram_traffic.json")
+    src = src or os.path.join(ROOT, "paper_2601_04359_b200", "csrc", "pc_attend_tc.cu")
     try:
         r = json.load(open(rec))
         data = open(src, "rb").read()

@@ -128,3 +128,22 @@ def test_kv_head_split_ranks_agree_on_the_selection():
     assert kv_split.head_slice(1, 2, 24, 8) == (4, 8, 12, 24)
     with pytest.raises(ValueError):
         kv_split.head_slice(0, 3, 24, 8)
+
+
+def test_recorded_dram_traffic_is_dropped_when_the_kernel_source_changes(tmp_path):
+    """The bench line's roofline.traffic comes from a record that names the git blob of the attention kernel's source:
+    it is reported while that file is unchanged and becomes null as soon as the file differs."""
+    src = os.path.join(ROOT, "paper_2601_04359_b200", "csrc", "pc_attend_tc.cu")
+    rec = json.load(open(os.path.join(ROOT, "profiles", "attend_dram_traffic.json")))
+    assert bench.attend_traffic() in (None, rec["dram_bytes_read"] + rec["dram_bytes_write"])
+    changed = tmp_path / "pc_attend_tc.cu"
+    changed.write_bytes(open(src, "rb").read() + b"\n// touched\n")
+    assert bench.attend_traffic(src=str(changed)) is None
+    same = tmp_path / "same.cu"
+    same.write_bytes(b"x")
+    import hashlib
+    fake = tmp_path / "rec.json"
+    fake.write_text(json.dumps({"dram_bytes_read": 5, "dram_bytes_write": 7,
+                                "source_blob": hashlib.sha1(b"blob 1\0x").hexdigest()}))
+    assert bench.attend_traffic(rec=str(fake), src=str(same)) == 12
+    assert bench.attend_traffic(rec=str(tmp_path / "missing.json"), src=str(same)) is None
