@@ -328,6 +328,21 @@ def run_cuda(args):
         pc.pc_set_timing_skip(c, [])
         pc.pc_set_timing(c, False)
 
+    # ---- yardstick for the HBM-bound kernels: a kernel that only streams the history keys the scoring kernel reads (same
+    # access pattern, no arithmetic), by an event pair per launch and back to back, over the rotating layers
+    probe_out = torch.empty(cfg.n_src, dtype=torch.int32, device="cuda")
+    stream_fn = lambda i: pc.pc_probe_stream_read(layers[i % N_LAYERS].cache.history.k, probe_out, stream=stream)
+    for i in range(4):
+        stream_fn(i)
+    singles = []
+    for i in range(40):
+        torch.cuda.synchronize()
+        e0.record(stream); stream_fn(i); e1.record(stream)
+        torch.cuda.synchronize()
+        singles.append(e0.elapsed_time(e1))
+    stream_single_ms = float(np.median(singles))
+    stream_b2b_ms = timed(stream_fn, 100)
+
     # ---- the same frame through the three separate calls (pc_score, pc_compact, pc_attend_frame: eight launches)
     for i in range(3):
         step_separate(i)
@@ -552,10 +567,15 @@ def run_cuda(args):
             "pack": hbm_entry(pack_bytes, kern_ms["pack"], pipelined.get("pack")),
             "score_plus_pack": hbm_entry(score_bytes + pack_bytes, both_ms, both_pipe) if both_ms else None,
             "how": "bytes / kernel duration.  `frac`: between the library's CUDA event marks around the kernel alone; an event "
-                   "between two kernels drains the stream, so this span also holds a launch from an idle GPU (a plain "
-                   "streaming read of the score kernel's bytes timed that way reaches 0.69 of the copy peak on this GPU, "
-                   "0.90 back to back).  `frac_pipelined`: the mark in front of the kernel left out, the common span of the "
+                   "between two kernels drains the stream, so this span also holds a launch from an idle GPU (see "
+                   "stream_read_yardstick for what a plain streaming read of the score kernel's bytes reaches that way).  `frac_pipelined`: the mark in front of the kernel left out, the common span of the "
                    "kernel and the one before it minus that kernel's own span: the duration as in the untimed step",
+            "stream_read_yardstick": {
+                "bytes": cfg.n_src * row,
+                "single_launch": {"ms": stream_single_ms, "frac": hbm(cfg.n_src * row, stream_single_ms) / peaks["hbm_gbs"]},
+                "back_to_back": {"ms": stream_b2b_ms, "frac": hbm(cfg.n_src * row, stream_b2b_ms) / peaks["hbm_gbs"]},
+                "what": "pc_probe_stream_read over the same history keys: what a kernel that only streams the scoring kernel's "
+                        "bytes reaches here, timed by an event pair around one launch from an idle GPU and back to back"},
             "peak": peaks["hbm_gbs"], "peak_source": peaks["source"]},
     }
     if world == 1 and not args.no_cpu_baseline:

@@ -407,6 +407,13 @@ enum { PC_MARK_SCORE0 = 0, PC_MARK_QPOOL = 1, PC_MARK_SCORE = 2, PC_MARK_SELECT 
 pc_status pc_set_timing_skip(pc_ctx *ctx, uint32_t mark_mask);
 pc_status pc_get_span(pc_ctx *ctx, int32_t mark_a, int32_t mark_b, float *ms);
 
+/* Measurement support (the paper has no counterpart): streams n_rows rows of row_bytes (a multiple of 512) from device
+ * memory with the access pattern of the scoring kernel — 16-byte streaming loads, two rows per warp in flight — and
+ * writes one 32-bit word per row; no arithmetic beyond an xor.  Timed beside the scoring and pack kernels it says what
+ * a kernel that only moves those bytes reaches on the GPU at hand, by an event pair per launch and back to back.
+ *   src device [n_rows][row_bytes]; out device [n_rows] uint32.  Errors: PC_ERR_INVALID_ARG, PC_ERR_CUDA. */
+pc_status pc_probe_stream_read(const void *src, int32_t n_rows, int32_t row_bytes, uint32_t *out, void *stream);
+
 const char *pc_status_string(pc_status s);
 
 #ifdef __cplusplus

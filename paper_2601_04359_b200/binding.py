@@ -27,7 +27,7 @@ EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact"
            "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_append_masked", "pc_window_update", "pc_window_cache",
            "pc_window_state", "pc_attend_prepare", "pc_attend_prepared", "pc_attend_mass", "pc_frame_step",
            "pc_forget_anchors", "pc_set_wait_limit_us", "pc_test_expect_extra_bytes", "pc_window_step", "pc_window_step_host", "pc_set_timing_skip",
-           "pc_get_span"]
+           "pc_get_span", "pc_probe_stream_read"]
 
 
 class pc_layer_desc(C.Structure):
@@ -116,6 +116,7 @@ def load() -> C.CDLL:
     lib.pc_get_timing.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
     lib.pc_set_timing_skip.argtypes = [C.c_void_p, C.c_uint32]
     lib.pc_get_span.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_float)]
+    lib.pc_probe_stream_read.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     lib.pc_frame_step_host.argtypes = [C.c_void_p, C.POINTER(pc_host_frame), C.POINTER(pc_device_workspace),
                                        C.POINTER(pc_budget_params), C.c_int32, C.c_void_p]
     lib.pc_score_tokens_static.argtypes = [C.POINTER(pc_layer_desc), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
@@ -380,6 +381,13 @@ def pc_get_span(ctx: Context, a: str, b: str) -> float:
     ms = C.c_float(-1.0)
     _check(load().pc_get_span(ctx.handle, MARKS[a], MARKS[b], C.byref(ms)), "pc_get_span")
     return float(ms.value)
+
+
+def pc_probe_stream_read(rows: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """Stream the rows of a [n][...] tensor from device memory (one 32-bit word out per row): a bandwidth yardstick."""
+    n = rows.shape[0]
+    row_bytes = rows[0].numel() * rows.element_size()
+    _check(load().pc_probe_stream_read(_ptr(rows), n, row_bytes, _ptr(out), _stream(stream)), "pc_probe_stream_read")
 
 
 def pc_frame_step_host(ctx: Context, host: dict, ws_src: Cache, ws_dst: Cache, ws: dict, kind: int, param: float,
