@@ -185,3 +185,28 @@ def test_fused_step_rejects_bad_arguments_before_enqueueing_anything():
     assert pc.pc_poll_status(ctx) == pc.PC_OK and pc.pc_poll_status(tight) == pc.PC_OK
     assert (out == 7.0).all() and (host(dst.history.k) == 3.0).all()
     ctx.close(); tight.close()
+
+
+def test_attention_mass_after_a_fused_step_equals_the_mass_after_the_separate_calls():
+    """pc_attend_mass reads the rotated keys and queries the last attention call left in the context; after a fused step
+    those were written by the query pass, the pack kernel and the kept anchor keys, and must serve it just the same."""
+    cfg = wl.small_bf16(n_frames=3, grid=(11, 13), n_text=130, total=260, seed=43)
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    b = cfg.budget
+    budget = pc.pc_plan_budget(b.kind, b.param, b.total, b.keep_full, L.frame_count)
+    n_sel = int(budget.sum())
+    n_keys = cfg.n_anchor + n_sel
+    ref_ctx, ctx = make_ctx(cfg), make_ctx(cfg)
+    _, sel0, dst0, _, lse0 = _separate(ref_ctx, D, budget, 0, n_sel)
+    want = pc.pc_attend_mass(ref_ctx, lse0, n_keys).clone()
+    for step in range(2):
+        dst = D.empty_packed(n_sel + 3)
+        _, _, _, lse = pc.pc_frame_step(ctx, D.cache, budget, 0, dst, D.q, D.q_pos, want_lse=True)
+        got = pc.pc_attend_mass(ctx, lse, n_keys)
+        assert pc.pc_poll_status(ctx) == pc.PC_OK and _same(got, want)
+    sel_np = sel0.cpu().numpy()[:n_sel]
+    wk, _, wp = oracle.pack(L.hist_k, L.hist_v, L.hist_pos, sel_np, 0)
+    ref = oracle.attend_mass(L.q, L.q_pos, [(L.anchor_k, L.anchor_pos), (wk, wp)], cfg.rope_base)
+    assert (np.abs(host(got).astype(np.float64) - ref) <= 5e-3 * ref + 1e-3 / n_keys).all()
+    ref_ctx.close(); ctx.close()
