@@ -13,6 +13,7 @@
 #include <algorithm>
 
 #include "pc_common.cuh"
+#include "pc_select.cuh"
 
 namespace {
 
@@ -280,125 +281,20 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict_
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Select.  One block per frame.  Scores map to 32-bit keys whose unsigned order is the score order (-0 folded onto
-// +0).  An 8-bit-digit radix descent finds the key T of the budget-th best token and how many keys beat it; a final
-// ordered sweep keeps every key > T and the lowest-index (budget - beaten) keys == T, writing ascending indices.
+// Select.  One block per frame runs the block-level selection of pc_select.cuh and writes the kept tokens' indices in
+// ascending order.
 // ---------------------------------------------------------------------------------------------------------
-struct FrameTab { int4 f[PC_MAX_FRAMES]; };   // (first token, tokens, budget, output offset)
-
-__device__ __forceinline__ uint32_t score_key(float s) {
-    uint32_t u = __float_as_uint(s);
-    if ((u << 1) == 0) u = 0;                       // -0 -> +0
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 constexpr int SEL_THREADS = 512;
-constexpr int SEL_CACHE = 4096;   // keys of a frame kept in shared memory; longer frames re-read the rest from global
-
-// Exclusive block scan of a small per-thread value; total = sum over the block.
-__device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int &total) {
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += n;
-    }
-    __syncthreads();                                // warp_sums may still be read from the previous call
-    if (lane == 31) warp_sums[w] = inc;
-    __syncthreads();
-    int base = 0, tot = 0;
-#pragma unroll
-    for (int i = 0; i < SEL_THREADS / 32; ++i) {
-        int s = warp_sums[i];
-        if (i < w) base += s;
-        tot += s;
-    }
-    total = tot;
-    return base + inc - v;
-}
 
 __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict__ scores, const __grid_constant__ FrameTab tab,
                                                        int32_t *__restrict__ sel_idx, int32_t *status) {
     pc_grid_dep_launch();
     pc_grid_dep_wait();
-    __shared__ uint32_t keys[SEL_CACHE];
-    __shared__ int hist[256];
-    __shared__ int warp_sums[SEL_THREADS / 32];
-    __shared__ uint32_t sh_prefix;
-    __shared__ int sh_want;
+    __shared__ SelectShared<SEL_THREADS> sm;
     const int4 fr = tab.f[blockIdx.x];
-    const int first = fr.x, n = fr.y, budget = fr.z, out0 = fr.w;
-    if (budget <= 0 || n <= 0) return;
-    const float *s = scores + first;
-    const int lane = threadIdx.x & 31;
-
-    for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
-        const float v = s[j];
-        if (v != v) pc_flag(status, PC_ERR_INVALID_ARG, PC_WHERE_SELECT_NAN);
-        if (j < SEL_CACHE) keys[j] = score_key(v);
-    }
-    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
-    __syncthreads();
-    auto key_at = [&](int j) { return j < SEL_CACHE ? keys[j] : score_key(s[j]); };
-
-    uint32_t prefix = 0, mask = 0;
-    int want = budget;                               // rank, among keys matching the prefix, of the threshold key
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int j = threadIdx.x; j < n; j += SEL_THREADS) {
-            const uint32_t key = key_at(j);
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
-        }
-        __syncthreads();
-        if (threadIdx.x < 32) {
-            // lane l owns digits 255 - 8l down to 248 - 8l; an inclusive scan over lanes counts keys from the top digit down
-            int c[8], mine = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { c[i] = hist[255 - 8 * lane - i]; mine += c[i]; }
-            int inc = mine;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int v = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc += v;
-            }
-            const int before = inc - mine;
-            if (before < want && want <= inc) {      // exactly one lane: the threshold digit is among its eight
-                int w = want - before, digit = 255 - 8 * lane;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (c[i] >= w) { digit = 255 - 8 * lane - i; break; }
-                    w -= c[i];
-                }
-                sh_prefix = prefix | ((uint32_t)digit << shift);
-                sh_want = w;
-            }
-        }
-        __syncthreads();
-        prefix = sh_prefix;
-        want = sh_want;
-        mask |= 255u << shift;
-        if (threadIdx.x < 256) hist[threadIdx.x] = 0;
-        __syncthreads();
-    }
-    // prefix is now the threshold key T: every key above it is kept, and the `want` lowest-index keys equal to it.
-    // One scan per 512 keys carries both counts (keys above T in the low half, keys equal to T in the high half).
-    const uint32_t T = prefix;
-    int gt_seen = 0, eq_seen = 0;
-    for (int j0 = 0; j0 < n; j0 += SEL_THREADS) {
-        const int j = j0 + threadIdx.x;
-        const bool in = j < n;
-        const uint32_t key = in ? key_at(j) : 0u;
-        const int is_gt = in && key > T, is_eq = in && key == T;
-        int total;
-        const int ex = block_exclusive_scan(is_gt | (is_eq << 16), warp_sums, total);
-        const int gt_before = gt_seen + (ex & 0xFFFF), eq_before = eq_seen + (ex >> 16);
-        if (is_gt || (is_eq && eq_before < want)) {
-            const int at = gt_before + min(eq_before, want);
-            if (at < budget) sel_idx[out0 + at] = first + j;
-        }
-        gt_seen += total & 0xFFFF;
-        eq_seen += total >> 16;
-    }
+    if (fr.z <= 0 || fr.y <= 0) return;
+    const int out0 = fr.w;
+    frame_select<SEL_THREADS>(scores, fr, sm, status, [&](int at, int idx) { sel_idx[out0 + at] = idx; });
 }
 
 // Enqueue the query pass and the scoring kernel on caller-given scratch (a context's, or the library's fixed array).
