@@ -76,6 +76,59 @@ def test_random_shapes_against_the_oracle(seed):
         ctx.close()
 
 
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_random_fused_steps_against_the_separate_calls_and_the_oracle(seed):
+    """pc_frame_step on random shapes: the bits of pc_score -> pc_compact -> pc_attend_frame (scores, indices, packed
+    rows, output, log-sum-exp), twice in a row (the second step finds the anchors' rotated keys kept), with and without
+    anchors, with and without a rebase; the output also against the oracle's attention over the oracle's pack of the
+    selected rows."""
+    rng = np.random.default_rng(100 + seed)
+    same = lambda a, b: torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+    for case in range(5):
+        hq, hkv = HEADS[rng.integers(len(HEADS))]
+        grid = (int(rng.integers(1, 20)), int(rng.integers(1, 30)))
+        n_frames, n_text = int(rng.integers(1, 7)), int(rng.integers(1, 200))
+        n = grid[0] * grid[1]
+        total = int(rng.integers(0, n_frames * n + 1))
+        keep_full = int(rng.integers(0, 3)) if total >= 2 * n else 0
+        kind = list(DECAY)[rng.integers(4)]
+        delta_t = int(rng.integers(0, 2)) * 4
+        anchors = bool(rng.integers(4))                      # one case in four has no anchors
+        cfg = replace(wl.small_bf16(n_frames=n_frames, grid=grid, n_text=n_text, total=total, kind=kind, param=DECAY[kind],
+                                    keep_full=min(keep_full, n_frames), seed=3000 + 10 * seed + case), n_q_heads=hq, n_kv_heads=hkv)
+        what = f"{cfg.name} heads {hq}/{hkv} text {n_text} budget {total}/{keep_full} decay {kind} delta_t {delta_t} anchors {anchors}"
+        L = wl.make_layer(cfg)
+        if not anchors:
+            L.anchor_k, L.anchor_v, L.anchor_pos = L.anchor_k[:0], L.anchor_v[:0], L.anchor_pos[:0]
+        D = DeviceLayer(L)
+        b = cfg.budget
+        budget = pc.pc_plan_budget(b.kind, b.param, b.total, b.keep_full, L.frame_count)
+        n_sel = int(budget.sum())
+        if n_sel == 0 and not anchors:
+            continue                                         # nothing to attend to: an argument error, covered elsewhere
+        ref_ctx, ctx = make_ctx(cfg), make_ctx(cfg)
+        scores0, sel0 = pc.pc_score(ref_ctx, D.cache, D.q, D.q_pos, budget)
+        dst0 = D.empty_packed(n_sel + 3, poison=5.0)
+        pc.pc_compact(ref_ctx, D.cache, sel0, budget, delta_t, dst0)
+        out0, lse0 = pc.pc_attend_frame(ref_ctx, dst0, None, D.q, D.q_pos, want_lse=True)
+        assert pc.pc_poll_status(ref_ctx) == pc.PC_OK, what
+        for step in range(2):
+            dst = D.empty_packed(n_sel + 3, poison=5.0)
+            out, scores, sel, lse = pc.pc_frame_step(ctx, D.cache, budget, delta_t, dst, D.q, D.q_pos, want_lse=True)
+            assert pc.pc_poll_status(ctx) == pc.PC_OK, what
+            assert same(scores[:cfg.n_src], scores0[:cfg.n_src]) and same(sel[:n_sel], sel0[:n_sel]), what
+            assert same(dst.history.k, dst0.history.k) and same(dst.history.v, dst0.history.v), what
+            assert same(dst.history.pos, dst0.history.pos) and dst.history.n_tokens == n_sel, what
+            assert same(out, out0) and same(lse, lse0), what
+        sel_np = sel.cpu().numpy()[:n_sel]
+        wk, wv, wp = oracle.pack(L.hist_k, L.hist_v, L.hist_pos, sel_np, delta_t)
+        segs = [s for s in [(L.anchor_k, L.anchor_v, L.anchor_pos), (wk, wv, wp)] if len(s[0])]
+        want, want_lse = oracle.attend(L.q, L.q_pos, segs, cfg.rope_base, want_lse=True)
+        assert np.abs(host(out).astype(np.float64) - want).max() <= 2e-2, what
+        assert np.abs(host(lse) - want_lse).max() <= 2e-2, what
+        ref_ctx.close(); ctx.close()
+
+
 @pytest.mark.parametrize("seed", [0, 1, 2])
 def test_random_cache_windows_against_the_reference(seed):
     """Seeded random cache-window runs (window length 1-6, all decay kernels, budgets from a few tokens to several frames,
