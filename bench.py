@@ -343,6 +343,12 @@ def run_cuda(args):
     stream_single_ms = float(np.median(singles))
     stream_b2b_ms = timed(stream_fn, 100)
 
+    # ---- yardstick for the attention kernel: its tensor-core issue stream alone (no loads, no softmax), one CTA per SM, a few
+    # milliseconds per form: cycles per 128 x 128 x 16 multiply-add and the SM clock under that load
+    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
+    mma = {form: pc.pc_probe_mma_rate(ctx, form, rounds=2000) for form in ("qk", "pv", "mix")}
+    assert pc.pc_poll_status(ctx) == pc.PC_OK
+
     # ---- the same frame through the three separate calls (pc_score, pc_compact, pc_attend_frame: eight launches)
     for i in range(3):
         step_separate(i)
@@ -545,6 +551,14 @@ def run_cuda(args):
                      "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
                      "flops_per_launch": flops, "ms_per_launch": att_ms, "ms_per_launch_single_kernel_span": att_span_ms,
                      "frac_by_single_kernel_span": flops / (att_span_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                     "mma_yardstick": {
+                         "cycles_per_mma": {k: round(v[0], 2) for k, v in mma.items()}, "sm_ghz_under_load": {k: round(v[1], 3) for k, v in mma.items()},
+                         "tflops_mix_never_waiting": 524288.0 * sm_count * mma["mix"][1] * 1e9 / mma["mix"][0] / 1e12,
+                         "frac_of_yardstick": achieved / (524288.0 * sm_count * mma["mix"][1] * 1e9 / mma["mix"][0] / 1e12),
+                         "what": "pc_probe_mma_rate: the kernel's own tcgen05.mma stream (Q K^T from shared memory, P V with P in "
+                                 "tensor memory, and both in the kernel's order) issued back to back on every SM with nothing else "
+                                 "running; 524,288 flop per multiply-add x SMs x clock / cycles is what the tensor cores deliver "
+                                 "to this instruction mix when they never wait"},
                      "how": "flops / the kernel's mean duration by CUDA events on the launching stream: the event mark in front "
                             "of the kernel left out, span of the pack kernel and this one minus the pack kernel's own span (the "
                             "duration as in the untimed step); the kernel runs inside a long power-capped step, for which the "

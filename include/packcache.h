@@ -414,6 +414,17 @@ pc_status pc_get_span(pc_ctx *ctx, int32_t mark_a, int32_t mark_b, float *ms);
  *   src device [n_rows][row_bytes]; out device [n_rows] uint32.  Errors: PC_ERR_INVALID_ARG, PC_ERR_CUDA. */
 pc_status pc_probe_stream_read(const void *src, int32_t n_rows, int32_t row_bytes, uint32_t *out, void *stream);
 
+/* Measurement support (the paper has no counterpart): the tensor-core issue stream of the attention kernel alone.  n_cta
+ * CTAs (one per SM; more than the GPU has SMs run in waves) each issue `rounds` rounds of the 128 x 128 x 16 bf16
+ * multiply-adds the attention kernel issues per key tile for its two query tiles — form 0: the Q K^T ones only (both
+ * operands in shared memory, 16 per round); form 1: the P V ones only (A in tensor memory, 16 per round); form 2: both in
+ * the kernel's order (32 per round) — on pseudo-random operands, two rounds in flight, and record the SM cycles and the
+ * global-timer nanoseconds the rounds took.  cycles / (rounds x multiply-adds per round) is what one multiply-add costs
+ * when the tensor core never waits; cycles / nanos is the SM clock under that load.  Waits are bounded like the
+ * attention kernel's (pc_set_wait_limit_us; a give-up shows in pc_poll_status).
+ *   cycles, nanos device [n_cta] int64.  Errors: PC_ERR_INVALID_ARG, PC_ERR_UNSUPPORTED, PC_ERR_CUDA. */
+pc_status pc_probe_mma_rate(pc_ctx *ctx, int32_t form, int32_t rounds, int32_t n_cta, int64_t *cycles, int64_t *nanos, void *stream);
+
 const char *pc_status_string(pc_status s);
 
 #ifdef __cplusplus

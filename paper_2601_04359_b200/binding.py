@@ -27,7 +27,7 @@ EXPORTS = ["pc_create", "pc_destroy", "pc_plan_budget", "pc_score", "pc_compact"
            "pc_window_create", "pc_window_destroy", "pc_window_append", "pc_window_append_masked", "pc_window_update", "pc_window_cache",
            "pc_window_state", "pc_attend_prepare", "pc_attend_prepared", "pc_attend_mass", "pc_frame_step",
            "pc_forget_anchors", "pc_set_wait_limit_us", "pc_test_expect_extra_bytes", "pc_window_step", "pc_window_step_host", "pc_set_timing_skip",
-           "pc_get_span", "pc_probe_stream_read"]
+           "pc_get_span", "pc_probe_stream_read", "pc_probe_mma_rate"]
 
 
 class pc_layer_desc(C.Structure):
@@ -117,6 +117,7 @@ def load() -> C.CDLL:
     lib.pc_set_timing_skip.argtypes = [C.c_void_p, C.c_uint32]
     lib.pc_get_span.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_float)]
     lib.pc_probe_stream_read.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+    lib.pc_probe_mma_rate.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.pc_frame_step_host.argtypes = [C.c_void_p, C.POINTER(pc_host_frame), C.POINTER(pc_device_workspace),
                                        C.POINTER(pc_budget_params), C.c_int32, C.c_void_p]
     lib.pc_score_tokens_static.argtypes = [C.POINTER(pc_layer_desc), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
@@ -388,6 +389,23 @@ def pc_probe_stream_read(rows: torch.Tensor, out: torch.Tensor, stream=None) -> 
     n = rows.shape[0]
     row_bytes = rows[0].numel() * rows.element_size()
     _check(load().pc_probe_stream_read(_ptr(rows), n, row_bytes, _ptr(out), _stream(stream)), "pc_probe_stream_read")
+
+
+MMA_FORMS = {"qk": (0, 16), "pv": (1, 16), "mix": (2, 32)}   # form id, multiply-adds per round
+
+
+def pc_probe_mma_rate(ctx: Context, form: str, rounds: int = 2000, n_cta: int | None = None, stream=None):
+    """The attention kernel's tensor-core issue stream alone (form "qk", "pv" or "mix").  Returns (cycles per multiply-add,
+    SM clock in GHz), each the median over the CTAs (one per SM unless n_cta says otherwise).  Synchronises."""
+    fid, per_round = MMA_FORMS[form]
+    if n_cta is None:
+        n_cta = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    cycles = torch.zeros(n_cta, dtype=torch.int64, device="cuda")
+    nanos = torch.zeros(n_cta, dtype=torch.int64, device="cuda")
+    _check(load().pc_probe_mma_rate(ctx.handle, fid, rounds, n_cta, _ptr(cycles), _ptr(nanos), _stream(stream)), "pc_probe_mma_rate")
+    torch.cuda.synchronize()
+    c, n = cycles.double(), nanos.double().clamp(min=1.0)
+    return float((c / (rounds * per_round)).median()), float((c / n).median())
 
 
 def pc_frame_step_host(ctx: Context, host: dict, ws_src: Cache, ws_dst: Cache, ws: dict, kind: int, param: float,

@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libpackcache.so")
 SOURCES = ["pc_api.cu", "pc_score.cu", "pc_pack.cu", "pc_attend.cu", "pc_attend_simt.cu", "pc_attend_tc.cu",
-           "pc_mass.cu", "pc_host_step.cu", "pc_window.cu", "pc_probe.cu"]
+           "pc_mass.cu", "pc_host_step.cu", "pc_window.cu", "pc_probe.cu", "pc_probe_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",
               "-I", INCLUDE, "-I", CSRC]
