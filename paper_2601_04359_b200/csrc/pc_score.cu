@@ -329,7 +329,7 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
 #define PC_QPREP_CASE(CPW)                                                                                           \
     {                                                                                                               \
         static int smem_of[PC_MAX_DEVICES] = {};                      /* largest dynamic size allowed so far */      \
-        if (q_smem > 48 * 1024 && smem_of[dev_id] < q_smem) {                                                       \
+        if (q_smem + 1024 > 48 * 1024 && smem_of[dev_id] < q_smem) {   /* the block's static words count, too */    \
             PC_CUDA_TRY(cudaFuncSetAttribute(k_qprep<T, CPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, q_smem)); \
             smem_of[dev_id] = q_smem;                                                                               \
         }                                                                                                           \

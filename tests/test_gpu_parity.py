@@ -367,6 +367,24 @@ def test_score_valid_mask_and_pooling_at_scale():
     ctx.close()
 
 
+@pytest.mark.parametrize("heads", [(96, 8), (48, 16), (32, 8)])
+def test_score_with_wide_query_rows(heads):
+    """The query pass keeps a token's rotated row in shared memory as fp32: 96 heads x 128 is exactly 48 KB, the most a
+    launch gets without asking for more (the block's own static words come on top); 48 and 32 heads sit below."""
+    from dataclasses import replace
+    cfg = replace(wl.small_bf16(n_frames=2, grid=(5, 7), n_text=20, total=30, keep_full=0, seed=41), n_q_heads=heads[0], n_kv_heads=heads[1])
+    L = wl.make_layer(cfg)
+    D = DeviceLayer(L)
+    ctx = make_ctx(cfg)
+    budget = _plan(cfg)
+    scores, sel = pc.pc_score(ctx, D.cache, D.q, D.q_pos, budget)
+    _ok(ctx)
+    ref = oracle.score(L.hist_k, L.hist_pos, L.q, L.q_pos, cfg.rope_base)
+    assert (np.abs(host(scores)[:cfg.n_src].astype(np.float64) - ref) <= score_tolerance(ref, L.frame_count)).all()
+    _valid_topk(host(scores)[:cfg.n_src], sel.cpu().numpy()[:budget.sum()], L.frame_count, budget)
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------------- errors
 def test_host_detected_errors():
     cfg = wl.CONFIGS["tiny"]
