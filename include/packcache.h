@@ -103,6 +103,10 @@ typedef struct {
 /* Create / destroy a context on the current CUDA device.  Builds the rotary
  * cos/sin tables (Sec. 3.1: pair i of d/2 turns with axis i mod 3 at frequency
  * base^(-(i div 3)/n_axis)) and allocates scratch for max_q / max_keys.
+ * Shapes: head_dim 64 or 128; n_q_heads a multiple of n_kv_heads; at most 4096 elements in a key row over all KV heads.
+ * Scoring (pc_score, pc_frame_step, the cache window) further needs a key row (n_kv_heads * head_dim elements of the
+ * dtype) of 512, 1024, 1536, 2048, 3072 or 4096 bytes and a query row that is a multiple of 512 bytes, and returns
+ * PC_ERR_UNSUPPORTED otherwise, before anything is enqueued; pc_compact and pc_attend_frame take any accepted shape.
  * Errors: PC_ERR_UNSUPPORTED, PC_ERR_INVALID_ARG, PC_ERR_CUDA. */
 pc_status pc_create(const pc_layer_desc *desc, pc_ctx **out);
 pc_status pc_destroy(pc_ctx *ctx);

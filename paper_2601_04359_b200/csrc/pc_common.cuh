@@ -255,6 +255,7 @@ pc_status pc_launch_pack(pc_ctx *ctx, const void *src_k, const void *src_v, cons
                          cudaStream_t stream);
 // pc_score / pc_compact with the extras of the fused frame step: q_rot_out (NULL or the context's rotated-query scratch,
 // filled by the query pass that also pools), k_rot_dst (as pc_launch_pack)
+bool pc_score_supports(const pc_layer_desc &D);   // the row widths the query pass and the scoring kernel take
 pc_status pc_score_impl(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q, const int32_t *budget,
                         const uint8_t *valid, const float *scores_override, float *scores, int32_t *sel_idx, void *q_rot_out,
                         cudaStream_t stream);

@@ -172,7 +172,9 @@ pc_status pc_launch_pack(pc_ctx *ctx, const void *src_k, const void *src_v, cons
         switch (row_bytes) {
         case 512: PC_LAUNCH((k_pack_rot<1>), dim3(blocks2), dim3(PACK_THREADS), 0, stream, PC_PACK_ROT_ARGS); break;
         case 1024: PC_LAUNCH((k_pack_rot<2>), dim3(blocks2), dim3(PACK_THREADS), 0, stream, PC_PACK_ROT_ARGS); break;
+        case 1536: PC_LAUNCH((k_pack_rot<3>), dim3(blocks2), dim3(PACK_THREADS), 0, stream, PC_PACK_ROT_ARGS); break;
         case 2048: PC_LAUNCH((k_pack_rot<4>), dim3(blocks2), dim3(PACK_THREADS), 0, stream, PC_PACK_ROT_ARGS); break;
+        case 3072: PC_LAUNCH((k_pack_rot<6>), dim3(blocks2), dim3(PACK_THREADS), 0, stream, PC_PACK_ROT_ARGS); break;
         case 4096: PC_LAUNCH((k_pack_rot<8>), dim3(blocks2), dim3(PACK_THREADS), 0, stream, PC_PACK_ROT_ARGS); break;
         default: return PC_ERR_UNSUPPORTED;
         }

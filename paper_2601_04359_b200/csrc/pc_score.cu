@@ -374,6 +374,18 @@ pc_status enqueue_score(const pc_layer_desc &D, int sm_count, const pc_rope_dev 
 
 }  // namespace
 
+// The shapes the query pass and the scoring kernel are built for: a key row of 512, 1024, 1536, 2048, 3072 or 4096 bytes
+// over all KV heads, a query row that is a multiple of 512 bytes and splits into at most 32 warps' parts.
+bool pc_score_supports(const pc_layer_desc &D) {
+    const int elem = D.dtype == PC_BF16 ? 2 : 4, per = 16 / elem;
+    const int row = D.n_kv_heads * D.head_dim, q_row = D.n_q_heads * D.head_dim;
+    if (row % (32 * per) || q_row % (32 * per) || (32 * per) % D.head_dim) return false;
+    const int cpl = row / per / 32, qcpl = q_row / per / 32;
+    if (cpl != 1 && cpl != 2 && cpl != 3 && cpl != 4 && cpl != 6 && cpl != 8) return false;
+    const int cpw = qcpl % 3 == 0 ? 3 : (qcpl % 4 == 0 ? 4 : (qcpl % 2 == 0 ? 2 : 1));
+    return qcpl / cpw <= 32;
+}
+
 pc_status pc_score_impl(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q, const int32_t *budget,
                         const uint8_t *valid, const float *scores_override, float *scores, int32_t *sel_idx, void *q_rot_out,
                         cudaStream_t stream) {
@@ -403,6 +415,7 @@ pc_status pc_score_impl(pc_ctx *ctx, const pc_cache *src, const void *q, const i
             if (!q || !q_pos || n_q <= 0 || !scores) return PC_ERR_INVALID_ARG;
             if (!pc_aligned16(q) || !pc_aligned16(q_pos) || !pc_aligned16(scores)) return PC_ERR_INVALID_ARG;
             if (n_q > ctx->desc.max_q) return PC_ERR_CAPACITY;
+            if (!pc_score_supports(ctx->desc)) return PC_ERR_UNSUPPORTED;      // before anything is enqueued
             const size_t row = (size_t)ctx->desc.n_kv_heads * ctx->desc.head_dim;
             if (ctx->qpool_dirty) {          // an earlier call stopped between the query pass and the scoring kernel
                 PC_CUDA_TRY(cudaMemsetAsync(ctx->qpool_fx, 0, (PC_FX_REPLICAS * row + 1) * sizeof(long long), stream));

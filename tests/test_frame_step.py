@@ -7,6 +7,8 @@ anchors' rotated keys are kept from step to step), so the comparison covers thos
 runs with the anchors' keys kept from the first, a third one after the anchors changed in place."""
 from __future__ import annotations
 
+from dataclasses import replace
+
 import numpy as np
 import pytest
 import torch
@@ -40,6 +42,10 @@ CASES = {
                                          keep_full=0, seed=5),
     "several_tiles": lambda: wl.small_bf16(n_frames=4, grid=(12, 21), n_text=130, total=700, keep_full=1, seed=31),
     "no_anchors": lambda: wl.small_bf16(n_frames=3, grid=(9, 15), n_text=37, total=200, keep_full=0, seed=32),
+    # key rows of 1536, 3072 and 4096 bytes (6, 12 and 16 KV heads): the other widths the pack kernel rotates
+    "rows_1536": lambda: replace(wl.small_bf16(n_frames=2, grid=(7, 9), n_text=20, total=70, keep_full=0, seed=33), n_q_heads=12, n_kv_heads=6),
+    "rows_3072": lambda: replace(wl.small_bf16(n_frames=2, grid=(7, 9), n_text=20, total=70, keep_full=1, seed=34), n_q_heads=24, n_kv_heads=12),
+    "rows_4096": lambda: replace(wl.small_bf16(n_frames=2, grid=(7, 9), n_text=20, total=70, keep_full=0, seed=35), n_q_heads=32, n_kv_heads=16),
 }
 
 

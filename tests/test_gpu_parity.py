@@ -419,6 +419,18 @@ def test_host_detected_errors():
         pc.Context(5, 2, 64, pc.PC_F32, 10000.0, (8, 8, 8), 8, 8)
     with pytest.raises(pc.PackCacheError):
         pc.Context(4, 2, 48, pc.PC_F32, 10000.0, (8, 8, 8), 8, 8)
+    # key rows the scoring kernels are not built for are refused by the call, with nothing enqueued:
+    # 32 KV heads x 128 bf16 = 8192 bytes, 5 x 128 bf16 = 1280 bytes (not a multiple of 512), 1 x 128 bf16 = 256 bytes
+    for hq, hkv in [(32, 32), (5, 5), (2, 1)]:
+        odd = pc.Context(hq, hkv, 128, pc.PC_BF16, 10000.0, (64, 64, 64), 8, 64)
+        k = torch.zeros((16, hkv, 128), dtype=torch.bfloat16, device="cuda")
+        q = torch.zeros((8, hq, 128), dtype=torch.bfloat16, device="cuda")
+        pos = torch.zeros((16, 4), dtype=torch.int32, device="cuda")
+        cache = pc.Cache(pc.Segment.empty(), pc.Segment(k, k.clone(), pos, 16), [16])
+        with pytest.raises(pc.PackCacheError) as e:
+            pc.pc_score(odd, cache, q, pos[:8], np.array([4], np.int32))
+        assert e.value.status == pc.PC_ERR_UNSUPPORTED and pc.pc_poll_status(odd) == pc.PC_OK
+        odd.close()
     _ok(ctx)
 
 
