@@ -119,6 +119,10 @@ extern "C" pc_status pc_frame_step(pc_ctx *ctx, const pc_cache *src, const int32
         k_rot_dst = static_cast<char *>(ctx->k_rot) + (size_t)anchor_tiles * tile * row_bytes;
         ctx->prepared_n_seg = 0;                       // the scratch no longer holds a key set of pc_attend_prepare
     }
+    // what the pack stage would refuse (a destination that overlaps the source, a misaligned or missing buffer) is refused
+    // now, before the scoring stage enqueues anything
+    st = pc_compact_check(ctx, src, sel_idx, budget, dst, nullptr, nullptr);
+    if (st != PC_OK) return st;
     ctx->last_n_q = 0;
     ctx->q_rot_n = 0;
     st = pc_score_impl(ctx, src, q, q_pos, n_q, budget, nullptr, nullptr, scores, sel_idx, tc ? ctx->q_rot : nullptr, stream);

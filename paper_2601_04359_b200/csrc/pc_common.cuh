@@ -259,6 +259,8 @@ bool pc_score_supports(const pc_layer_desc &D);   // the row widths the query pa
 pc_status pc_score_impl(pc_ctx *ctx, const pc_cache *src, const void *q, const int32_t *q_pos, int32_t n_q, const int32_t *budget,
                         const uint8_t *valid, const float *scores_override, float *scores, int32_t *sel_idx, void *q_rot_out,
                         cudaStream_t stream);
+pc_status pc_compact_check(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget, const pc_cache *dst,
+                           int64_t *n_sel_out, int64_t *n_src_out);   // every host-side check of pc_compact_impl, nothing enqueued
 pc_status pc_compact_impl(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget, int32_t delta_t,
                           pc_cache *dst, void *k_rot_dst, cudaStream_t stream);
 // log2(e) / sqrt(d): folded into the rotated queries of the tensor-core attention kernel (its softmax runs in base 2)

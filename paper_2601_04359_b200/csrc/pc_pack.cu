@@ -116,8 +116,9 @@ bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
 
 }  // namespace
 
-pc_status pc_compact_impl(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget, int32_t delta_t,
-                          pc_cache *dst, void *k_rot_dst, cudaStream_t stream) {
+// Every host-side check of a compaction, nothing enqueued: n_sel / n_src out (either may be NULL).
+pc_status pc_compact_check(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget, const pc_cache *dst,
+                           int64_t *n_sel_out, int64_t *n_src_out) {
     if (!ctx || !src || !dst || !budget) return PC_ERR_INVALID_ARG;
     if (src->n_frames < 0 || (src->n_frames > 0 && !src->frame_count)) return PC_ERR_INVALID_ARG;
     pc_status st = pc_check_segment(&src->history, true);
@@ -131,6 +132,8 @@ pc_status pc_compact_impl(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_i
     }
     if (n_src != src->history.n_tokens) return PC_ERR_INVALID_ARG;
     if (n_sel > dst->history.capacity) return PC_ERR_CAPACITY;
+    if (n_sel_out) *n_sel_out = n_sel;
+    if (n_src_out) *n_src_out = n_src;
     if (n_sel == 0) return PC_OK;
     if (!sel_idx || !pc_aligned16(sel_idx)) return PC_ERR_INVALID_ARG;
     const pc_segment &D = dst->history;
@@ -142,6 +145,16 @@ pc_status pc_compact_impl(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_i
         overlaps(src->history.k, src_bytes, D.v, dst_bytes) || overlaps(src->history.v, src_bytes, D.k, dst_bytes) ||
         overlaps(src->history.pos, (size_t)n_src * 16, D.pos, (size_t)n_sel * 16))
         return PC_ERR_INVALID_ARG;
+    return PC_OK;
+}
+
+pc_status pc_compact_impl(pc_ctx *ctx, const pc_cache *src, const int32_t *sel_idx, const int32_t *budget, int32_t delta_t,
+                          pc_cache *dst, void *k_rot_dst, cudaStream_t stream) {
+    int64_t n_sel = 0, n_src = 0;
+    pc_status st = pc_compact_check(ctx, src, sel_idx, budget, dst, &n_sel, &n_src);
+    if (st != PC_OK) return st;
+    if (n_sel == 0) return PC_OK;
+    const pc_segment &D = dst->history;
     pc_mark(ctx, PC_MARK_PACK0, stream);
     st = pc_launch_pack(ctx, src->history.k, src->history.v, src->history.pos, sel_idx, (int)n_sel, (int)n_src, delta_t, D.k, D.v,
                         D.pos, k_rot_dst, stream);

@@ -158,7 +158,7 @@ def test_fused_step_at_the_benchmark_size_matches_the_separate_calls():
 
 def test_fused_step_rejects_bad_arguments_before_enqueueing_anything():
     """Host-detectable errors return at once: a destination that is too small, a null output, too many queries for
-    the context, a budget above a frame's tokens; none of them leaves a device-side status or touches the outputs."""
+    the context, a budget above a frame's tokens, a destination that overlaps the source; none of them leaves a device-side status or touches the outputs."""
     cfg = wl.small_bf16(n_frames=3, grid=(8, 9), total=100, seed=42)
     L = wl.make_layer(cfg)
     D = DeviceLayer(L)
@@ -187,9 +187,14 @@ def test_fused_step_rejects_bad_arguments_before_enqueueing_anything():
     st = lib.pc_frame_step(ctx.handle, C.byref(cs), bud.ctypes.data_as(C.POINTER(C.c_int32)), 0, C.byref(cd), D.q.data_ptr(),
                            D.q_pos.data_ptr(), cfg.n_q, None, None, None, None, None)          # no output buffer
     assert st == pc.PC_ERR_INVALID_ARG
+    # what only the pack stage would notice is refused before the scoring stage runs: a destination that is the source
+    scores = torch.full((cfg.n_src,), 5.0, dtype=torch.float32, device="cuda")
+    with pytest.raises(pc.PackCacheError) as e:
+        pc.pc_frame_step(ctx, D.cache, budget, 0, D.cache, D.q, D.q_pos, scores=scores, out=out)
+    assert e.value.status == pc.PC_ERR_INVALID_ARG
     torch.cuda.synchronize()
     assert pc.pc_poll_status(ctx) == pc.PC_OK and pc.pc_poll_status(tight) == pc.PC_OK
-    assert (out == 7.0).all() and (host(dst.history.k) == 3.0).all()
+    assert (out == 7.0).all() and (host(dst.history.k) == 3.0).all() and (scores == 5.0).all()
     ctx.close(); tight.close()
 
 
