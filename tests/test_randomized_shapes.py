@@ -21,6 +21,23 @@ HEADS = [(24, 8), (8, 8), (16, 4), (32, 8), (6, 2), (4, 2), (12, 4), (2, 2)]
 DECAY = {wl.HALFLIFE: 2.0, wl.LINEAR: 0.0, wl.GEOMETRIC: 0.6, wl.CLOSED_HALF: 0.5}
 
 
+def attention_within_bounds(got: np.ndarray, want: np.ndarray, want_abs: np.ndarray) -> bool:
+    """2e-2 wherever a bf16 result can meet it, and everywhere a bound made of what the arithmetic can add.  With a few
+    dozen keys and V's outlier channels a result can pass 4, where bf16 numbers are 2^-5 apart: storing it alone then costs
+    up to 1.6e-2 (seen: 4.1048 stored as 4.125), so the absolute bound is asked of results below 4 only.  Element-wise:
+    one bf16 spacing of the result (storing it), plus 2^-6 * sum_j p_j |v_j| (want_abs: the oracle's attention over |V|),
+    plus 1e-3.  The middle term: a probability reaches the tensor core with three bf16 roundings behind it, its own and
+    those of the rotated query and key (through the logit), 2^-9 relative each; over thousands of keys they cancel, over a
+    handful they do not.  Seen over 300 random cases: at most 2^-7.3 of the sum (3 to 12 keys), below 2^-8 from 30 keys on."""
+    from .test_gpu_parity import bf16_ulp
+    err = np.abs(got - want)
+    return bool((err[np.abs(want) < 4.0] <= 2e-2).all() and (err <= bf16_ulp(want) + 2.0 ** -6 * want_abs + 1e-3).all())
+
+
+def abs_v(segs):
+    return [(k, np.abs(v), p) for k, v, p in segs]
+
+
 @pytest.mark.parametrize("seed", [0, 1, 2, 3, 4])
 def test_random_shapes_against_the_oracle(seed):
     rng = np.random.default_rng(seed)
@@ -65,7 +82,7 @@ def test_random_shapes_against_the_oracle(seed):
         out, lse = pc.pc_attend_frame(ctx, dst, D.current if with_cur else None, D.q, D.q_pos, want_lse=True)
         want, want_lse = oracle.attend(L.q, L.q_pos, segs, cfg.rope_base, want_lse=True)
         assert pc.pc_poll_status(ctx) == pc.PC_OK, what
-        assert np.abs(host(out).astype(np.float64) - want).max() <= 2e-2, what
+        assert attention_within_bounds(host(out).astype(np.float64), want, oracle.attend(L.q, L.q_pos, abs_v(segs), cfg.rope_base)), what
         assert np.abs(host(lse) - want_lse).max() <= 2e-2, what
         if hkv * cfg.head_dim % 256 == 0 and impl == 0:
             n_keys = sum(len(s[0]) for s in segs)
@@ -124,7 +141,7 @@ def test_random_fused_steps_against_the_separate_calls_and_the_oracle(seed):
         wk, wv, wp = oracle.pack(L.hist_k, L.hist_v, L.hist_pos, sel_np, delta_t)
         segs = [s for s in [(L.anchor_k, L.anchor_v, L.anchor_pos), (wk, wv, wp)] if len(s[0])]
         want, want_lse = oracle.attend(L.q, L.q_pos, segs, cfg.rope_base, want_lse=True)
-        assert np.abs(host(out).astype(np.float64) - want).max() <= 2e-2, what
+        assert attention_within_bounds(host(out).astype(np.float64), want, oracle.attend(L.q, L.q_pos, abs_v(segs), cfg.rope_base)), what
         assert np.abs(host(lse) - want_lse).max() <= 2e-2, what
         ref_ctx.close(); ctx.close()
 
