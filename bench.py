@@ -167,6 +167,15 @@ def oracle_sample(cfg, layer, n_score: int, n_rows: int, s32=None):
     return total * 1e3, what
 
 
+def bench_config(cfg, n_sel: int, world: int) -> dict:
+    """The `config` object of the JSON line, the same for both arms (the reference arm runs the CUDA arm's configuration)."""
+    return {"workload": WORKLOAD, "n_frames": cfg.n_frames, "frame_tokens": cfg.frame_tokens,
+            "n_anchor": cfg.n_anchor, "retained": int(n_sel), "keys_attended": int(cfg.n_anchor + n_sel), "n_q": cfg.n_q,
+            "heads": f"{cfg.n_q_heads}q/{cfg.n_kv_heads}kv", "head_dim": cfg.head_dim,
+            "budget": "2 newest frames whole + 6048 at half-life 4", "mode": "one-shot compaction every frame",
+            "l2": f"inputs rotate over {N_LAYERS} layers (~{0.2 * N_LAYERS:.1f} GB; L2 is 126 MB)", "parallelism": f"replicas x{world}"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -189,8 +198,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": v, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "n_frames": cfg.n_frames, "frame_tokens": cfg.frame_tokens,
-                       "n_anchor": cfg.n_anchor, "retained": cfg.budget.total},
+            "config": bench_config(cfg, cfg.budget.total, max(args.gpus, 1)),
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -528,11 +536,7 @@ def run_cuda(args):
         "metric": METRIC, "value": ms_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "n_frames": cfg.n_frames, "frame_tokens": cfg.frame_tokens,
-                   "n_anchor": cfg.n_anchor, "retained": n_sel, "keys_attended": n_keys, "n_q": cfg.n_q,
-                   "heads": f"{cfg.n_q_heads}q/{cfg.n_kv_heads}kv", "head_dim": cfg.head_dim,
-                   "budget": "2 newest frames whole + 6048 at half-life 4", "mode": "one-shot compaction every frame",
-                   "l2": f"inputs rotate over {N_LAYERS} layers (~{0.2 * N_LAYERS:.1f} GB; L2 is 126 MB)", "parallelism": f"replicas x{world}"},
+        "config": bench_config(cfg, n_sel, world),
         "timed_regions": {"count": len(regions), "steps_each": args.steps, "median_ms_per_step": ms_step,
                           "min_ms_per_step": float(min(regions)), "max_ms_per_step": float(max(regions))},
         "replicas": {"frames_per_s": replica_frames_per_s(ms_step, world), "what": "every rank steps its own layers; per-frame latency is "
