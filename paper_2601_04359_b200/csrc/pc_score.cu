@@ -284,7 +284,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 2) k_score(const T *__restrict_
 // Select.  One block per frame runs the block-level selection of pc_select.cuh and writes the kept tokens' indices in
 // ascending order.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int SEL_THREADS = 512;
+constexpr int SEL_THREADS = 1024;
 
 __global__ void __launch_bounds__(SEL_THREADS) k_select(const float *__restrict__ scores, const __grid_constant__ FrameTab tab,
                                                        int32_t *__restrict__ sel_idx, int32_t *status) {
